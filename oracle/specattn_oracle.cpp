@@ -1,0 +1,325 @@
+// SpecAttn verification hot path -- CPU ORACLE.
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the plain, slow, obviously-correct
+// statement of what the hot path computes.  It shares no code, header, table
+// or helper with the CUDA library and must never be called from the product
+// path: only the tests, the smoke check and the benchmark's CPU-baseline leg
+// may load it.
+//
+// What it states (paper passages in brackets):
+//   O1  aggregate   a_bar[i] = sum over draft heads h and speculated queries s
+//                   of A[h,s,i]                        [Sec. 3.4 item 1: one row
+//                   a_{f(j)} per verifier layer; Alg. 1 "Sparse Attention Mask
+//                   Creation": one token set per layer from the gamma maps]
+//   O2  nucleus     the smallest largest-first prefix whose mass reaches
+//                   p * sum(a_bar), ties at the threshold all kept
+//                                                      [App. A Eq. 7; Alg. 2:
+//                   target mass p*sum(a), membership test a_i >= theta]
+//   O3  attention   softmax(q K^T / sqrt(d)) V restricted to the kept set
+//                                                      [Eq. 1 restricted to the
+//                   index set I of Eq. 2-3; normalised over I]
+//
+// Arithmetic: O1 is a chain of IEEE binary32 additions in a fixed order (this
+// defines the aggregated value bit for bit); every mass in O2 and everything
+// in O3 is binary64.  Compile WITHOUT fast-math and with -ffp-contract=off.
+//
+// Parity pins (tests/test_oracle_pins.py): worked rows with exact dyadic
+// sums, brute-force subset enumeration, Alg. 2 bisection run to convergence,
+// closed forms, monotonicity / permutation / scaling invariants for O2; a
+// dense fp64 library softmax-attention, single-token, zero-key and LSE-merge
+// identities and the App. A error bound for O3; an order-sensitive fp32 sum
+// for O1.  No function here is "parity unpinned".
+
+#include <algorithm>
+#include <cfloat>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <numeric>
+#include <vector>
+
+#if defined(_OPENMP)
+#include <omp.h>
+#endif
+
+namespace {
+
+inline double bf16_bits_to_double(uint16_t h) {
+  uint32_t u = static_cast<uint32_t>(h) << 16;
+  float f;
+  std::memcpy(&f, &u, sizeof(f));
+  return static_cast<double>(f);
+}
+
+// A probability is valid when it is a finite number >= 0 (-0.0 counts as 0).
+inline bool valid_prob(float x) { return (x >= 0.0f) && (x <= FLT_MAX); }
+
+}  // namespace
+
+extern "C" {
+
+enum {
+  ORACLE_OK = 0,
+  ORACLE_INVALID_PROB = 1,
+  ORACLE_OVERFLOW = 2,
+};
+
+int specattn_oracle_num_threads(void) {
+#if defined(_OPENMP)
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+// ---------------------------------------------------------------------------
+// O1.  Aggregated draft attention row for one (draft layer, sequence, group).
+//   A          [n_heads, gamma, L_stride] binary32, position contiguous
+//   head_group NULL: every head feeds the row; else only heads with
+//              head_group[h] == g
+//   a_bar      [L] output
+// Order of the binary32 additions: start from +0, heads ascending, inside a
+// head the speculated queries ascending.  Returns ORACLE_INVALID_PROB if any
+// contributing input is negative, NaN or infinite (the row is still written).
+// [Sec. 3.4 item 1; Alg. 1 "Sparse Attention Mask Creation"]
+// ---------------------------------------------------------------------------
+int specattn_oracle_aggregate(const float* A, int n_heads, int gamma, int64_t L_stride, int L,
+                              const int32_t* head_group, int g, float* a_bar) {
+  int status = ORACLE_OK;
+  for (int i = 0; i < L; ++i) {
+    float acc = 0.0f;
+    for (int h = 0; h < n_heads; ++h) {
+      if (head_group != nullptr && head_group[h] != g) continue;
+      for (int s = 0; s < gamma; ++s) {
+        const float x = A[(static_cast<int64_t>(h) * gamma + s) * L_stride + i];
+        if (!valid_prob(x)) status = ORACLE_INVALID_PROB;
+        acc = acc + x;
+      }
+    }
+    a_bar[i] = acc;
+  }
+  return status;
+}
+
+// ---------------------------------------------------------------------------
+// O2.  Top-p nucleus of one non-negative row by explicit full sort.
+//   total  = sum_i (double) a[i], index order
+//   p >= 1: every position is kept (a rule, not arithmetic)
+//   else    target = (double) p * total; positions sorted by value descending
+//           (index ascending among equals); C_k = running binary64 sum in that
+//           order; k* = min{k : C_k >= target}; theta = value of the k*-th;
+//           kept = {i : a[i] >= theta}, emitted in ascending position.
+//   diag[0..5] = total, target, M_gt (mass strictly above theta),
+//                M_ge (mass of the kept set), margin, theta
+//   margin = min(M_ge - target, target - M_gt) / total  (1 when total == 0 or
+//            p >= 1): how far the decision is from flipping.
+// Writes at most idx_cap positions; returns the true kept count.
+// [App. A Eq. 7; Alg. 2 lines "M_target <- p * sum a" and "T_s <- {i: a_i >= theta}"]
+// ---------------------------------------------------------------------------
+int64_t specattn_oracle_nucleus(const float* a, int L, float p, int32_t* idx, int64_t idx_cap,
+                                double* diag) {
+  double total = 0.0;
+  for (int i = 0; i < L; ++i) total += static_cast<double>(a[i]);
+  double target = static_cast<double>(p) * total;
+  double m_gt = 0.0, m_ge = total, margin = 1.0, theta = 0.0;
+  int64_t count = 0;
+
+  if (L > 0 && !(p >= 1.0f)) {
+    std::vector<int32_t> order(L);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(),
+                     [a](int32_t x, int32_t y) { return a[x] > a[y]; });
+    double c = 0.0;
+    int k_star = L;  // 1-based length of the prefix
+    std::vector<double> prefix(L);
+    for (int k = 0; k < L; ++k) {
+      c += static_cast<double>(a[order[k]]);
+      prefix[k] = c;
+      if (c >= target) {
+        k_star = k + 1;
+        break;
+      }
+    }
+    const float th = a[order[k_star - 1]];
+    theta = static_cast<double>(th);
+    // first position of the tie group in sorted order
+    int first = k_star - 1;
+    while (first > 0 && a[order[first - 1]] == th) --first;
+    m_gt = (first > 0) ? prefix[first - 1] : 0.0;
+    // extend the running sum to the end of the tie group
+    int last = k_star;  // exclusive
+    double cg = prefix[k_star - 1];
+    while (last < L && a[order[last]] == th) {
+      cg += static_cast<double>(a[order[last]]);
+      ++last;
+    }
+    m_ge = cg;
+    margin = (total > 0.0) ? std::min(m_ge - target, target - m_gt) / total : 1.0;
+    for (int i = 0; i < L; ++i) {
+      if (a[i] >= th) {
+        if (count < idx_cap) idx[count] = i;
+        ++count;
+      }
+    }
+  } else {
+    for (int i = 0; i < L; ++i) {
+      if (count < idx_cap) idx[count] = i;
+      ++count;
+    }
+    theta = 0.0;
+  }
+  if (diag != nullptr) {
+    diag[0] = total;
+    diag[1] = target;
+    diag[2] = m_gt;
+    diag[3] = m_ge;
+    diag[4] = margin;
+    diag[5] = theta;
+  }
+  return count;
+}
+
+// ---------------------------------------------------------------------------
+// O1 + O2 over a whole step: every draft layer that some target layer maps to,
+// every sequence, every group.
+//   draft_probs[u]  [B, n_heads, gamma, L_stride] binary32 (NULL allowed for
+//                   draft layers no target layer maps to)
+//   layer_map       [n_target_layers] in [-1, n_draft_layers); -1 = dense layer
+//   idx             [n_draft_layers, B, G, idx_stride]   ascending positions
+//   counts, status  [n_draft_layers, B, G]
+//   diag            [n_draft_layers, B, G, 6] or NULL (see specattn_oracle_nucleus)
+// A row with an invalid probability gets status INVALID_PROB and count 0.  A
+// list longer than idx_stride is cut to its first idx_stride positions, keeps
+// its true count and gets OVERFLOW.  Lists of unmapped draft layers are left
+// untouched.                                  [Alg. 1 lines "i* <- f(j)", "T_j <- ..."]
+// ---------------------------------------------------------------------------
+void specattn_oracle_select_topp(const float* const* draft_probs, int n_draft_layers,
+                                 const int32_t* layer_map, int n_target_layers, int B, int n_heads,
+                                 int gamma, int G, int64_t L_stride, const int32_t* kv_len,
+                                 const int32_t* head_group, float p, int32_t* idx,
+                                 int64_t idx_stride, int32_t* counts, int32_t* status,
+                                 double* diag) {
+  std::vector<char> used(n_draft_layers, 0);
+  for (int j = 0; j < n_target_layers; ++j)
+    if (layer_map[j] >= 0 && layer_map[j] < n_draft_layers) used[layer_map[j]] = 1;
+  const int64_t n_lists = static_cast<int64_t>(n_draft_layers) * B * G;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t li = 0; li < n_lists; ++li) {
+    const int u = static_cast<int>(li / (static_cast<int64_t>(B) * G));
+    const int b = static_cast<int>((li / G) % B);
+    const int g = static_cast<int>(li % G);
+    if (!used[u]) continue;
+    const int L = kv_len[b];
+    std::vector<float> a_bar(std::max(L, 1));
+    const float* A = draft_probs[u] + static_cast<int64_t>(b) * n_heads * gamma * L_stride;
+    int st = specattn_oracle_aggregate(A, n_heads, gamma, L_stride, L, head_group, g,
+                                       a_bar.data());
+    double* dg = diag ? diag + li * 6 : nullptr;
+    if (st == ORACLE_INVALID_PROB) {
+      counts[li] = 0;
+      status[li] = ORACLE_INVALID_PROB;
+      if (dg) for (int k = 0; k < 6; ++k) dg[k] = std::numeric_limits<double>::quiet_NaN();
+      continue;
+    }
+    int64_t c = specattn_oracle_nucleus(a_bar.data(), L, p, idx + li * idx_stride, idx_stride, dg);
+    counts[li] = static_cast<int32_t>(c);
+    status[li] = (c > idx_stride) ? ORACLE_OVERFLOW : ORACLE_OK;
+  }
+}
+
+// ---------------------------------------------------------------------------
+// O3 core.  Softmax attention of M query rows over c gathered key/value rows.
+//   q  [M, d] bf16 bits, K and V [c, d] bf16 bits (row stride given in elements)
+//   s_i = (q . k_i) * scale ; m = max_i s_i ; l = sum_i exp(s_i - m)
+//   out[r, :] = sum_i exp(s_i - m) v_i / l ;  lse[r] = m + ln l   (natural log)
+//   c == 0: out = 0, lse = -inf.
+// [Eq. 1, restricted to the selected set I of Eq. 2-3 and normalised over I]
+// ---------------------------------------------------------------------------
+void specattn_oracle_attend_rows(const uint16_t* q, int64_t q_stride, const uint16_t* K,
+                                 int64_t k_stride, const uint16_t* V, int64_t v_stride, int M,
+                                 int64_t c, int d, double scale, double* out, double* lse) {
+  std::vector<double> s(std::max<int64_t>(c, 1));
+  for (int r = 0; r < M; ++r) {
+    double* o = out + static_cast<int64_t>(r) * d;
+    for (int e = 0; e < d; ++e) o[e] = 0.0;
+    if (c == 0) {
+      lse[r] = -std::numeric_limits<double>::infinity();
+      continue;
+    }
+    double m = -std::numeric_limits<double>::infinity();
+    for (int64_t i = 0; i < c; ++i) {
+      double dot = 0.0;
+      for (int e = 0; e < d; ++e)
+        dot += bf16_bits_to_double(q[r * q_stride + e]) * bf16_bits_to_double(K[i * k_stride + e]);
+      s[i] = dot * scale;
+      m = std::max(m, s[i]);
+    }
+    double l = 0.0;
+    for (int64_t i = 0; i < c; ++i) l += std::exp(s[i] - m);
+    for (int64_t i = 0; i < c; ++i) {
+      const double w = std::exp(s[i] - m) / l;
+      for (int e = 0; e < d; ++e) o[e] += w * bf16_bits_to_double(V[i * v_stride + e]);
+    }
+    lse[r] = m + std::log(l);
+  }
+}
+
+// ---------------------------------------------------------------------------
+// O3 over one target layer of a paged cache.
+//   q          [B, T, H_q, d] bf16 bits
+//   kv_pages   bf16 bits; element (page, kv, slot, head, e) at
+//              page*stride_page + kv*stride_kv + slot*stride_slot + head*stride_head + e
+//              (kv = 0 keys, 1 values)
+//   block_table[b*bt_stride + i/page_size] = page of position i; NULL = the
+//              cache is contiguous: position i of sequence b is at page
+//              b*ceil(max_len/page_size)+i/page_size with max_len = bt_stride
+//              (bt_stride is then read as "pages per sequence")
+//   idx/counts the lists of ONE draft layer: [B, G, idx_stride], [B, G];
+//              dense != 0: every position < kv_len[b] is attended, lists unread
+//   query head h uses kv head h / (H_q/H_kv) and list g = (G == 1 ? 0 : kv head)
+//   out [B, T, H_q, d] and lse [B, T, H_q] binary64.
+// All T queries and all heads of a group share one list.
+// [Alg. 1 "Verification with Sparse Attention": one mask per layer for the
+//  gamma+1 verifier predictions; Eq. 1-3]
+// ---------------------------------------------------------------------------
+void specattn_oracle_sparse_verify(int B, int T, int Hq, int Hkv, int d, int page_size, int G,
+                                   const uint16_t* q, const uint16_t* kv_pages, int64_t stride_page,
+                                   int64_t stride_kv, int64_t stride_slot, int64_t stride_head,
+                                   const int32_t* block_table, int64_t bt_stride,
+                                   const int32_t* kv_len, const int32_t* idx, int64_t idx_stride,
+                                   const int32_t* counts, int dense, double scale, double* out,
+                                   double* lse) {
+  const int grp = Hq / Hkv;
+  if (scale == 0.0) scale = 1.0 / std::sqrt(static_cast<double>(d));
+  const int64_t n_units = static_cast<int64_t>(B) * Hkv;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t unit = 0; unit < n_units; ++unit) {
+    const int b = static_cast<int>(unit / Hkv);
+    const int hk = static_cast<int>(unit % Hkv);
+    const int g = (G == 1) ? 0 : hk;
+    const int64_t li = static_cast<int64_t>(b) * G + g;
+    const int64_t c = dense ? kv_len[b] : std::min<int64_t>(counts[li], idx_stride);
+    std::vector<uint16_t> Kr(std::max<int64_t>(c, 1) * d), Vr(std::max<int64_t>(c, 1) * d);
+    for (int64_t k = 0; k < c; ++k) {
+      const int64_t pos = dense ? k : idx[li * idx_stride + k];
+      const int64_t logical_page = pos / page_size;
+      const int64_t page = block_table ? block_table[b * bt_stride + logical_page]
+                                       : b * bt_stride + logical_page;
+      const int64_t slot = pos % page_size;
+      const uint16_t* base = kv_pages + page * stride_page + slot * stride_slot + hk * stride_head;
+      std::memcpy(&Kr[k * d], base, sizeof(uint16_t) * d);
+      std::memcpy(&Vr[k * d], base + stride_kv, sizeof(uint16_t) * d);
+    }
+    for (int t = 0; t < T; ++t) {
+      for (int hh = 0; hh < grp; ++hh) {
+        const int h = hk * grp + hh;
+        const int64_t row = (static_cast<int64_t>(b) * T + t) * Hq + h;
+        specattn_oracle_attend_rows(q + row * d, d, Kr.data(), d, Vr.data(), d, 1, c, d, scale,
+                                    out + row * d, lse + row);
+      }
+    }
+  }
+}
+
+}  // extern "C"
