@@ -1,0 +1,229 @@
+/* specattn.h -- C ABI of the SpecAttn verification hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, as hand-written CUDA kernels, the per-step work that the SpecAttn
+ * verifier performs for each of its layers:
+ *
+ *   select:  sum the mapped draft layer's attention probabilities over draft heads and the
+ *            gamma speculated queries, find the exact top-p nucleus of context positions
+ *            without sorting (a radix threshold search over the binary32 bit pattern with
+ *            per-bin counts and masses) and emit the kept positions as ascending index lists.
+ *   verify:  grouped-query sparse decode attention of the gamma+1 verification queries over
+ *            only the listed rows of a paged bf16 K/V cache, returning outputs and LSE.
+ *
+ * Conventions common to every entry point
+ *   - Pointers are DEVICE pointers unless the comment says HOST.  The caller owns every
+ *     buffer; the library never allocates or frees device memory and never synchronises.
+ *     Work is enqueued on the CUDA stream passed as `cuda_stream` (a cudaStream_t cast to
+ *     void*; NULL = the legacy default stream) and is complete when that stream reaches it.
+ *   - Return value: SPECATTN_OK (0) = enqueued; a negative SPECATTN_ERR_* = argument error
+ *     detected on the host, nothing was launched.  Data-dependent problems are reported per
+ *     list / per sequence in device status words as SPECATTN_ROW_* bit flags; the device
+ *     code never traps.
+ *   - `struct_size` must be sizeof() of the struct the caller was compiled against.
+ *   - Strides are in ELEMENTS of the array they index.
+ */
+#ifndef SPECATTN_H_
+#define SPECATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- host-side return codes ------------------------------------------------------------ */
+#define SPECATTN_OK 0
+#define SPECATTN_ERR_NULL (-1)        /* a required pointer is NULL */
+#define SPECATTN_ERR_STRUCT_SIZE (-2) /* struct_size does not match this library */
+#define SPECATTN_ERR_RANGE (-3)       /* a scalar is outside its documented range */
+#define SPECATTN_ERR_ALIGN (-4)       /* a pointer or stride breaks the 16-byte rules */
+#define SPECATTN_ERR_WORKSPACE (-5)   /* workspace missing or smaller than *_workspace_bytes() */
+#define SPECATTN_ERR_UNSUPPORTED (-6) /* shape outside what the kernels are built for */
+#define SPECATTN_ERR_CUDA (-7)        /* the CUDA runtime refused the launch */
+
+/* ---- device-side per-list / per-sequence status flags ---------------------------------- */
+#define SPECATTN_ROW_OK 0
+#define SPECATTN_ROW_INVALID_PROB 1 /* a contributing probability was negative, NaN or Inf */
+#define SPECATTN_ROW_OVERFLOW 2     /* the list has more entries than idx_stride; truncated */
+#define SPECATTN_ROW_BAD_INDEX 4    /* verify met a position or page id out of range */
+#define SPECATTN_ROW_TIMEOUT 8      /* a bounded device-side wait ran out; outputs invalid */
+
+/* ---- limits ---------------------------------------------------------------------------- */
+#define SPECATTN_MAX_DRAFT_LAYERS 64
+#define SPECATTN_MAX_DRAFT_HEADS 256
+#define SPECATTN_MAX_ROWS_PER_LIST 1024  /* contributing (head, query) rows per list */
+#define SPECATTN_MAX_KV_LEN 327680       /* positions per sequence for select (8 x 40960) */
+#define SPECATTN_MAX_VERIFY_UNITS 2048   /* batch * n_kv_heads for verify */
+#define SPECATTN_MAX_QUERY_ROWS 64       /* n_q * (n_q_heads / n_kv_heads) for verify */
+
+/* ========================================================================================
+ * specattn_select_topp -- token selection.
+ *
+ * Paper: Sec. 3.4 ("Sorting-Free Top-p Nucleus Selection"), Alg. 2, and the top-p objective
+ * of App. A Eq. 7; the per-layer use is Alg. 1, block "Sparse Attention Mask Creation".
+ *
+ * For every draft layer u that some target layer maps to (layer_map[j] == u), every sequence
+ * b and every group g:
+ *   a_bar[i] = +0 + sum over heads h feeding g (ascending) of sum over s < gamma (ascending)
+ *              of draft_probs[u][b, h, s, i],   i < kv_len[b]        (binary32 adds, this order)
+ *   total    = sum_i a_bar[i];  target = (double) p * total            (Alg. 2: p * sum a)
+ *   theta    = the largest row value v whose mass {a_bar >= v} reaches target -- the fixed
+ *              point of Alg. 2's bisection, identical to the sorted-prefix nucleus of Eq. 7
+ *   list     = ascending { i : a_bar[i] >= theta }  (ties at theta all kept)
+ *   p >= 1 keeps every position; an all-zero row keeps every position.
+ * Draft layers no target layer maps to are skipped and their outputs left untouched.
+ *
+ * Outputs per (u, b, g), all indexed [n_draft_layers, batch, n_groups]:
+ *   idx     int32 [.., idx_stride]: the list, first min(count, idx_stride) entries
+ *   counts  int32: the true list length (also when it exceeds idx_stride)
+ *   row_status int32: SPECATTN_ROW_* flags.  INVALID_PROB => count 0, list unspecified.
+ *   diag    optional double [.., 4] = {total, target, mass strictly above theta,
+ *           mass of the kept set}; NULL to skip.
+ *
+ * Requirements: 1 <= n_draft_layers <= 64; n_draft_heads <= 256; gamma >= 1; L_stride a
+ * multiple of 4 and <= SPECATTN_MAX_KV_LEN; every draft_probs[u] 16-byte aligned;
+ * 0 <= kv_len[b] <= L_stride (larger values are clamped); 0 < p (NaN rejected);
+ * n_groups >= 1; head_group (HOST, may be NULL = every head feeds every group) values in
+ * [0, n_groups).  No workspace is needed: each list is held in the shared memory of one
+ * thread-block cluster.
+ * ======================================================================================== */
+typedef struct specattn_select_args {
+  uint32_t struct_size;
+  int32_t n_draft_layers;
+  int32_t n_target_layers;
+  int32_t batch;
+  int32_t n_draft_heads;
+  int32_t gamma;
+  int32_t n_groups;
+  int64_t L_stride;
+  const float* const* draft_probs; /* HOST array [n_draft_layers] of device pointers to
+                                      binary32 [batch, n_draft_heads, gamma, L_stride];
+                                      entries of unmapped layers may be NULL */
+  const int32_t* kv_len;           /* [batch] */
+  const int32_t* layer_map;        /* HOST [n_target_layers], values in [-1, n_draft_layers);
+                                      -1 marks a dense target layer */
+  const int32_t* head_group;       /* HOST [n_draft_heads] or NULL */
+  float p;
+  int32_t* idx;
+  int64_t idx_stride;
+  int32_t* counts;
+  int32_t* row_status;
+  double* diag;
+} specattn_select_args;
+
+int specattn_select_topp(const specattn_select_args* args, void* cuda_stream);
+
+/* ========================================================================================
+ * specattn_sparse_verify -- sparse attention of one target layer.
+ *
+ * Paper: Eq. 1 restricted to the selected index set I of Eq. 2-3 (softmax normalised over I;
+ * the un-normalised form of Eq. 2 is out * exp(lse - lse_dense)); Sec. 3.5; Alg. 1, block
+ * "Verification with Sparse Attention" (one list per layer shared by all gamma+1 queries).
+ *
+ * For sequence b, query t < n_q and query head h (kv head hk = h / (n_q_heads/n_kv_heads),
+ * list g = 0 if n_groups == 1 else hk):
+ *   s_i = sm_scale * q[b,t,h,:] . K[i, hk, :]  for i in the list;  m = max s_i
+ *   out[b,t,h,:] = sum_i exp(s_i - m) V[i, hk, :] / sum_i exp(s_i - m)
+ *   lse[b,t,h]   = m + ln sum_i exp(s_i - m)          (natural log)
+ * An empty list gives out = 0, lse = -inf.  Position i of sequence b lives in page
+ * block_table[b * block_table_stride + i / page_size] at slot i % page_size; with
+ * block_table == NULL the cache is contiguous and that page is
+ * b * block_table_stride + i / page_size (block_table_stride = pages per sequence).
+ * Element (page, kv, slot, head, e) of kv_pages is at
+ *   page*stride_page + kv*stride_kv + slot*stride_slot + head*stride_head + e,
+ * kv = 0 for keys and 1 for values.
+ *
+ * idx / counts point at the lists of ONE draft layer: idx [batch, n_groups, idx_stride],
+ * counts [batch, n_groups] (entries beyond idx_stride are ignored).  dense != 0 attends every
+ * position below kv_len[b] and reads neither idx nor counts (both may be NULL).
+ *
+ * Requirements: head_dim == 128; n_q * (n_q_heads / n_kv_heads) <= 64; batch * n_kv_heads
+ * <= 2048; q, kv_pages 16-byte aligned and all four strides multiples of 8; out 16-byte
+ * aligned.  status (int32 [batch], optional) receives SPECATTN_ROW_BAD_INDEX when a listed
+ * position is outside [0, kv_len[b]) or a page id outside [0, n_pages) (such entries are
+ * read from position 0 / page 0 instead; n_pages == 0 disables the page check).
+ *
+ * workspace: at least specattn_verify_workspace_bytes() bytes, 256-byte aligned, prepared
+ * once with specattn_verify_workspace_init() and then reusable by consecutive calls on the
+ * same stream; two calls that may overlap on the GPU need separate workspaces.
+ * ======================================================================================== */
+typedef struct specattn_verify_args {
+  uint32_t struct_size;
+  int32_t batch;
+  int32_t n_q;
+  int32_t n_q_heads;
+  int32_t n_kv_heads;
+  int32_t head_dim;
+  int32_t page_size;
+  int32_t n_groups;
+  int32_t dense;
+  const void* q;        /* bf16 [batch, n_q, n_q_heads, head_dim] */
+  const void* kv_pages; /* bf16 pool of this target layer */
+  int64_t n_pages;
+  int64_t stride_page, stride_kv, stride_slot, stride_head;
+  const int32_t* block_table;
+  int64_t block_table_stride;
+  const int32_t* kv_len; /* [batch] */
+  const int32_t* idx;
+  int64_t idx_stride;
+  const int32_t* counts;
+  float sm_scale;        /* 0 => 1/sqrt(head_dim) */
+  float* out;            /* binary32 [batch, n_q, n_q_heads, head_dim] */
+  float* lse;            /* binary32 [batch, n_q, n_q_heads] */
+  int32_t* status;       /* [batch] or NULL */
+  void* workspace;
+  size_t workspace_bytes;
+} specattn_verify_args;
+
+/* Bytes of workspace specattn_sparse_verify needs for these shapes on the current device
+ * (0 on argument error).  Depends only on the scalar fields. */
+size_t specattn_verify_workspace_bytes(const specattn_verify_args* args);
+
+/* Zero the arrival counters at the head of a verify workspace (enqueued on the stream).
+ * Call once after allocating it; the kernels leave the counters zero when they finish. */
+int specattn_verify_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+int specattn_sparse_verify(const specattn_verify_args* args, void* cuda_stream);
+
+/* ========================================================================================
+ * specattn_verify_step_host -- one whole verification step from HOST buffers.
+ *
+ * Alg. 1, blocks "Sparse Attention Mask Creation" and "Verification with Sparse Attention":
+ * one select over the mapped draft layers, then one sparse verify per target layer, with the
+ * step's inputs and results crossing PCIe inside the call.  In stream order it
+ *   1. copies draft_probs_host[u] -> select.draft_probs[u] for every mapped draft layer,
+ *   2. runs specattn_select_topp(select),
+ *   3. for each target layer j: copies q_host[j] -> verify[j].q, runs
+ *      specattn_sparse_verify(verify[j]) and copies verify[j].out / .lse -> out_host[j] /
+ *      lse_host[j].
+ * `select` and `verify[j]` are complete device-side argument structs (their device buffers,
+ * including the staging buffers the copies land in, are the caller's); verify[j].idx/counts
+ * must already point at the lists of layer_map[j] (or dense be set where layer_map[j] < 0).
+ * Host buffers should be pinned for the copies to be asynchronous.  Nothing is synchronised:
+ * the results are in the host buffers once the stream has drained.
+ * ======================================================================================== */
+typedef struct specattn_step_host_args {
+  uint32_t struct_size;
+  int32_t n_target_layers;
+  const specattn_select_args* select;     /* HOST */
+  const float* const* draft_probs_host;   /* HOST [n_draft_layers] of HOST pointers */
+  const specattn_verify_args* verify;     /* HOST [n_target_layers] */
+  const void* const* q_host;              /* HOST [n_target_layers] of HOST pointers (bf16) */
+  float* const* out_host;                 /* HOST [n_target_layers] of HOST pointers */
+  float* const* lse_host;                 /* HOST [n_target_layers] of HOST pointers */
+} specattn_step_host_args;
+
+int specattn_verify_step_host(const specattn_step_host_args* args, void* cuda_stream);
+
+/* Text for a SPECATTN_ERR_* return code (static storage, never NULL). */
+const char* specattn_status_string(int code);
+
+/* Number of kernels this library has launched in the calling process since load (for
+ * accounting in benchmarks); thread-safe. */
+int64_t specattn_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECATTN_H_ */

@@ -1,0 +1,649 @@
+// specattn_sparse_verify: grouped-query sparse decode attention of the gamma+1 verification
+// queries over the selected rows of a paged bf16 K/V cache, for sm_100a.
+//
+// Paper: Eq. 1 restricted to the index set I of Eq. 2-3 (normalised over I), Sec. 3.5, and
+// Alg. 1's "Verification with Sparse Attention" (one list per layer, shared by all gamma+1
+// queries and by all heads of a GQA group).  The paper feeds a CSR mask to a library
+// block-sparse kernel; here the ascending index lists are consumed directly.
+//
+// Mapping to the GPU.  The work of a call is the list of (sequence, kv head) units, unit u
+// holding count(u) tokens; it is cut into atoms of 16 tokens and the atoms are dealt evenly
+// and contiguously to one persistent CTA per SM, so ragged batches balance without any host
+// knowledge of the counts.  Inside a CTA
+//   - four producer warps resolve position -> (page, slot) through the block table and fetch
+//     each selected 256-byte K row and V row with one 1-D bulk async copy (TMA unit, no tensor
+//     map) into a padded, bank-conflict-free shared-memory tile; a 4-stage ring of 64-token
+//     tiles guarded by full/empty mbarriers keeps >100 KB of reads in flight per SM;
+//   - the consumer warps own one 16-row slab of the (gamma+1) x group query block and a share
+//     of every tile's keys: S = Q K^T and O += P V run on the tensor cores (bf16 mma.sync,
+//     fp32 accumulate; P is split into two bf16 terms so that it carries 16 mantissa bits),
+//     online softmax in fp32 registers in the log2 domain;
+//   - at the end of a unit the key-split warps combine through shared memory; a unit that was
+//     cut between CTAs is finished by whichever CTA arrives last at the unit's counter, which
+//     merges all partial (O, m, l) records in a fixed order -- nobody ever waits on a peer.
+// Every mbarrier wait is bounded; on expiry the CTA flags SPECATTN_ROW_TIMEOUT and leaves.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <atomic>
+
+#include "ptx.cuh"
+#include "specattn.h"
+
+namespace specattn {
+
+extern std::atomic<long long> g_launch_count;
+int device_sm_count();
+
+namespace {
+
+constexpr int kD = 128;            // head dimension
+constexpr int kRowBytes = kD * 2;  // one K or V row of one head
+constexpr int kPitch = kRowBytes + 16;  // shared-memory row pitch: ldmatrix hits 8 distinct 16-byte lanes
+constexpr int kStageTok = 64;
+constexpr int kStages = 4;
+constexpr int kProdWarps = 4;  // one per stage
+constexpr int kAtom = 16;
+constexpr int kMaxUnits = SPECATTN_MAX_VERIFY_UNITS;
+constexpr int kRec = 68 * 32;  // floats of one warp's (acc[64], m0, l0, m1, l1) record, lane-major
+constexpr int kCountersPerUnit = 4;
+constexpr size_t kCounterBytes = static_cast<size_t>(kMaxUnits) * kCountersPerUnit * sizeof(unsigned int);
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct VerifyParams {
+  int B, T, Hq, Hkv, grp, M, G, dense;
+  int page_size, page_shift;  // page_shift >= 0 when page_size is a power of two
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* kv;
+  long long n_pages, s_page, s_kv, s_slot, s_head;
+  const int* bt;
+  long long bt_stride;
+  const int* kv_len;
+  const int* idx;
+  long long idx_stride;
+  const int* counts;
+  float scale_log2;
+  float* out;
+  float* lse;
+  int* status;
+  unsigned int* counters;
+  float* partials;
+};
+
+template <int MT, int KS>
+struct VShared {
+  alignas(128) unsigned char kv[kStages][2][kStageTok * kPitch];
+  alignas(16) unsigned char q[MT * 16 * kPitch];
+  float scratch[MT][(KS / 2 > 0) ? KS / 2 : 1][kRec];
+  alignas(8) unsigned long long full[kStages];
+  unsigned long long empty[kStages];
+  unsigned long long q_full, q_empty;
+  int unit_start[kMaxUnits + 1];
+  int unit_cnt[kMaxUnits];
+  volatile int abort_flag;
+};
+
+__device__ __forceinline__ int unit_count(const VerifyParams& P, int u) {
+  const int b = u / P.Hkv;
+  long long c;
+  if (P.dense) {
+    c = P.kv_len[b];
+  } else {
+    const int g = (P.G == 1) ? 0 : (u % P.Hkv);
+    c = P.counts[static_cast<long long>(b) * P.G + g];
+    if (c > P.idx_stride) c = P.idx_stride;
+  }
+  if (c < 0) c = 0;
+  return static_cast<int>(c);
+}
+
+// First atom of CTA i when n atoms are dealt to np CTAs.
+__device__ __forceinline__ int cta_first_atom(long long i, long long n, long long np) {
+  return static_cast<int>(i * n / np);
+}
+// The CTA that owns atom x.
+__device__ __forceinline__ int cta_of_atom(long long x, long long n, long long np) {
+  long long i = ((x + 1) * np + n - 1) / n - 1;
+  if (i > np - 1) i = np - 1;
+  return static_cast<int>(i);
+}
+
+// Scales that bring a running maximum m and an incoming maximum im to their common maximum.
+__device__ __forceinline__ void merge_scales(float m, float im, float& mn, float& a_old, float& a_in) {
+  mn = fmaxf(m, im);
+  const float base = (mn == -INFINITY) ? 0.f : mn;
+  a_old = ex2(m - base);   // ex2(-inf) = 0
+  a_in = ex2(im - base);
+}
+
+template <int MT, int KS>
+__global__ void __launch_bounds__((MT * KS + kProdWarps) * 32, 1)
+sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
+  using Sh = VShared<MT, KS>;
+  constexpr int NC = MT * KS;                  // consumer warps
+  constexpr int NT = (NC + kProdWarps) * 32;   // threads
+  constexpr int KPW = kStageTok / KS;          // keys per consumer warp per stage
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  Sh& sh = *reinterpret_cast<Sh*>(smem_raw);
+
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const int warp = tid >> 5;
+  const int U = P.B * P.Hkv;
+
+  // ---- set-up: zero the tiles (stale rows must stay finite), barriers, unit prefix ------------
+  {
+    uint4* z = reinterpret_cast<uint4*>(sh.kv);
+    for (int i = tid; i < static_cast<int>(sizeof(sh.kv) / 16); i += NT) z[i] = make_uint4(0u, 0u, 0u, 0u);
+    uint4* zq = reinterpret_cast<uint4*>(sh.q);
+    for (int i = tid; i < static_cast<int>(sizeof(sh.q) / 16); i += NT) zq[i] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sh.full[s], 1);
+      mbar_init(&sh.empty[s], NC);
+    }
+    mbar_init(&sh.q_full, 1);
+    mbar_init(&sh.q_empty, NC);
+    mbar_fence_init();
+    sh.abort_flag = 0;
+    sh.unit_start[0] = 0;
+  }
+  for (int u = tid; u < U; u += NT) {
+    const int c = unit_count(P, u);
+    sh.unit_cnt[u] = c;
+    sh.unit_start[u + 1] = (c + kAtom - 1) / kAtom;
+  }
+  fence_proxy_async();
+  __syncthreads();
+  if (warp == 0) {  // inclusive scan of the atom counts, 32 at a time
+    int carry = 0;
+    for (int base = 0; base < U; base += 32) {
+      const int u = base + lane;
+      int v = (u < U) ? sh.unit_start[u + 1] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += n;
+      }
+      if (u < U) sh.unit_start[u + 1] = v + carry;
+      carry += __shfl_sync(0xffffffffu, v, 31);
+    }
+  }
+  __syncthreads();
+
+  // units with an empty list: out = 0, lse = -inf
+  for (int u = blockIdx.x; u < U; u += gridDim.x) {
+    if (sh.unit_cnt[u] != 0) continue;
+    const int b = u / P.Hkv, kvh = u % P.Hkv;
+    for (int e = tid; e < P.M * kD; e += NT) {
+      const int r = e / kD, t = r / P.grp, h = kvh * P.grp + r % P.grp;
+      P.out[((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD + e % kD] = 0.f;
+      if (e % kD == 0) P.lse[(static_cast<long long>(b) * P.T + t) * P.Hq + h] = -INFINITY;
+    }
+  }
+
+  const long long N = sh.unit_start[U];
+  const long long NP = (N < static_cast<long long>(gridDim.x)) ? N : static_cast<long long>(gridDim.x);
+  if (static_cast<long long>(blockIdx.x) >= NP) return;
+  const int a0 = cta_first_atom(blockIdx.x, N, NP);
+  const int a1 = cta_first_atom(blockIdx.x + 1, N, NP);
+
+  // unit holding atom a0
+  int u_first;
+  {
+    int lo = 0, hi = U - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (sh.unit_start[mid] <= a0) lo = mid; else hi = mid - 1;
+    }
+    u_first = lo;
+    while (sh.unit_start[u_first + 1] <= a0) ++u_first;  // skip empty units that share the start
+  }
+
+  if (warp >= NC) {
+    // =========================== producer warps ===========================================
+    const int pw = warp - NC;
+    int it = 0, seg = 0;
+    int last_it = -1;
+    int a = a0, u = u_first;
+    bool dead = false;
+    while (a < a1 && !dead) {
+      const int us = sh.unit_start[u], ue = sh.unit_start[u + 1];
+      const int seg_hi = min(a1, ue);
+      const int b = u / P.Hkv, kvh = u % P.Hkv;
+      const int tok_lo = (a - us) * kAtom;
+      const int tok_hi = min(sh.unit_cnt[u], (seg_hi - us) * kAtom);
+      const int kvlen_b = P.kv_len[b];
+      const int* list = P.dense ? nullptr
+                                : P.idx + (static_cast<long long>(b) * P.G + ((P.G == 1) ? 0 : kvh)) * P.idx_stride;
+      const __nv_bfloat16* kv_head = P.kv + static_cast<long long>(kvh) * P.s_head;
+      bool first = true;
+      for (int t0 = tok_lo; t0 < tok_hi; t0 += kStageTok, ++it, first = false) {
+        if ((it % kProdWarps) != pw) continue;
+        const int s = it % kStages;
+        const unsigned ph = (it / kStages) & 1u;
+        if (!mbar_wait(&sh.empty[s], ph ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
+        if (first) {
+          // the query block of this unit: M rows of 256 bytes
+          if (!mbar_wait(&sh.q_empty, (seg & 1u) ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
+          if (lane == 0) mbar_arrive_expect_tx(&sh.q_full, static_cast<uint32_t>(P.M) * kRowBytes);
+          __syncwarp();
+          for (int r = lane; r < P.M; r += 32) {
+            const int t = r / P.grp, h = kvh * P.grp + r % P.grp;
+            bulk_g2s(sh.q + r * kPitch, P.q + ((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD,
+                     kRowBytes, &sh.q_full);
+          }
+        }
+        const int ntok = min(kStageTok, tok_hi - t0);
+        if (lane == 0) mbar_arrive_expect_tx(&sh.full[s], static_cast<uint32_t>(ntok) * 2u * kRowBytes);
+        __syncwarp();
+        bool bad = false;
+#pragma unroll
+        for (int jj = 0; jj < kStageTok / 32; ++jj) {
+          const int j = lane + jj * 32;
+          if (j < ntok) {
+            int pos = P.dense ? (t0 + j) : __ldg(list + t0 + j);
+            if (pos < 0 || pos >= kvlen_b) { bad = true; pos = 0; }
+            const int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
+            const int slot = pos - lp * P.page_size;
+            long long page = P.bt ? static_cast<long long>(__ldg(P.bt + b * P.bt_stride + lp))
+                                  : (b * P.bt_stride + lp);
+            if (page < 0 || (P.n_pages > 0 && page >= P.n_pages)) { bad = true; page = 0; }
+            const __nv_bfloat16* src = kv_head + page * P.s_page + static_cast<long long>(slot) * P.s_slot;
+            bulk_g2s(sh.kv[s][0] + j * kPitch, src, kRowBytes, &sh.full[s]);
+            bulk_g2s(sh.kv[s][1] + j * kPitch, src + P.s_kv, kRowBytes, &sh.full[s]);
+          }
+        }
+        if (bad && P.status) atomicOr(P.status + b, SPECATTN_ROW_BAD_INDEX);
+        last_it = it;
+      }
+      a = seg_hi;
+      ++seg;
+      if (a == ue) {
+        ++u;
+        while (u < U && sh.unit_start[u + 1] == sh.unit_start[u]) ++u;
+      }
+    }
+    if (sh.abort_flag && last_it >= 0) {
+      // give this warp's last copies a bounded chance to land before the CTA retires
+      mbar_wait(&sh.full[last_it % kStages], (last_it / kStages) & 1u, nullptr);
+    }
+    return;
+  }
+
+  // =============================== consumer warps ===========================================
+  const int mt = warp / KS;   // 16-row slab of the query block
+  const int ks = warp % KS;   // share of each tile's keys
+  const int g = lane >> 2, tq = lane & 3;
+  const int lm = lane >> 3, lr = lane & 7;  // ldmatrix: matrix id, row within it
+  const uint32_t q_addr = smem_u32(sh.q) + (mt * 16 + (lm & 1) * 8 + lr) * kPitch + (lm >> 1) * 16;
+  // per-lane byte offsets inside a tile for the K (non-transposed) and V (transposed) fragments
+  const uint32_t k_off = ((lm >> 1) * 8 + lr) * kPitch + (lm & 1) * 16;
+  const uint32_t v_off = ((lm & 1) * 8 + lr) * kPitch + (lm >> 1) * 16;
+
+  // A warp that meets a failed wait raises abort_flag and stops computing, but still walks
+  // through the combine barriers of the segment it is in; every warp re-reads the flag right
+  // after those barriers, so a whole key-split group always leaves together.
+  int it = 0, seg = 0;
+  int a = a0, u = u_first;
+  bool ok = true;
+  while (a < a1) {
+    const int us = sh.unit_start[u], ue = sh.unit_start[u + 1];
+    const int seg_hi = min(a1, ue);
+    const int b = u / P.Hkv, kvh = u % P.Hkv;
+    const int tok_lo = (a - us) * kAtom;
+    const int tok_hi = min(sh.unit_cnt[u], (seg_hi - us) * kAtom);
+
+    // query fragments of this unit
+    uint32_t qf[8][4];
+    ok = mbar_wait(&sh.q_full, seg & 1u, &sh.abort_flag);
+    if (!ok) sh.abort_flag = 1;
+#pragma unroll
+    for (int kk = 0; kk < 8; ++kk) ldmatrix_x4(qf[kk], q_addr + kk * 32);
+    __syncwarp();
+    if (ok && lane == 0) mbar_arrive(&sh.q_empty);
+
+    float acc[16][4];
+#pragma unroll
+    for (int n = 0; n < 16; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+    for (int t0 = tok_lo; ok && t0 < tok_hi; t0 += kStageTok, ++it) {
+      const int s = it % kStages;
+      const unsigned ph = (it / kStages) & 1u;
+      if (!mbar_wait(&sh.full[s], ph, &sh.abort_flag)) { sh.abort_flag = 1; ok = false; break; }
+      const int ntok = min(kStageTok, tok_hi - t0);
+      const uint32_t k_base = smem_u32(sh.kv[s][0]);
+      const uint32_t v_base = smem_u32(sh.kv[s][1]);
+#pragma unroll
+      for (int sub = 0; sub < KPW / 16; ++sub) {
+        const int key0 = ks * KPW + sub * 16;
+        if (key0 >= ntok) break;
+        const int valid = ntok - key0;  // keys of this 16-block that exist (may exceed 16)
+        float sc[2][4];
+#pragma unroll
+        for (int n = 0; n < 2; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          uint32_t kf[4];
+          ldmatrix_x4(kf, k_base + key0 * kPitch + k_off + kk * 32);
+          mma_bf16(sc[0], qf[kk], kf[0], kf[1]);
+          mma_bf16(sc[1], qf[kk], kf[2], kf[3]);
+        }
+#pragma unroll
+        for (int n = 0; n < 2; ++n)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int key = n * 8 + tq * 2 + (i & 1);
+            sc[n][i] = (key < valid) ? sc[n][i] * P.scale_log2 : -INFINITY;
+          }
+        float mx0 = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
+        float mx1 = fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3]));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+        const float base0 = (mn0 == -INFINITY) ? 0.f : mn0;
+        const float base1 = (mn1 == -INFINITY) ? 0.f : mn1;
+        const float al0 = ex2(m0 - base0), al1 = ex2(m1 - base1);
+        m0 = mn0;
+        m1 = mn1;
+        float p[2][4];
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+          p[n][0] = ex2(sc[n][0] - base0);
+          p[n][1] = ex2(sc[n][1] - base0);
+          p[n][2] = ex2(sc[n][2] - base1);
+          p[n][3] = ex2(sc[n][3] - base1);
+        }
+        l0 = l0 * al0 + (p[0][0] + p[0][1] + p[1][0] + p[1][1]);
+        l1 = l1 * al1 + (p[0][2] + p[0][3] + p[1][2] + p[1][3]);
+#pragma unroll
+        for (int n = 0; n < 16; ++n) {
+          acc[n][0] *= al0;
+          acc[n][1] *= al0;
+          acc[n][2] *= al1;
+          acc[n][3] *= al1;
+        }
+        // P = P_hi + P_lo, two bf16 terms
+        uint32_t phi[4], plo[4];
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+#pragma unroll
+          for (int hrow = 0; hrow < 2; ++hrow) {
+            const float x = p[n][hrow * 2], y = p[n][hrow * 2 + 1];
+            const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
+            const float xr = x - __bfloat162float(xh), yr = y - __bfloat162float(yh);
+            __nv_bfloat162 hi2;
+            hi2.x = xh;
+            hi2.y = yh;
+            phi[n * 2 + hrow] = *reinterpret_cast<uint32_t*>(&hi2);
+            plo[n * 2 + hrow] = pack_bf16(xr, yr);
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          uint32_t vf[4];
+          ldmatrix_x4_trans(vf, v_base + key0 * kPitch + v_off + j * 32);
+          mma_bf16(acc[2 * j], phi, vf[0], vf[1]);
+          mma_bf16(acc[2 * j + 1], phi, vf[2], vf[3]);
+          mma_bf16(acc[2 * j], plo, vf[0], vf[1]);
+          mma_bf16(acc[2 * j + 1], plo, vf[2], vf[3]);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.empty[s]);
+    }
+
+    // ---- end of the segment: row sums across the quad, then combine the key-split warps ------
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+#pragma unroll
+    for (int half = KS / 2; half >= 1; half >>= 1) {
+      if (ks >= half && ks < 2 * half) {
+        float* rec = sh.scratch[mt][ks - half];
+#pragma unroll
+        for (int n = 0; n < 16; ++n)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) rec[(n * 4 + i) * 32 + lane] = acc[n][i];
+        rec[64 * 32 + lane] = m0;
+        rec[65 * 32 + lane] = l0;
+        rec[66 * 32 + lane] = m1;
+        rec[67 * 32 + lane] = l1;
+      }
+      named_bar_sync(1 + mt, KS * 32);
+      if (ks < half) {
+        const float* rec = sh.scratch[mt][ks];
+        float mn, ao, ai;
+        merge_scales(m0, rec[64 * 32 + lane], mn, ao, ai);
+        l0 = l0 * ao + rec[65 * 32 + lane] * ai;
+        m0 = mn;
+        float mn1, ao1, ai1;
+        merge_scales(m1, rec[66 * 32 + lane], mn1, ao1, ai1);
+        l1 = l1 * ao1 + rec[67 * 32 + lane] * ai1;
+        m1 = mn1;
+#pragma unroll
+        for (int n = 0; n < 16; ++n) {
+          acc[n][0] = acc[n][0] * ao + rec[(n * 4 + 0) * 32 + lane] * ai;
+          acc[n][1] = acc[n][1] * ao + rec[(n * 4 + 1) * 32 + lane] * ai;
+          acc[n][2] = acc[n][2] * ao1 + rec[(n * 4 + 2) * 32 + lane] * ai1;
+          acc[n][3] = acc[n][3] * ao1 + rec[(n * 4 + 3) * 32 + lane] * ai1;
+        }
+      }
+      named_bar_sync(1 + mt, KS * 32);
+    }
+
+    if (sh.abort_flag) { ok = false; break; }
+
+    if (ks == 0) {
+      const bool whole = (a == us) && (seg_hi == ue);
+      bool finish = whole;
+      if (!whole) {
+        // publish this CTA's share of the unit, then see whether it was the last to arrive
+        float* rec = P.partials + (static_cast<size_t>(2 * blockIdx.x + (a == a0 ? 0 : 1)) * MT + mt) * kRec;
+#pragma unroll
+        for (int n = 0; n < 16; ++n)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) __stcg(rec + (n * 4 + i) * 32 + lane, acc[n][i]);
+        __stcg(rec + 64 * 32 + lane, m0);
+        __stcg(rec + 65 * 32 + lane, l0);
+        __stcg(rec + 66 * 32 + lane, m1);
+        __stcg(rec + 67 * 32 + lane, l1);
+        __threadfence();
+        __syncwarp();
+        const int i_lo = cta_of_atom(us, N, NP), i_hi = cta_of_atom(ue - 1, N, NP);
+        unsigned int old = 0;
+        if (lane == 0) old = atomicAdd(P.counters + u * kCountersPerUnit + mt, 1u);
+        old = __shfl_sync(0xffffffffu, old, 0);
+        if (old == static_cast<unsigned int>(i_hi - i_lo)) {
+          finish = true;
+          __threadfence();
+          // merge every contributor's record in CTA order (the own one included, from memory)
+          m0 = m1 = -INFINITY;
+          l0 = l1 = 0.f;
+#pragma unroll
+          for (int n = 0; n < 16; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+          for (int i = i_lo; i <= i_hi; ++i) {
+            const int first_atom = cta_first_atom(i, N, NP);
+            const float* r2 = P.partials + (static_cast<size_t>(2 * i + (first_atom >= us ? 0 : 1)) * MT + mt) * kRec;
+            float mn, ao, ai;
+            merge_scales(m0, __ldcg(r2 + 64 * 32 + lane), mn, ao, ai);
+            l0 = l0 * ao + __ldcg(r2 + 65 * 32 + lane) * ai;
+            m0 = mn;
+            float mn1, ao1, ai1;
+            merge_scales(m1, __ldcg(r2 + 66 * 32 + lane), mn1, ao1, ai1);
+            l1 = l1 * ao1 + __ldcg(r2 + 67 * 32 + lane) * ai1;
+            m1 = mn1;
+#pragma unroll
+            for (int n = 0; n < 16; ++n) {
+              acc[n][0] = acc[n][0] * ao + __ldcg(r2 + (n * 4 + 0) * 32 + lane) * ai;
+              acc[n][1] = acc[n][1] * ao + __ldcg(r2 + (n * 4 + 1) * 32 + lane) * ai;
+              acc[n][2] = acc[n][2] * ao1 + __ldcg(r2 + (n * 4 + 2) * 32 + lane) * ai1;
+              acc[n][3] = acc[n][3] * ao1 + __ldcg(r2 + (n * 4 + 3) * 32 + lane) * ai1;
+            }
+          }
+          if (lane == 0) P.counters[u * kCountersPerUnit + mt] = 0u;  // ready for the next call
+        }
+      }
+      if (finish) {
+        const float inv0 = (l0 > 0.f) ? 1.f / l0 : 0.f;
+        const float inv1 = (l1 > 0.f) ? 1.f / l1 : 0.f;
+        const int r0 = mt * 16 + g, r1 = r0 + 8;
+        if (r0 < P.M) {
+          const int t = r0 / P.grp, h = kvh * P.grp + r0 % P.grp;
+          const long long row = (static_cast<long long>(b) * P.T + t) * P.Hq + h;
+          float* o = P.out + row * kD + tq * 2;
+#pragma unroll
+          for (int n = 0; n < 16; ++n)
+            *reinterpret_cast<float2*>(o + n * 8) = make_float2(acc[n][0] * inv0, acc[n][1] * inv0);
+          if (tq == 0) P.lse[row] = (l0 > 0.f) ? (m0 + log2f(l0)) * kLn2 : -INFINITY;
+        }
+        if (r1 < P.M) {
+          const int t = r1 / P.grp, h = kvh * P.grp + r1 % P.grp;
+          const long long row = (static_cast<long long>(b) * P.T + t) * P.Hq + h;
+          float* o = P.out + row * kD + tq * 2;
+#pragma unroll
+          for (int n = 0; n < 16; ++n)
+            *reinterpret_cast<float2*>(o + n * 8) = make_float2(acc[n][2] * inv1, acc[n][3] * inv1);
+          if (tq == 0) P.lse[row] = (l1 > 0.f) ? (m1 + log2f(l1)) * kLn2 : -INFINITY;
+        }
+      }
+    }
+
+    a = seg_hi;
+    ++seg;
+    if (a == ue) {
+      ++u;
+      while (u < U && sh.unit_start[u + 1] == sh.unit_start[u]) ++u;
+    }
+  }
+  if (!ok && P.status && lane == 0) atomicOr(P.status, SPECATTN_ROW_TIMEOUT);
+}
+
+template <int MT, int KS>
+cudaError_t launch(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
+  const size_t smem = sizeof(VShared<MT, KS>) + 128;
+  cudaError_t err = cudaFuncSetAttribute(sparse_verify_kernel<MT, KS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (err != cudaSuccess) return err;
+  sparse_verify_kernel<MT, KS><<<n_ctas, (MT * KS + kProdWarps) * 32, smem, stream>>>(P);
+  return cudaGetLastError();
+}
+
+int m_tiles(const specattn_verify_args& A) {
+  const int grp = A.n_q_heads / A.n_kv_heads;
+  return (A.n_q * grp + 15) / 16;
+}
+
+int validate(const specattn_verify_args* args) {
+  if (args == nullptr) return SPECATTN_ERR_NULL;
+  if (args->struct_size != sizeof(specattn_verify_args)) return SPECATTN_ERR_STRUCT_SIZE;
+  const specattn_verify_args& A = *args;
+  if (A.batch < 0 || A.n_q < 1 || A.n_q_heads < 1 || A.n_kv_heads < 1 || A.page_size < 1 || A.n_groups < 1)
+    return SPECATTN_ERR_RANGE;
+  if (A.n_q_heads % A.n_kv_heads != 0) return SPECATTN_ERR_RANGE;
+  if (A.n_groups != 1 && A.n_groups != A.n_kv_heads) return SPECATTN_ERR_RANGE;
+  if (A.head_dim != kD) return SPECATTN_ERR_UNSUPPORTED;
+  if (A.n_q * (A.n_q_heads / A.n_kv_heads) > SPECATTN_MAX_QUERY_ROWS) return SPECATTN_ERR_UNSUPPORTED;
+  if (static_cast<long long>(A.batch) * A.n_kv_heads > kMaxUnits) return SPECATTN_ERR_UNSUPPORTED;
+  return SPECATTN_OK;
+}
+
+size_t workspace_bytes_for(const specattn_verify_args& A, int n_ctas) {
+  return kCounterBytes + static_cast<size_t>(2) * n_ctas * m_tiles(A) * kRec * sizeof(float);
+}
+
+}  // namespace
+}  // namespace specattn
+
+using specattn::VerifyParams;
+
+extern "C" size_t specattn_verify_workspace_bytes(const specattn_verify_args* args) {
+  if (specattn::validate(args) != SPECATTN_OK) return 0;
+  const int n = specattn::device_sm_count();
+  if (n <= 0) return 0;
+  return specattn::workspace_bytes_for(*args, n);
+}
+
+extern "C" int specattn_verify_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (workspace == nullptr) return SPECATTN_ERR_NULL;
+  if (workspace_bytes < specattn::kCounterBytes) return SPECATTN_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return SPECATTN_ERR_ALIGN;
+  if (cudaMemsetAsync(workspace, 0, specattn::kCounterBytes, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+    cudaGetLastError();
+    return SPECATTN_ERR_CUDA;
+  }
+  return SPECATTN_OK;
+}
+
+extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cuda_stream) {
+  const int v = specattn::validate(args);
+  if (v != SPECATTN_OK) return v;
+  const specattn_verify_args& A = *args;
+  if (A.batch == 0) return SPECATTN_OK;
+  if (!A.q || !A.kv_pages || !A.kv_len || !A.out || !A.lse || !A.workspace) return SPECATTN_ERR_NULL;
+  if (!A.dense && (!A.idx || !A.counts)) return SPECATTN_ERR_NULL;
+  if (!A.dense && A.idx_stride < 0) return SPECATTN_ERR_RANGE;
+  if (A.block_table_stride < 0 || A.n_pages < 0) return SPECATTN_ERR_RANGE;
+  auto mis = [](const void* p, uintptr_t a) { return reinterpret_cast<uintptr_t>(p) % a != 0; };
+  if (mis(A.q, 16) || mis(A.kv_pages, 16) || mis(A.out, 16) || mis(A.workspace, 256)) return SPECATTN_ERR_ALIGN;
+  if (A.stride_page % 8 || A.stride_kv % 8 || A.stride_slot % 8 || A.stride_head % 8) return SPECATTN_ERR_ALIGN;
+  const int n_ctas = specattn::device_sm_count();
+  if (n_ctas <= 0) return SPECATTN_ERR_CUDA;
+  if (A.workspace_bytes < specattn::workspace_bytes_for(A, n_ctas)) return SPECATTN_ERR_WORKSPACE;
+
+  VerifyParams P;
+  memset(&P, 0, sizeof(P));
+  P.B = A.batch;
+  P.T = A.n_q;
+  P.Hq = A.n_q_heads;
+  P.Hkv = A.n_kv_heads;
+  P.grp = A.n_q_heads / A.n_kv_heads;
+  P.M = P.T * P.grp;
+  P.G = A.n_groups;
+  P.dense = A.dense ? 1 : 0;
+  P.page_size = A.page_size;
+  P.page_shift = -1;
+  for (int s = 0; s < 31; ++s)
+    if ((1 << s) == A.page_size) P.page_shift = s;
+  P.q = static_cast<const __nv_bfloat16*>(A.q);
+  P.kv = static_cast<const __nv_bfloat16*>(A.kv_pages);
+  P.n_pages = A.n_pages;
+  P.s_page = A.stride_page;
+  P.s_kv = A.stride_kv;
+  P.s_slot = A.stride_slot;
+  P.s_head = A.stride_head;
+  P.bt = A.block_table;
+  P.bt_stride = A.block_table_stride;
+  P.kv_len = A.kv_len;
+  P.idx = A.idx;
+  P.idx_stride = A.idx_stride;
+  P.counts = A.counts;
+  const float scale = (A.sm_scale != 0.f) ? A.sm_scale : 1.0f / sqrtf(static_cast<float>(A.head_dim));
+  P.scale_log2 = scale * specattn::kLog2e;
+  P.out = A.out;
+  P.lse = A.lse;
+  P.status = A.status;
+  P.counters = static_cast<unsigned int*>(A.workspace);
+  P.partials = reinterpret_cast<float*>(static_cast<unsigned char*>(A.workspace) + specattn::kCounterBytes);
+
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t err;
+  switch (specattn::m_tiles(A)) {
+    case 1: err = specattn::launch<1, 4>(P, n_ctas, stream); break;
+    case 2: err = specattn::launch<2, 4>(P, n_ctas, stream); break;
+    case 3: err = specattn::launch<3, 2>(P, n_ctas, stream); break;
+    default: err = specattn::launch<4, 2>(P, n_ctas, stream); break;
+  }
+  if (err != cudaSuccess) return SPECATTN_ERR_CUDA;
+  specattn::g_launch_count.fetch_add(1, std::memory_order_relaxed);
+  return SPECATTN_OK;
+}

@@ -1,0 +1,100 @@
+"""One SpecAttn verification step as a reusable launch plan: the device buffers and the C
+argument structs are prepared once, ``run()`` then issues one specattn_select_topp and one
+specattn_sparse_verify per target layer on a stream (Alg. 1, blocks "Sparse Attention Mask
+Creation" and "Verification with Sparse Attention").  Orchestration only; every computation
+happens in the library's kernels."""
+from __future__ import annotations
+
+import ctypes as C
+from typing import Sequence
+
+import torch
+
+from . import (SelectArgs, VerifyArgs, SpecAttnError, lib, make_select_args, make_verify_args,
+               verify_step_host, verify_workspace, _stream_ptr)
+
+__all__ = ["VerifyStep"]
+
+
+class VerifyStep:
+    def __init__(self, *, layer_map: Sequence[int], n_draft_layers: int, batch: int,
+                 n_draft_heads: int, gamma: int, L_stride: int, n_q_heads: int, p: float,
+                 kv_pools: Sequence[torch.Tensor], kv_len: torch.Tensor,
+                 block_table: torch.Tensor | None, pages_per_seq: int | None = None,
+                 n_groups: int = 1, head_group: Sequence[int] | None = None,
+                 idx_stride: int | None = None, sm_scale: float = 0.0, device=None):
+        dev = device or kv_pools[0].device
+        self.layer_map = [int(x) for x in layer_map]
+        self.n_layers = len(self.layer_map)
+        assert len(kv_pools) == self.n_layers
+        used = sorted({u for u in self.layer_map if u >= 0})
+        self.used = used
+        B, T = batch, gamma + 1
+        d = kv_pools[0].shape[-1]
+        self.draft_probs = [torch.zeros((B, n_draft_heads, gamma, L_stride), dtype=torch.float32, device=dev)
+                            if u in used else None for u in range(n_draft_layers)]
+        stride = int(L_stride if idx_stride is None else idx_stride)
+        self.idx = torch.zeros((n_draft_layers, B, n_groups, stride), dtype=torch.int32, device=dev)
+        self.counts = torch.full((n_draft_layers, B, n_groups), -1, dtype=torch.int32, device=dev)
+        self.row_status = torch.full((n_draft_layers, B, n_groups), -1, dtype=torch.int32, device=dev)
+        self.diag = torch.zeros((n_draft_layers, B, n_groups, 4), dtype=torch.float64, device=dev)
+        self.kv_len, self.block_table, self.kv_pools = kv_len, block_table, list(kv_pools)
+        self.q = [torch.zeros((B, T, n_q_heads, d), dtype=torch.bfloat16, device=dev) for _ in range(self.n_layers)]
+        self.out = [torch.empty((B, T, n_q_heads, d), dtype=torch.float32, device=dev) for _ in range(self.n_layers)]
+        self.lse = [torch.empty((B, T, n_q_heads), dtype=torch.float32, device=dev) for _ in range(self.n_layers)]
+        self.status = torch.zeros((self.n_layers, B), dtype=torch.int32, device=dev)
+        self.select_args, self._keep = make_select_args(
+            self.draft_probs, kv_len, self.layer_map, p, n_groups=n_groups, head_group=head_group,
+            idx=self.idx, counts=self.counts, row_status=self.row_status, diag=self.diag)
+        self.verify_args: list[VerifyArgs] = []
+        self.workspace = None
+        for j, u in enumerate(self.layer_map):
+            a = make_verify_args(self.q[j], kv_pools[j], kv_len, block_table=block_table,
+                                 pages_per_seq=pages_per_seq,
+                                 idx=None if u < 0 else self.idx[u], counts=None if u < 0 else self.counts[u],
+                                 n_groups=n_groups, dense=u < 0, sm_scale=sm_scale, out=self.out[j],
+                                 lse=self.lse[j], status=self.status[j])
+            if self.workspace is None:
+                self.workspace = verify_workspace(a, dev)
+            a.workspace, a.workspace_bytes = self.workspace.data_ptr(), self.workspace.numel()
+            self.verify_args.append(a)
+
+    # ---- inputs -------------------------------------------------------------------------------
+    def load_inputs(self, draft_probs_host: Sequence[torch.Tensor | None], q_host: Sequence[torch.Tensor]):
+        """Plain (untimed) upload of a step's inputs into the plan's device buffers."""
+        for u in self.used:
+            self.draft_probs[u].copy_(draft_probs_host[u], non_blocking=True)
+        for j in range(self.n_layers):
+            self.q[j].copy_(q_host[j], non_blocking=True)
+
+    # ---- launches -----------------------------------------------------------------------------
+    def run_select(self, stream=None):
+        rc = lib().specattn_select_topp(C.byref(self.select_args), _stream_ptr(stream))
+        if rc != 0:
+            raise SpecAttnError(rc, "specattn_select_topp")
+
+    def run_verify(self, j: int, stream=None):
+        rc = lib().specattn_sparse_verify(C.byref(self.verify_args[j]), _stream_ptr(stream))
+        if rc != 0:
+            raise SpecAttnError(rc, "specattn_sparse_verify")
+
+    def run(self, stream=None):
+        """Device-resident step: 1 select launch + n_layers verify launches."""
+        sp = _stream_ptr(stream)
+        L = lib()
+        rc = L.specattn_select_topp(C.byref(self.select_args), sp)
+        if rc != 0:
+            raise SpecAttnError(rc, "specattn_select_topp")
+        for a in self.verify_args:
+            rc = L.specattn_sparse_verify(C.byref(a), sp)
+            if rc != 0:
+                raise SpecAttnError(rc, "specattn_sparse_verify")
+
+    def run_host(self, draft_probs_host, q_host, out_host, lse_host, stream=None):
+        """Whole step from pinned host tensors through specattn_verify_step_host."""
+        verify_step_host(self.select_args, draft_probs_host, self.verify_args, q_host, out_host,
+                         lse_host, stream)
+
+    @property
+    def launches_per_step(self) -> int:
+        return 1 + self.n_layers

@@ -1,0 +1,181 @@
+"""GPU parity of specattn_select_topp (through the C ABI) against the CPU oracle.
+
+Index lists must match the sorted-prefix nucleus of App. A Eq. 7 / Alg. 2 bit for bit; rows whose
+boundary mass lies within 1e-5 of p are counted apart and may only differ by a neighbouring
+threshold."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+from gpu_util import compare_lists, dev, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_rows(rows: np.ndarray, kv_len, p, idx_stride=None):
+    """R = 1: each row is its own list.  rows [n_rows, L_stride] float32."""
+    import paper_2510_27641_b200 as sa
+    n_rows, Ls = rows.shape
+    kv = np.asarray(kv_len, np.int32) if np.ndim(kv_len) else np.full(n_rows, kv_len, np.int32)
+    probs = rows.reshape(n_rows, 1, 1, Ls)
+    gi, gc, gs, gd = sa.select_topp([to_dev(probs)], to_dev(kv), [0], p, idx_stride=idx_stride,
+                                    want_diag=True)
+    torch.cuda.synchronize()
+    oi, oc, os_, od = oracle.select_topp([probs], np.zeros(1, np.int32), kv, p, idx_stride=idx_stride)
+    st = compare_lists(lambda i: rows[i, :kv[i]], p, gi.cpu().numpy(), gc.cpu().numpy(),
+                       gs.cpu().numpy(), oi, oc, os_, od)
+    return st, gd.cpu().numpy(), od
+
+
+@pytest.mark.parametrize("family", wl.TOPP_FAMILIES)
+@pytest.mark.parametrize("n", [1024, 8192, 40000])
+def test_row_families_match_oracle(family, n):
+    rows = wl.topp_rows(family, 24, n, seed=n)
+    for p in wl.TOPP_PS:
+        st, gd, od = _run_rows(rows, n, p)
+        assert st["n"] == 24
+        # masses reported by the kernel agree with the oracle's binary64 sums
+        assert np.allclose(gd.reshape(-1, 4), od.reshape(-1, 6)[:, :4], rtol=1e-9, atol=0)
+
+
+def test_long_rows_span_a_full_cluster():
+    rows = wl.topp_rows("uniform", 3, 131072, seed=5)
+    rows = np.concatenate([rows, wl.topp_rows("quantised", 3, 131072, seed=6),
+                           wl.topp_rows("zipf", 2, 131072, seed=7)])
+    for p in (0.5, 0.99):
+        st, _, _ = _run_rows(rows, 131072, p)
+        assert st["n"] == 8
+
+
+def test_ragged_lengths_and_tails():
+    rng = np.random.default_rng(0)
+    Ls = 5000
+    lens = np.array([0, 1, 2, 3, 4, 5, 31, 32, 33, 1023, 1025, 4093, 4999, 5000], np.int32)
+    rows = np.zeros((len(lens), Ls), np.float32)
+    for i, L in enumerate(lens):
+        rows[i, :L] = rng.random(L, dtype=np.float32) ** 3
+        rows[i, L:] = 7.0      # beyond kv_len: must be ignored entirely
+    for p in (0.3, 0.9):
+        st, _, _ = _run_rows(rows, lens, p)
+        assert st["n"] == len(lens)
+
+
+def test_degenerate_rows():
+    n = 4096
+    rows = np.zeros((8, n), np.float32)
+    rows[0] = 0.25                       # constant: everything ties
+    rows[1, 1234] = 1.0                  # one-hot
+    # row 2 all zero: everything ties at zero
+    rows[3] = np.float32(1e-42)          # denormal constant
+    rows[4, :] = np.where(np.arange(n) % 2 == 0, 0.5, 0.0)
+    rows[5, :100] = np.exp2(-np.arange(100, dtype=np.float32))  # spans 100 exponents
+    rows[6, :] = 1.0
+    rows[6, 7] = 3.0e38                  # huge dynamic range
+    rows[7, :] = np.float32(np.nextafter(np.float32(1), np.float32(2)))
+    rows[7, ::3] = 1.0                   # two values one ulp apart
+    for p in (0.001, 0.5, 0.999):
+        st, _, _ = _run_rows(rows, n, p)
+        assert st["n"] == 8
+    import paper_2510_27641_b200 as sa
+    gi, gc, gs, _ = sa.select_topp([to_dev(rows.reshape(8, 1, 1, n))], to_dev(np.full(8, n, np.int32)), [0], 0.5)
+    assert gc.cpu().numpy().ravel().tolist()[:3] == [n, 1, n]
+
+
+def test_p_one_keeps_everything_and_zeros():
+    rows = wl.topp_rows("zipf", 4, 3000, seed=1)
+    rows[:, ::7] = 0.0
+    st, _, _ = _run_rows(rows, np.array([3000, 2999, 17, 0], np.int32), 1.0)
+    assert st["exact"] == 4
+
+
+def test_invalid_probabilities_are_flagged_per_list():
+    import paper_2510_27641_b200 as sa
+    rows = wl.topp_rows("uniform", 6, 9000, seed=2)
+    rows[1, 8999] = np.nan
+    rows[2, 0] = -1e-30
+    rows[3, 4500] = np.inf
+    rows[4, 100] = -0.0          # minus zero is a valid zero
+    rows[5, 8000] = -1.0         # beyond kv_len below: not an input
+    kv = np.array([9000, 9000, 9000, 9000, 9000, 7000], np.int32)
+    st, _, _ = _run_rows(rows, kv, 0.9)
+    assert st["n"] == 6
+    _, _, gs, _ = sa.select_topp([to_dev(rows.reshape(6, 1, 1, 9000))], to_dev(kv), [0], 0.9)
+    assert gs.cpu().numpy().ravel().tolist() == [0, sa.ROW_INVALID_PROB, sa.ROW_INVALID_PROB,
+                                                 sa.ROW_INVALID_PROB, 0, 0]
+
+
+def test_capacity_overflow_truncates_and_reports_true_count():
+    rows = wl.topp_rows("uniform", 5, 4096, seed=3)
+    st, _, _ = _run_rows(rows, 4096, 0.9, idx_stride=100)
+    assert st["n"] == 5
+
+
+@pytest.mark.parametrize("G", [1, 2, 4])
+def test_aggregation_over_heads_queries_layers_and_groups(G):
+    import paper_2510_27641_b200 as sa
+    B, H, gamma, n_d = 3, 12, 5, 3
+    kv_len = np.array([4096, 1000, 2731], np.int32)
+    Ls = 4096
+    probs = [wl.draft_probs(7, u, kv_len, H, gamma, Ls, sink=6.0, slope=0.004) if u != 1 else None
+             for u in range(n_d)]
+    layer_map = np.array([-1, 0, 0, 2, 2, 2], np.int32)
+    hg = None if G == 1 else (np.arange(H) * G // H).astype(np.int32)
+    for p in (0.9, 0.95):
+        gi, gc, gs, gd = sa.select_topp([None if x is None else to_dev(x) for x in probs], to_dev(kv_len),
+                                        layer_map.tolist(), p, n_groups=G,
+                                        head_group=None if hg is None else hg.tolist(), want_diag=True)
+        torch.cuda.synchronize()
+        oi, oc, os_, od = oracle.select_topp(probs, layer_map, kv_len, p, n_groups=G, head_group=hg)
+
+        def row(i):
+            u, b, g = i // (B * G), (i // G) % B, i % G
+            return oracle.aggregate(probs[u][b], L=int(kv_len[b]), head_group=hg, g=g)[0]
+
+        st = compare_lists(row, p, gi.cpu().numpy(), gc.cpu().numpy(), gs.cpu().numpy(), oi, oc, os_, od)
+        assert st["n"] == 2 * B * G
+        assert np.all(gc.cpu().numpy()[1] == -1)      # unmapped layer untouched
+
+
+def test_order_of_the_binary32_adds_is_heads_then_queries():
+    import paper_2510_27641_b200 as sa
+    big = np.float32(2.0 ** 24)
+    A = np.zeros((1, 2, 2, 8), np.float32)
+    A[0, :, :, 0] = [[big, 1.0], [1.0, 0.0]]    # ((2^24 + 1) + 1) + 0 = 2^24 in binary32
+    A[0, :, :, 1] = [[1.0, 1.0], [big, 0.0]]    # exact 2^24 + 2
+    A[0, :, :, 2] = 16777217.5                  # rounds per add; just another large value
+    A[0, :, :, 3:] = 1.0
+    kv = np.array([8], np.int32)
+    gi, gc, _, gd = sa.select_topp([to_dev(A)], to_dev(kv), [0], 0.2, want_diag=True)
+    oi, oc, _, od = oracle.select_topp([A], np.zeros(1, np.int32), kv, 0.2)
+    assert gc.item() == oc.item() and np.array_equal(gi.cpu().numpy()[0, 0, 0, :oc.item()], oi[0, 0, 0, :oc.item()])
+    assert gd.cpu().numpy()[0, 0, 0, 0] == od[0, 0, 0, 0]   # totals equal bit for bit: same a_bar
+
+
+def test_argument_errors_are_synchronous_and_launch_nothing():
+    import paper_2510_27641_b200 as sa
+    probs = to_dev(wl.topp_rows("uniform", 2, 1024, 0).reshape(2, 1, 1, 1024))
+    kv = to_dev(np.full(2, 1024, np.int32))
+    before = sa.kernel_launch_count()
+    for bad_p in (0.0, -0.5, float("nan")):
+        with pytest.raises(sa.SpecAttnError) as e:
+            sa.select_topp([probs], kv, [0], bad_p)
+        assert e.value.code == -3
+    with pytest.raises(sa.SpecAttnError) as e:
+        sa.select_topp([probs], kv, [1], 0.5)          # layer_map out of range
+    assert e.value.code == -3
+    with pytest.raises(sa.SpecAttnError) as e:
+        sa.select_topp([probs[:, :, :, :1022].contiguous()], kv, [0], 0.5)   # L_stride % 4 != 0
+    assert e.value.code == -4
+    assert sa.kernel_launch_count() == before
+    # repeated calls are deterministic
+    a = sa.select_topp([probs], kv, [0], 0.7)
+    b = sa.select_topp([probs], kv, [0], 0.7)
+    torch.cuda.synchronize()
+    assert torch.equal(a[1], b[1])
+    n = int(a[1][0, 0, 0])
+    assert torch.equal(a[0][0, 0, 0, :n], b[0][0, 0, 0, :n])
+    assert sa.kernel_launch_count() == before + 2

@@ -1,0 +1,186 @@
+"""End-to-end parity of a whole verification step (select -> sparse verify per target layer)
+against the CPU oracle, on the benchmark configurations at reduced and at full shapes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+from gpu_util import check_attention, compare_lists, dev, to_dev
+from workloads import bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def _build(cfg, n_groups=1, head_group=None, dense_first=0):
+    from paper_2510_27641_b200.step import VerifyStep
+    si = wl.make_step_inputs(cfg)
+    if dense_first:
+        si.layer_map[:dense_first] = -1
+    pools = [wl.kv_pool(cfg.seed, j, si.n_pages, cfg.page_size, cfg.n_kv_heads, cfg.head_dim, device=dev())
+             for j in range(cfg.n_target_layers)]
+    kv_len = to_dev(si.kv_len)
+    bt = None if si.block_table is None else to_dev(si.block_table)
+    step = VerifyStep(layer_map=si.layer_map.tolist(), n_draft_layers=cfg.n_draft_layers, batch=cfg.batch,
+                      n_draft_heads=cfg.n_draft_heads, gamma=cfg.gamma, L_stride=si.L_stride,
+                      n_q_heads=cfg.n_q_heads, p=cfg.p, kv_pools=pools, kv_len=kv_len, block_table=bt,
+                      pages_per_seq=si.pages_per_seq, n_groups=n_groups, head_group=head_group)
+    step.load_inputs([None if x is None else torch.from_numpy(x) for x in si.draft_probs],
+                     [bf16.bits_to_torch(q) for q in si.q])
+    return si, pools, step
+
+
+def _check_step(cfg, si, pools, step, layers, n_groups=1, head_group=None):
+    oi, oc, os_, od = oracle.select_topp(si.draft_probs, si.layer_map, si.kv_len, cfg.p,
+                                         n_groups=n_groups, head_group=head_group)
+    B, G = cfg.batch, n_groups
+
+    def row(i):
+        u, b, g = i // (B * G), (i // G) % B, i % G
+        return oracle.aggregate(si.draft_probs[u][b], L=int(si.kv_len[b]), head_group=head_group, g=g)[0]
+
+    st = compare_lists(row, cfg.p, step.idx.cpu().numpy(), step.counts.cpu().numpy(),
+                       step.row_status.cpu().numpy(), oi, oc, os_, od)
+    worst = (0.0, 0.0)
+    for j in layers:
+        u = int(si.layer_map[j])
+        kv_bits = bf16.torch_to_bits(pools[j].cpu())
+        # the oracle attends the GPU's own lists, so attention parity does not hinge on a
+        # near-boundary row having taken the neighbouring threshold
+        idx = step.idx[u].cpu().numpy() if u >= 0 else None
+        cnt = step.counts[u].cpu().numpy() if u >= 0 else None
+        ro, rl = oracle.sparse_verify(si.q[j], kv_bits, wl.kv_strides(cfg.page_size, cfg.n_kv_heads, cfg.head_dim),
+                                      si.block_table, si.kv_len, idx, cnt, n_kv_heads=cfg.n_kv_heads,
+                                      page_size=cfg.page_size, n_groups=n_groups, dense=u < 0,
+                                      pages_per_seq=si.pages_per_seq)
+        e = check_attention(step.out[j], step.lse[j], ro, rl)
+        worst = (max(worst[0], e[0]), max(worst[1], e[1]))
+    assert int(step.status.abs().sum()) == 0
+    return st, worst
+
+
+def test_config0_full_size():
+    cfg = wl.config0()
+    si, pools, step = _build(cfg)
+    step.run()
+    torch.cuda.synchronize()
+    st, worst = _check_step(cfg, si, pools, step, [0])
+    assert st["n"] == 1
+
+
+def test_config1_shape_reduced_layers_and_context():
+    cfg = wl.config1().scaled(n_target_layers=5, n_draft_layers=3, batch=3, ctx=6000)
+    si, pools, step = _build(cfg, dense_first=1)
+    step.run()
+    torch.cuda.synchronize()
+    st, worst = _check_step(cfg, si, pools, step, range(5))
+    assert st["n"] == len(set(si.layer_map.tolist()) - {-1}) * 3
+
+
+def test_config3_ragged_reduced():
+    cfg = wl.config3().scaled(batch=9, ctx=9000, ctx_min=300)
+    si, pools, step = _build(cfg)
+    step.run()
+    torch.cuda.synchronize()
+    st, worst = _check_step(cfg, si, pools, step, [0])
+    assert st["n"] == 9 and len(set(si.kv_len.tolist())) > 5
+
+
+def test_config4_shape_reduced_with_per_head_lists():
+    cfg = wl.config4(n_target_layers=2).scaled(batch=2, ctx=20000, n_draft_layers=2)
+    hg = (np.arange(16) * 8 // 16).astype(np.int32)
+    si, pools, step = _build(cfg, n_groups=8, head_group=hg.tolist())
+    step.run()
+    torch.cuda.synchronize()
+    st, worst = _check_step(cfg, si, pools, step, [0, 1], n_groups=8, head_group=hg)
+    # p = 1 on the same kernel equals the dense flag
+    from paper_2510_27641_b200.step import VerifyStep
+    step1 = VerifyStep(layer_map=si.layer_map.tolist(), n_draft_layers=2, batch=2, n_draft_heads=16, gamma=4,
+                       L_stride=si.L_stride, n_q_heads=64, p=1.0, kv_pools=pools, kv_len=step.kv_len,
+                       block_table=step.block_table)
+    step1.load_inputs([None if x is None else torch.from_numpy(x) for x in si.draft_probs],
+                      [bf16.bits_to_torch(q) for q in si.q])
+    step1.run()
+    stepd = VerifyStep(layer_map=[-1, -1], n_draft_layers=2, batch=2, n_draft_heads=16, gamma=4,
+                       L_stride=si.L_stride, n_q_heads=64, p=1.0, kv_pools=pools, kv_len=step.kv_len,
+                       block_table=step.block_table)
+    stepd.load_inputs([None, None], [bf16.bits_to_torch(q) for q in si.q])
+    stepd.run()
+    torch.cuda.synchronize()
+    for j in range(2):
+        assert torch.equal(step1.out[j], stepd.out[j]) and torch.equal(step1.lse[j], stepd.lse[j])
+    u = int(si.layer_map[0])
+    assert step1.counts[u].cpu().numpy().ravel().tolist() == [20000, 20000]
+
+
+def test_host_buffer_step_matches_device_resident_step():
+    cfg = wl.config1().scaled(n_target_layers=4, n_draft_layers=2, batch=2, ctx=3000)
+    si, pools, step = _build(cfg)
+    step.run()
+    torch.cuda.synchronize()
+    ref_out = [o.clone() for o in step.out]
+    ref_lse = [l.clone() for l in step.lse]
+    ref_idx, ref_cnt = step.idx.clone(), step.counts.clone()
+    # wipe device-side inputs and results, then run the whole step from pinned host memory
+    for t in step.draft_probs:
+        if t is not None:
+            t.zero_()
+    for j in range(4):
+        step.q[j].zero_()
+        step.out[j].zero_()
+    step.counts.fill_(-1)
+    dp_host = [None if x is None else torch.from_numpy(x).pin_memory() for x in si.draft_probs]
+    q_host = [bf16.bits_to_torch(q).pin_memory() for q in si.q]
+    out_host = [torch.zeros(o.shape, dtype=torch.float32).pin_memory() for o in step.out]
+    lse_host = [torch.zeros(l.shape, dtype=torch.float32).pin_memory() for l in step.lse]
+    step.run_host(dp_host, q_host, out_host, lse_host)
+    torch.cuda.synchronize()
+    assert torch.equal(step.counts, ref_cnt)
+    for j in range(4):
+        assert torch.equal(out_host[j], ref_out[j].cpu()) and torch.equal(lse_host[j], ref_lse[j].cpu())
+
+
+@pytest.mark.parametrize("which", ["cfg1", "cfg3"])
+def test_full_size_sampled_outputs(which):
+    """Full batch / context of configs 1 and 3 (two target layers for config 1): every list is
+    compared; attention is checked on sampled (layer, sequence, kv head) units whose K/V rows
+    are regenerated on the CPU from the hashed pool definition."""
+    if which == "cfg1":
+        cfg = wl.config1().scaled(n_target_layers=2)
+    else:
+        cfg = wl.config3()
+    si, pools, step = _build(cfg)
+    step.run()
+    torch.cuda.synchronize()
+    oi, oc, os_, od = oracle.select_topp(si.draft_probs, si.layer_map, si.kv_len, cfg.p)
+    B = cfg.batch
+
+    def row(i):
+        u, b = i // B, i % B
+        return oracle.aggregate(si.draft_probs[u][b], L=int(si.kv_len[b]))[0]
+
+    st = compare_lists(row, cfg.p, step.idx.cpu().numpy(), step.counts.cpu().numpy(),
+                       step.row_status.cpu().numpy(), oi, oc, os_, od)
+    assert st["n"] == len(set(si.layer_map.tolist())) * B
+    rng = np.random.default_rng(0)
+    sp, sk, ss, sh = wl.kv_strides(cfg.page_size, cfg.n_kv_heads, cfg.head_dim)
+    grp = cfg.n_q_heads // cfg.n_kv_heads
+    d = cfg.head_dim
+    for _ in range(6):
+        j = int(rng.integers(0, cfg.n_target_layers))
+        b = int(rng.integers(0, B))
+        hk = int(rng.integers(0, cfg.n_kv_heads))
+        u = int(si.layer_map[j])
+        c = int(step.counts[u, b, 0])
+        pos = step.idx[u, b, 0, :c].cpu().numpy().astype(np.int64)
+        page = si.block_table[b, pos // cfg.page_size].astype(np.int64)
+        base = page * sp + (pos % cfg.page_size) * ss + hk * sh
+        flat = torch.from_numpy(base)[:, None] + torch.arange(d)[None, :]
+        K = bf16.torch_to_bits(wl.kv_values(cfg.seed, j, flat))
+        V = bf16.torch_to_bits(wl.kv_values(cfg.seed, j, flat + sk))
+        qrows = si.q[j][b][:, hk * grp:(hk + 1) * grp, :].reshape(-1, d)
+        ro, rl = oracle.attend_rows(qrows, K, V)
+        go = step.out[j][b, :, hk * grp:(hk + 1) * grp, :].reshape(-1, d)
+        gl = step.lse[j][b, :, hk * grp:(hk + 1) * grp].reshape(-1)
+        check_attention(go, gl, ro, rl)
+    assert int(step.status.abs().sum()) == 0

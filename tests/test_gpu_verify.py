@@ -1,0 +1,173 @@
+"""GPU parity of specattn_sparse_verify (through the C ABI) against the CPU oracle's fp64
+attention restricted to the listed rows (Eq. 1 over the index set of Eq. 2-3)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+from gpu_util import bf16_to_dev, check_attention, dev, to_dev
+from workloads import bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def _make_case(seed, B, T, Hq, Hkv, page, lens, G=1, counts=None, shuffle=True, d=128):
+    rng = np.random.default_rng(seed)
+    lens = np.asarray(lens, np.int32)
+    pages_per_seq = max(1, (int(lens.max()) + page - 1) // page)
+    n_pages = B * pages_per_seq
+    kv = wl.kv_pool(seed, 0, n_pages, page, Hkv, d)                      # torch bf16 on CPU
+    bt = wl.block_table(seed, B, pages_per_seq, n_pages, shuffle=shuffle)
+    q = wl.queries(seed, 0, B, T, Hq, d)
+    stride = max(1, int(lens.max()))
+    idx = np.zeros((B, G, stride), np.int32)
+    cnt = np.zeros((B, G), np.int32)
+    for b in range(B):
+        for g in range(G):
+            c = int(counts[b][g]) if counts is not None else int(rng.integers(0, lens[b] + 1))
+            c = min(c, int(lens[b]))
+            sel = np.sort(rng.choice(int(lens[b]), size=c, replace=False)) if c else np.zeros(0, np.int64)
+            idx[b, g, :c] = sel
+            cnt[b, g] = c
+    return dict(q=q, kv=kv, bt=bt, lens=lens, idx=idx, cnt=cnt, page=page, Hkv=Hkv, G=G,
+                pages_per_seq=pages_per_seq)
+
+
+def _run(case, dense=False, use_bt=True, sm_scale=0.0, workspace=None):
+    import paper_2510_27641_b200 as sa
+    kv_d = case["kv"].to(dev())
+    out, lse, status = sa.sparse_verify(
+        bf16_to_dev(case["q"]), kv_d, to_dev(case["lens"]),
+        block_table=to_dev(case["bt"]) if use_bt else None, pages_per_seq=case["pages_per_seq"],
+        idx=None if dense else to_dev(case["idx"]), counts=None if dense else to_dev(case["cnt"]),
+        n_groups=case["G"], dense=dense, sm_scale=sm_scale, workspace=workspace)
+    torch.cuda.synchronize()
+    return out, lse, status
+
+
+def _oracle(case, dense=False, use_bt=True, scale=0.0):
+    kv_bits = bf16.torch_to_bits(case["kv"])
+    page, Hkv = case["page"], case["Hkv"]
+    return oracle.sparse_verify(case["q"], kv_bits, wl.kv_strides(page, Hkv, 128),
+                                case["bt"] if use_bt else None, case["lens"], case["idx"], case["cnt"],
+                                n_kv_heads=Hkv, page_size=page, n_groups=case["G"], dense=dense,
+                                scale=scale, pages_per_seq=case["pages_per_seq"])
+
+
+@pytest.mark.parametrize("T,Hq,Hkv", [(5, 32, 8), (6, 32, 8), (5, 64, 8), (2, 8, 2), (8, 16, 2), (1, 4, 4)])
+def test_query_block_shapes(T, Hq, Hkv):
+    case = _make_case(10 + T, 3, T, Hq, Hkv, 16, [700, 130, 1], counts=[[300], [130], [1]])
+    out, lse, status = _run(case)
+    check_attention(out, lse, *_oracle(case))
+    assert status.cpu().numpy().tolist() == [0, 0, 0]
+
+
+def test_list_lengths_around_tile_edges_and_empty_lists():
+    lens = [2000] * 14
+    counts = [[c] for c in (0, 1, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129)]
+    case = _make_case(20, 14, 5, 32, 8, 16, lens, counts=counts)
+    out, lse, _ = _run(case)
+    check_attention(out, lse, *_oracle(case))
+    assert torch.all(out[0] == 0) and torch.all(torch.isneginf(lse[0]))
+
+
+def test_long_lists_are_split_across_ctas_and_merged():
+    # one sequence, 2 kv heads: every unit is cut among ~74 CTAs and merged by the last arriver
+    case = _make_case(21, 1, 6, 8, 2, 16, [40000], counts=[[33333]])
+    out, lse, _ = _run(case)
+    check_attention(out, lse, *_oracle(case))
+    # bitwise reproducible regardless of which CTA happens to arrive last
+    out2, lse2, _ = _run(case)
+    assert torch.equal(out, out2) and torch.equal(lse, lse2)
+
+
+def test_ragged_batch_with_shared_workspace_reuse():
+    import paper_2510_27641_b200 as sa
+    rng = np.random.default_rng(3)
+    lens = rng.integers(1, 6000, size=12).tolist()
+    case = _make_case(22, 12, 5, 32, 8, 16, lens)
+    out, lse, _ = _run(case)
+    ref = _oracle(case)
+    check_attention(out, lse, *ref)
+    # the same workspace serves consecutive calls on a stream
+    kv_d = case["kv"].to(dev())
+    q_d, len_d, bt_d = bf16_to_dev(case["q"]), to_dev(case["lens"]), to_dev(case["bt"])
+    idx_d, cnt_d = to_dev(case["idx"]), to_dev(case["cnt"])
+    o = torch.empty_like(out)
+    l = torch.empty_like(lse)
+    args = sa.make_verify_args(q_d, kv_d, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d, out=o, lse=l)
+    ws = sa.verify_workspace(args)
+    for _ in range(3):
+        o.fill_(float("nan"))
+        sa.sparse_verify(q_d, kv_d, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d, out=o, lse=l, workspace=ws)
+        torch.cuda.synchronize()
+        assert torch.equal(o, out) and torch.equal(l, lse)
+
+
+def test_dense_flag_equals_full_list_and_contiguous_cache():
+    lens = [1000, 37, 2048]
+    case = _make_case(23, 3, 5, 32, 8, 16, lens, counts=[[1000], [37], [2048]], shuffle=False)
+    o_d, l_d, _ = _run(case, dense=True)
+    check_attention(o_d, l_d, *_oracle(case, dense=True))
+    o_f, l_f, _ = _run(case)                      # the p = 1 list
+    assert torch.equal(o_d, o_f) and torch.equal(l_d, l_f)
+    o_c, l_c, _ = _run(case, use_bt=False)        # identity block table == contiguous addressing
+    assert torch.equal(o_c, o_f) and torch.equal(l_c, l_f)
+    check_attention(o_c, l_c, *_oracle(case, use_bt=False))
+
+
+def test_per_kv_head_lists_page_sizes_and_scale():
+    for page in (1, 8, 16, 48):
+        case = _make_case(24 + page, 2, 5, 16, 4, page, [900, 333], G=4)
+        out, lse, _ = _run(case, sm_scale=0.05)
+        check_attention(out, lse, *_oracle(case, scale=0.05))
+
+
+def test_precision_when_few_tokens_dominate():
+    # two nearly tied dominant keys with large opposite values: exposes bf16 rounding of P
+    case = _make_case(30, 1, 5, 32, 8, 16, [64], counts=[[2]])
+    kvb = bf16.torch_to_bits(case["kv"]).copy()
+    vals = bf16.to_f32(kvb)
+    pages = case["bt"][0]
+    for k, pos in enumerate(case["idx"][0, 0, :2]):
+        vals[pages[pos // 16], 1, pos % 16] = 4.0 if k == 0 else -4.0
+        vals[pages[pos // 16], 0, pos % 16] *= 0.01
+    case["kv"] = bf16.bits_to_torch(bf16.from_f32(vals)).reshape(case["kv"].shape)
+    out, lse, _ = _run(case)
+    check_attention(out, lse, *_oracle(case))
+
+
+def test_bad_positions_and_pages_are_flagged_not_followed():
+    import paper_2510_27641_b200 as sa
+    case = _make_case(31, 3, 5, 32, 8, 16, [500, 500, 500], counts=[[100], [100], [100]])
+    case["idx"][1, 0, 5] = 500          # == kv_len: out of range
+    case["idx"][1, 0, 6] = -3
+    case["bt"][2, 0:32] = 10 ** 6       # page id far outside the pool
+    out, lse, status = _run(case)
+    st = status.cpu().numpy()
+    assert st[0] == 0 and st[1] == sa.ROW_BAD_INDEX and st[2] == sa.ROW_BAD_INDEX
+    assert torch.all(torch.isfinite(out))
+    ref_o, ref_l = _oracle(dict(case, idx=case["idx"][:1], cnt=case["cnt"][:1], lens=case["lens"][:1],
+                                bt=case["bt"][:1], q=case["q"][:1]))
+    check_attention(out[:1], lse[:1], ref_o, ref_l)
+
+
+def test_argument_errors():
+    import paper_2510_27641_b200 as sa
+    case = _make_case(32, 1, 5, 32, 8, 16, [64], counts=[[10]])
+    q_d, kv_d = bf16_to_dev(case["q"]), case["kv"].to(dev())
+    len_d, bt_d = to_dev(case["lens"]), to_dev(case["bt"])
+    idx_d, cnt_d = to_dev(case["idx"]), to_dev(case["cnt"])
+    with pytest.raises(sa.SpecAttnError) as e:     # 9 queries x group 8 = 72 rows > 64
+        q9 = torch.zeros((1, 9, 64, 128), dtype=torch.bfloat16, device=dev())
+        sa.sparse_verify(q9, kv_d, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d)
+    assert e.value.code == -6
+    tiny = torch.zeros(1024, dtype=torch.uint8, device=dev())
+    with pytest.raises(sa.SpecAttnError) as e:
+        sa.sparse_verify(q_d, kv_d, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d, workspace=tiny)
+    assert e.value.code == -5
+    with pytest.raises(sa.SpecAttnError) as e:     # misaligned K/V base
+        kv_off = kv_d.view(-1)[4:4 + 3 * 32768].view(3, 2, 16, 8, 128)
+        sa.sparse_verify(q_d, kv_off, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d)
+    assert e.value.code == -4
