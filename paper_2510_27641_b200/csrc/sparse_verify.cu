@@ -222,23 +222,23 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       const int* list = P.dense ? nullptr
                                 : P.idx + (static_cast<long long>(b) * P.G + ((P.G == 1) ? 0 : kvh)) * P.idx_stride;
       const __nv_bfloat16* kv_head = P.kv + static_cast<long long>(kvh) * P.s_head;
-      bool first = true;
-      for (int t0 = tok_lo; t0 < tok_hi; t0 += kStageTok, ++it, first = false) {
+      if (pw == 0) {
+        // The query block of this unit: M rows of 256 bytes.  Always the same warp, walking
+        // the segments in order, so its parity wait can never be satisfied by a stale phase.
+        if (!mbar_wait(&sh.q_empty, (seg & 1u) ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
+        if (lane == 0) mbar_arrive_expect_tx(&sh.q_full, static_cast<uint32_t>(P.M) * kRowBytes);
+        __syncwarp();
+        for (int r = lane; r < P.M; r += 32) {
+          const int t = r / P.grp, h = kvh * P.grp + r % P.grp;
+          bulk_g2s(sh.q + r * kPitch, P.q + ((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD,
+                   kRowBytes, &sh.q_full);
+        }
+      }
+      for (int t0 = tok_lo; t0 < tok_hi; t0 += kStageTok, ++it) {
         if ((it % kProdWarps) != pw) continue;
         const int s = it % kStages;
         const unsigned ph = (it / kStages) & 1u;
         if (!mbar_wait(&sh.empty[s], ph ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
-        if (first) {
-          // the query block of this unit: M rows of 256 bytes
-          if (!mbar_wait(&sh.q_empty, (seg & 1u) ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
-          if (lane == 0) mbar_arrive_expect_tx(&sh.q_full, static_cast<uint32_t>(P.M) * kRowBytes);
-          __syncwarp();
-          for (int r = lane; r < P.M; r += 32) {
-            const int t = r / P.grp, h = kvh * P.grp + r % P.grp;
-            bulk_g2s(sh.q + r * kPitch, P.q + ((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD,
-                     kRowBytes, &sh.q_full);
-          }
-        }
         const int ntok = min(kStageTok, tok_hi - t0);
         if (lane == 0) mbar_arrive_expect_tx(&sh.full[s], static_cast<uint32_t>(ntok) * 2u * kRowBytes);
         __syncwarp();

@@ -43,9 +43,11 @@ class VerifyStep:
         self.out = [torch.empty((B, T, n_q_heads, d), dtype=torch.float32, device=dev) for _ in range(self.n_layers)]
         self.lse = [torch.empty((B, T, n_q_heads), dtype=torch.float32, device=dev) for _ in range(self.n_layers)]
         self.status = torch.zeros((self.n_layers, B), dtype=torch.int32, device=dev)
-        self.select_args, self._keep = make_select_args(
-            self.draft_probs, kv_len, self.layer_map, p, n_groups=n_groups, head_group=head_group,
-            idx=self.idx, counts=self.counts, row_status=self.row_status, diag=self.diag)
+        self.select_args, self._keep = None, None
+        if used:   # a step whose layers are all dense has nothing to select
+            self.select_args, self._keep = make_select_args(
+                self.draft_probs, kv_len, self.layer_map, p, n_groups=n_groups, head_group=head_group,
+                idx=self.idx, counts=self.counts, row_status=self.row_status, diag=self.diag)
         self.verify_args: list[VerifyArgs] = []
         self.workspace = None
         for j, u in enumerate(self.layer_map):
@@ -69,6 +71,8 @@ class VerifyStep:
 
     # ---- launches -----------------------------------------------------------------------------
     def run_select(self, stream=None):
+        if self.select_args is None:
+            return
         rc = lib().specattn_select_topp(C.byref(self.select_args), _stream_ptr(stream))
         if rc != 0:
             raise SpecAttnError(rc, "specattn_select_topp")
@@ -82,9 +86,7 @@ class VerifyStep:
         """Device-resident step: 1 select launch + n_layers verify launches."""
         sp = _stream_ptr(stream)
         L = lib()
-        rc = L.specattn_select_topp(C.byref(self.select_args), sp)
-        if rc != 0:
-            raise SpecAttnError(rc, "specattn_select_topp")
+        self.run_select(stream)
         for a in self.verify_args:
             rc = L.specattn_sparse_verify(C.byref(a), sp)
             if rc != 0:
@@ -97,4 +99,4 @@ class VerifyStep:
 
     @property
     def launches_per_step(self) -> int:
-        return 1 + self.n_layers
+        return (1 if self.select_args is not None else 0) + self.n_layers

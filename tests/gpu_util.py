@@ -76,7 +76,9 @@ def compare_lists(a_rows, p, g_idx, g_counts, g_status, o_idx, o_counts, o_statu
 
 def lse_err(got: np.ndarray, ref: np.ndarray) -> float:
     both_inf = np.isneginf(got) & np.isneginf(ref)
-    d = np.abs(np.where(both_inf, 0.0, got - ref)) / np.maximum(1.0, np.abs(np.where(both_inf, 0.0, ref)))
+    with np.errstate(invalid="ignore"):
+        diff = got - ref
+    d = np.abs(np.where(both_inf, 0.0, diff)) / np.maximum(1.0, np.abs(np.where(both_inf, 0.0, ref)))
     return float(np.max(d)) if d.size else 0.0
 
 
