@@ -1,0 +1,465 @@
+#!/usr/bin/env python
+"""Benchmark of the SpecAttn verification hot path on B200.
+
+A step = one pass of the whole hot path over one synthetic batch: one specattn_select_topp over
+the mapped draft layers followed by one specattn_sparse_verify per target layer (33 launches on
+the default workload).  Default workload: the Llama-3-8B-shaped configuration -- 32 target
+layers, 4-layer 12-head draft, batch 8, context 32768, paged bf16 KV (page 16, shuffled block
+table), gamma = 5, p = 0.95.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--topp-sweep]
+
+Prints ONE JSON line (rank 0).  `value` is microseconds per step with all inputs resident in
+HBM (CUDA-graph replay of the step, CUDA events, max over ranks); `e2e` is the same step issued
+through specattn_verify_step_host from pinned host buffers (draft probabilities and queries go
+host->device, outputs and LSE come back, inside the timed region); `roofline` describes the
+dominant kernel (sparse verify) against the measured HBM copy bandwidth; `cpu_baseline` is the
+CPU oracle timed on a bounded sample of the same workload and scaled to a step.
+With N > 1 every rank runs its own batch of 8 sequences (batch sharding, no collective).
+`--impl reference` times the CPU oracle alone (rank 0) and prints the same line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "sparse_verify_step_time"
+UNIT = "us/step"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum per sparse_verify launch on this workload, from
+# the ncu capture summarised in profiles/sparse_verify_cfg1.md (None until captured).
+NCU_VERIFY_TRAFFIC_BYTES = None
+
+
+# ----------------------------------------------------------------------------------------------
+def _rank_env():
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
+            int(os.environ.get("WORLD_SIZE", "1")))
+
+
+def _measured_peaks():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        try:
+            d = json.loads(f.read_text())
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+               0x2: "applications_clocks_setting"}
+
+    def __init__(self, index: int, uuid: str | None = None, period_s: float = 0.01):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in self.REASONS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------------------------
+def build_step(cfg, dev):
+    import torch
+    import workloads as wl
+    from paper_2510_27641_b200.step import VerifyStep
+    from workloads import bf16
+    si = wl.make_step_inputs(cfg)
+    pools = [wl.kv_pool(cfg.seed, j, si.n_pages, cfg.page_size, cfg.n_kv_heads, cfg.head_dim, device=dev)
+             for j in range(cfg.n_target_layers)]
+    step = VerifyStep(layer_map=si.layer_map.tolist(), n_draft_layers=cfg.n_draft_layers, batch=cfg.batch,
+                      n_draft_heads=cfg.n_draft_heads, gamma=cfg.gamma, L_stride=si.L_stride,
+                      n_q_heads=cfg.n_q_heads, p=cfg.p, kv_pools=pools,
+                      kv_len=torch.from_numpy(si.kv_len).to(dev),
+                      block_table=None if si.block_table is None else torch.from_numpy(si.block_table).to(dev),
+                      pages_per_seq=si.pages_per_seq)
+    dp_host = [None if x is None else torch.from_numpy(x).pin_memory() for x in si.draft_probs]
+    q_host = [bf16.bits_to_torch(q).pin_memory() for q in si.q]
+    step.load_inputs(dp_host, q_host)
+    torch.cuda.synchronize()
+    return si, pools, step, dp_host, q_host
+
+
+def capture(fn):
+    import torch
+    import paper_2510_27641_b200 as sa
+    g = torch.cuda.CUDAGraph()
+    n0 = sa.kernel_launch_count()
+    with torch.cuda.graph(g):
+        fn()
+    return g, sa.kernel_launch_count() - n0
+
+
+def time_replays(g, steps, warmup, barrier=None):
+    """Microseconds per replay, CUDA events on the replaying (current) stream."""
+    import torch
+    for _ in range(warmup):
+        g.replay()
+    torch.cuda.synchronize()
+    if barrier is not None:
+        barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    if barrier is not None:
+        barrier()
+    return e0.elapsed_time(e1) * 1e3 / steps
+
+
+def verify_bytes(cfg, si, counts_layer):
+    """Algorithmic bytes of ONE sparse_verify launch: selected K and V rows, their indices, the
+    block-table entries of the touched pages, the queries and the outputs."""
+    c = counts_layer.astype(np.int64)          # [B, G]
+    kv = int(c.sum()) * cfg.n_kv_heads * cfg.head_dim * 2 * 2 if c.shape[1] == 1 \
+        else int(c.sum()) * cfg.head_dim * 2 * 2
+    idx_b = 4 * int(c.sum())
+    bt_b = 4 * int(np.minimum(c, (si.kv_len[:, None] + cfg.page_size - 1) // cfg.page_size).sum())
+    q_b = 2 * cfg.batch * cfg.n_q * cfg.n_q_heads * cfg.head_dim
+    o_b = 4 * cfg.batch * cfg.n_q * cfg.n_q_heads * (cfg.head_dim + 1)
+    return kv + idx_b + bt_b + q_b + o_b, kv
+
+
+def select_bytes(cfg, si, n_used, counts):
+    R = cfg.n_draft_heads * cfg.gamma
+    read = 4 * R * int(si.kv_len.astype(np.int64).sum()) * n_used
+    return read + 4 * int(counts[counts >= 0].sum())
+
+
+# ----------------------------------------------------------------------------------------------
+class OracleSample:
+    """The CPU oracle on a bounded sample of the workload, scaled to one step: selection
+    (O1 + O2) for every list of the step, attention (O3) for `n_attn_layers` target layers (all
+    sequences and heads), scaled by n_target_layers / n_attn_layers.  The K/V rows the oracle
+    reads come from the device pools when those exist (one device->host copy per sampled
+    layer, untimed); otherwise only the listed rows are regenerated on the CPU from the hashed
+    pool definition into a compact pool of the touched pages."""
+
+    def __init__(self, cfg, si, n_attn_layers, pools=None):
+        import torch
+        import oracle
+        import workloads as wl
+        from workloads import bf16
+        self.cfg, self.si, self.oracle = cfg, si, oracle
+        self.strides = wl.kv_strides(cfg.page_size, cfg.n_kv_heads, cfg.head_dim)
+        sp, sk, ss, sh = self.strides
+        oi, oc, _, _ = oracle.select_topp(si.draft_probs, si.layer_map, si.kv_len, cfg.p)
+        self.layers = list(range(cfg.n_target_layers))[:max(1, n_attn_layers)]
+        self.prepared = []
+        for j in self.layers:
+            u = int(si.layer_map[j])
+            if pools is not None:
+                self.prepared.append((bf16.torch_to_bits(pools[j].cpu()), si.block_table))
+                continue
+            bt_small = np.zeros_like(si.block_table)
+            n_small, flats, dsts = 0, [], []
+            for b in range(cfg.batch):
+                pos = oi[u, b, 0, :int(oc[u, b, 0])].astype(np.int64)
+                lps = np.unique(pos // cfg.page_size)
+                bt_small[b, lps] = n_small + np.arange(len(lps))
+                src_page = si.block_table[b, pos // cfg.page_size].astype(np.int64)
+                dst_page = bt_small[b, pos // cfg.page_size].astype(np.int64)
+                n_small += len(lps)
+                row = np.arange(cfg.n_kv_heads * cfg.head_dim, dtype=np.int64)     # all heads of a slot
+                for kvsel in (0, 1):
+                    flats.append((src_page * sp + kvsel * sk + (pos % cfg.page_size) * ss)[:, None] + row[None, :])
+                    dsts.append((dst_page * sp + kvsel * sk + (pos % cfg.page_size) * ss)[:, None] + row[None, :])
+            flat = torch.from_numpy(np.concatenate([f.reshape(-1) for f in flats]))
+            dst = np.concatenate([d.reshape(-1) for d in dsts])
+            kv_small = np.zeros(n_small * sp, dtype=np.uint16)
+            kv_small[dst] = bf16.torch_to_bits(wl.kv_values(cfg.seed, j, flat))
+            self.prepared.append((kv_small, bt_small))
+        self.oi, self.oc = oi, oc
+        self.cores = oracle.num_threads()
+
+    def step_us(self):
+        cfg, si, oracle = self.cfg, self.si, self.oracle
+        t0 = time.perf_counter()
+        oi, oc, _, _ = oracle.select_topp(si.draft_probs, si.layer_map, si.kv_len, cfg.p)
+        t_sel = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        for j, (kv_bits, bt) in zip(self.layers, self.prepared):
+            u = int(si.layer_map[j])
+            oracle.sparse_verify(si.q[j], kv_bits, self.strides, bt, si.kv_len, oi[u], oc[u],
+                                 n_kv_heads=cfg.n_kv_heads, page_size=cfg.page_size)
+        t_attn = time.perf_counter() - t0
+        scale = cfg.n_target_layers / len(self.layers)
+        sample = (f"select: all {int((oc >= 0).sum())} lists of the step ({t_sel:.3f} s); attention: "
+                  f"{len(self.layers)} of {cfg.n_target_layers} target layers, all sequences and heads "
+                  f"({t_attn:.3f} s), scaled x{scale:g}")
+        return (t_sel + t_attn * scale) * 1e6, sample
+
+
+def run_reference(args, cfg):
+    import workloads as wl
+    rank, _, world = _rank_env()
+    if rank != 0:
+        return
+    si = wl.make_step_inputs(cfg)
+    smp = OracleSample(cfg, si, n_attn_layers=2)
+    vals, sample = [], ""
+    t_start = time.perf_counter()
+    for k in range(args.warmup + args.steps):
+        us, sample = smp.step_us()
+        if k >= args.warmup:
+            vals.append(us)
+    v = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": round(v, 1), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(v / 1e3, 3), "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "n_target_layers": cfg.n_target_layers,
+                       "n_draft_layers": cfg.n_draft_layers, "batch_per_gpu": cfg.batch,
+                       "global_batch": cfg.batch, "ctx": cfg.ctx, "page_size": cfg.page_size,
+                       "gamma": cfg.gamma, "p": cfg.p, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
+                       "head_dim": cfg.head_dim},
+            "cpu_baseline": {"value": round(v, 1), "unit": UNIT, "cores": smp.cores, "kind": "oracle",
+                             "sample": sample + f"; wall {time.perf_counter() - t_start:.1f} s for all steps"},
+            "e2e": {"value": round(v, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+def topp_sweep(dev, reps=10):
+    """Selection micro-benchmark: 256 rows x n x p x family, rows/s per cell (R = 1)."""
+    import torch
+    import paper_2510_27641_b200 as sa
+    import workloads as wl
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    out = {}
+    for fam in wl.TOPP_FAMILIES:
+        for n in wl.TOPP_SIZES:
+            rows = torch.from_numpy(wl.topp_rows(fam, 256, n, seed=2)).to(dev).view(256, 1, 1, n)
+            kv = torch.full((256,), n, dtype=torch.int32, device=dev)
+            idx = torch.empty((1, 256, 1, n), dtype=torch.int32, device=dev)
+            cnt = torch.empty((1, 256, 1), dtype=torch.int32, device=dev)
+            st = torch.empty((1, 256, 1), dtype=torch.int32, device=dev)
+            for p in wl.TOPP_PS:
+                ts = []
+                for r in range(reps + 3):
+                    flush.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    sa.select_topp([rows], kv, [0], p, idx=idx, counts=cnt, row_status=st)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if r >= 3:
+                        ts.append(e0.elapsed_time(e1) * 1e3)
+                us = float(np.median(ts))
+                out[f"{fam}/n={n}/p={p}"] = {"us": round(us, 2), "rows_per_s": round(256 / us * 1e6),
+                                             "gbs": round(256 * n * 4 / us / 1e3, 1),
+                                             "kept_mean": float(cnt.float().mean().item())}
+            del rows, idx
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--topp-sweep", action="store_true", help="also run the 256-row selection micro-benchmark")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of target layers (debug)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    import workloads as wl
+    cfg = wl.config1()
+    if args.layers:
+        cfg = cfg.scaled(n_target_layers=args.layers)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2510_27641_b200 as sa
+    rank, local_rank, world = _rank_env()
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    barrier = None
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+        barrier = lambda: (dist.barrier(), torch.cuda.synchronize())
+
+    # every rank owns a batch of its own (batch sharding): same shapes, rank-specific seed
+    cfg_r = cfg.scaled(seed=cfg.seed + 1000 * rank) if world > 1 else cfg
+    si, pools, step, dp_host, q_host = build_step(cfg_r, dev)
+    step.run()
+    torch.cuda.synchronize()
+    counts = step.counts.cpu().numpy()
+    assert int(step.status.abs().sum()) == 0 and int((step.row_status.cpu().numpy() > 0).sum()) == 0
+
+    g_step, n_step = capture(step.run)
+    g_verify, n_verify = capture(lambda: [step.run_verify(j) for j in range(step.n_layers)])
+    g_select, n_select = capture(step.run_select)
+
+    try:
+        uuid = str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        uuid = None
+    sampler = ClockSampler(local_rank, uuid)
+    with sampler:
+        us_step = time_replays(g_step, args.steps, args.warmup, barrier)
+        us_verify_all = time_replays(g_verify, args.steps, args.warmup)
+        us_select = time_replays(g_select, args.steps, args.warmup)
+    clocks = sampler.summary()
+
+    # eager launches (no graph) for comparison
+    for _ in range(3):
+        step.run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_eager = max(3, min(args.steps, 20))
+    e0.record()
+    for _ in range(n_eager):
+        step.run()
+    e1.record()
+    torch.cuda.synchronize()
+    us_eager = e0.elapsed_time(e1) * 1e3 / n_eager
+
+    # end to end from pinned host buffers through the C ABI
+    out_host = [torch.empty(o.shape, dtype=torch.float32).pin_memory() for o in step.out]
+    lse_host = [torch.empty(l.shape, dtype=torch.float32).pin_memory() for l in step.lse]
+    n_e2e = max(3, min(args.steps, 20))
+    for _ in range(3):
+        step.run_host(dp_host, q_host, out_host, lse_host)
+    torch.cuda.synchronize()
+    if barrier is not None:
+        barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n_e2e):
+        step.run_host(dp_host, q_host, out_host, lse_host)
+    e1.record()
+    torch.cuda.synchronize()
+    us_e2e = e0.elapsed_time(e1) * 1e3 / n_e2e
+    assert torch.equal(out_host[-1], step.out[-1].cpu())
+    h2d = sum(t.numel() * 4 for t in dp_host if t is not None) + sum(t.numel() * 2 for t in q_host)
+    d2h = sum(t.numel() * 4 for t in out_host) + sum(t.numel() * 4 for t in lse_host)
+
+    if world > 1:
+        t = torch.tensor([us_step, us_e2e, us_verify_all, us_select], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        us_step, us_e2e, us_verify_all, us_select = t.tolist()
+
+    # ---- roofline of the dominant kernel (sparse verify) -------------------------------------
+    per_layer = [verify_bytes(cfg_r, si, counts[int(u)]) for u in si.layer_map]
+    bytes_launch = float(np.mean([b for b, _ in per_layer]))
+    kv_bytes_step = sum(k for _, k in per_layer)
+    dense_kv_step = int(si.kv_len.astype(np.int64).sum()) * cfg.n_kv_heads * cfg.head_dim * 4 * cfg.n_target_layers
+    us_launch = us_verify_all / step.n_layers
+    peak, peak_kind = _measured_peaks()
+    achieved = bytes_launch / us_launch / 1e3
+    n_used = len(step.used)
+    sel_b = select_bytes(cfg_r, si, n_used, counts)
+    roofline = {"kernel": "sparse_verify_kernel<2,4>", "bound": "hbm", "achieved": round(achieved, 1),
+                "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
+                "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
+                "traffic": NCU_VERIFY_TRAFFIC_BYTES, "bytes_per_launch": round(bytes_launch),
+                "us_per_launch": round(us_launch, 3),
+                "select": {"kernel": "select_topp_kernel", "bytes_per_launch": sel_b, "us_per_launch": round(us_select, 3),
+                           "achieved": round(sel_b / us_select / 1e3, 1),
+                           "frac": round(sel_b / us_select / 1e3 / peak, 4)}}
+
+    line = {"metric": METRIC, "value": round(us_step, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(us_step / 1e3, 6), "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "n_target_layers": cfg.n_target_layers,
+                       "n_draft_layers": cfg.n_draft_layers, "batch_per_gpu": cfg.batch,
+                       "global_batch": cfg.batch * world, "ctx": cfg.ctx, "page_size": cfg.page_size,
+                       "gamma": cfg.gamma, "p": cfg.p, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
+                       "head_dim": cfg.head_dim, "parallelism": f"batch-sharded x{world}, no collective",
+                       "launch": "CUDA graph of 1 select + 32 verify launches",
+                       "l2": "inputs exceed L2: 252 MB of draft rows and 1.3 GB of gathered K/V per step"},
+            "e2e": {"value": round(us_e2e, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(n_step * args.steps),
+            "clocks": clocks, "roofline": roofline,
+            "extra": {"us_verify_per_step": round(us_verify_all, 3), "us_select_per_step": round(us_select, 3),
+                      "us_step_eager_launches": round(us_eager, 3),
+                      "topp_lists_per_s": round(n_used * cfg.batch / us_select * 1e6),
+                      "topp_prob_rows_per_s": round(n_used * cfg.batch * cfg.n_draft_heads * cfg.gamma / us_select * 1e6),
+                      "kept_mean": float(counts[counts >= 0].mean()),
+                      "kv_bytes_touched_per_step": int(kv_bytes_step), "kv_bytes_dense_per_step": int(dense_kv_step),
+                      "kv_touched_fraction": round(kv_bytes_step / dense_kv_step, 5),
+                      "sequences_per_s": round(cfg.batch * world / us_step * 1e6, 1)}}
+
+    if rank == 0 and not args.no_cpu_baseline:
+        smp = OracleSample(cfg_r, si, n_attn_layers=8, pools=pools)
+        us_cpu, sample = smp.step_us()
+        line["cpu_baseline"] = {"value": round(us_cpu, 1), "unit": UNIT, "cores": smp.cores, "kind": "oracle",
+                                "sample": sample}
+    if rank == 0 and args.topp_sweep:
+        del g_step, g_verify, g_select
+        line["extra"]["topp_sweep"] = topp_sweep(dev)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -506,9 +506,25 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   if (slice > specattn::kSliceCap) return SPECATTN_ERR_UNSUPPORTED;
   const size_t smem = ((sizeof(specattn::Shared) + 15) / 16) * 16 + static_cast<size_t>(slice) * sizeof(float) + 16;
 
-  cudaError_t err = cudaFuncSetAttribute(specattn::select_topp_kernel,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-  if (err != cudaSuccess) return SPECATTN_ERR_CUDA;
+  // Opt in to large dynamic shared memory once per device (the full slice capacity), so that
+  // later calls issue nothing but the launch.
+  cudaError_t err = cudaSuccess;
+  {
+    static std::atomic<unsigned long long> done_mask{0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPECATTN_ERR_CUDA;
+    if (!((done_mask.load(std::memory_order_acquire) >> dev) & 1ull)) {
+      const size_t max_smem = ((sizeof(specattn::Shared) + 15) / 16) * 16 +
+                              static_cast<size_t>(specattn::kSliceCap) * sizeof(float) + 16;
+      err = cudaFuncSetAttribute(specattn::select_topp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(max_smem));
+      if (err != cudaSuccess) {
+        cudaGetLastError();
+        return SPECATTN_ERR_CUDA;
+      }
+      done_mask.fetch_or(1ull << dev, std::memory_order_release);
+    }
+  }
 
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));

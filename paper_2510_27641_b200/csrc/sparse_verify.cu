@@ -531,9 +531,17 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
 template <int MT, int KS>
 cudaError_t launch(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
   const size_t smem = sizeof(VShared<MT, KS>) + 128;
-  cudaError_t err = cudaFuncSetAttribute(sparse_verify_kernel<MT, KS>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  static std::atomic<unsigned long long> done_mask{0};  // per device: shared-memory opt-in done
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (!((done_mask.load(std::memory_order_acquire) >> dev) & 1ull)) {
+    err = cudaFuncSetAttribute(sparse_verify_kernel<MT, KS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               static_cast<int>(smem));
+    if (err != cudaSuccess) return err;
+    done_mask.fetch_or(1ull << dev, std::memory_order_release);
+  }
   sparse_verify_kernel<MT, KS><<<n_ctas, (MT * KS + kProdWarps) * 32, smem, stream>>>(P);
   return cudaGetLastError();
 }
