@@ -36,7 +36,7 @@ extern std::atomic<long long> g_launch_count;
 
 namespace {
 
-constexpr int kThreads = 512;
+constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kL1Bins = 2048;        // sign(0) + 8 exponent bits + 3 mantissa bits
 constexpr int kL23Bins = 1024;       // 10 mantissa bits per later level
@@ -223,7 +223,7 @@ __device__ double scan_bins(Shared& sh, int nbins, double carry_mass, unsigned i
   return all;
 }
 
-__global__ void __launch_bounds__(kThreads, 1) select_topp_kernel(const __grid_constant__ SelectParams P) {
+__global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_constant__ SelectParams P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
   float* a = reinterpret_cast<float*>(smem_raw + ((sizeof(Shared) + 15) / 16) * 16);

@@ -11,14 +11,17 @@
 // and contiguously to one persistent CTA per SM, so ragged batches balance without any host
 // knowledge of the counts.  Inside a CTA
 //   - four producer warps resolve position -> (page, slot) through the block table and fetch
-//     each selected 256-byte K row and V row with one 1-D bulk async copy (TMA unit, no tensor
-//     map) into a padded, bank-conflict-free shared-memory tile; a 4-stage ring of 64-token
-//     tiles guarded by full/empty mbarriers keeps >100 KB of reads in flight per SM;
-//   - the consumer warps own one 16-row slab of the (gamma+1) x group query block and a share
-//     of every tile's keys: S = Q K^T and O += P V run on the tensor cores (bf16 mma.sync,
+//     each selected 256-byte K row and V row with 16-byte cp.async copies (16 lanes per row,
+//     completion counted on an mbarrier) into a padded, bank-conflict-free shared-memory tile;
+//     a 4-stage ring of 64-token tiles guarded by full/empty mbarriers keeps >100 KB of reads
+//     in flight per SM.  (One 1-D bulk copy per row was measured first: the TMA unit retires
+//     about one such 256-byte request per 19 cycles per SM, capping the gather near 3.4 TB/s.)
+//   - the consumer warps own one 16-row slab of the (gamma+1) x group query block; the warps of
+//     a slab take alternate tiles (and, four to a slab, one 32-key half of them), so each warp
+//     runs long independent chains: S = Q K^T and O += P V on the tensor cores (bf16 mma.sync,
 //     fp32 accumulate; P is split into two bf16 terms so that it carries 16 mantissa bits),
 //     online softmax in fp32 registers in the log2 domain;
-//   - at the end of a unit the key-split warps combine through shared memory; a unit that was
+//   - at the end of a unit the warps of a slab combine through shared memory; a unit that was
 //     cut between CTAs is finished by whichever CTA arrives last at the unit's counter, which
 //     merges all partial (O, m, l) records in a fixed order -- nobody ever waits on a peer.
 // Every mbarrier wait is bounded; on expiry the CTA flags SPECATTN_ROW_TIMEOUT and leaves.
@@ -74,11 +77,12 @@ struct VerifyParams {
   float* partials;
 };
 
-template <int MT, int KS>
+// WPM = consumer warps per 16-row slab: 4 -> (stage parity, 32-key half), 2 -> (stage parity).
+template <int MT, int WPM>
 struct VShared {
   alignas(128) unsigned char kv[kStages][2][kStageTok * kPitch];
   alignas(16) unsigned char q[MT * 16 * kPitch];
-  float scratch[MT][(KS / 2 > 0) ? KS / 2 : 1][kRec];
+  float scratch[MT][WPM / 2][kRec];
   alignas(8) unsigned long long full[kStages];
   unsigned long long empty[kStages];
   unsigned long long q_full, q_empty;
@@ -120,13 +124,110 @@ __device__ __forceinline__ void merge_scales(float m, float im, float& mn, float
   a_in = ex2(im - base);
 }
 
-template <int MT, int KS>
-__global__ void __launch_bounds__((MT * KS + kProdWarps) * 32, 1)
+// Online-softmax state of one warp: rows g and g+8 of its 16-row slab, 128 output columns.
+struct WarpState {
+  float acc[16][4];
+  float m0, m1, l0, l1;
+};
+
+// One 32-key block: S = Q K^T (4 n-tiles), online softmax, O += P V with P = P_hi + P_lo.
+// `valid` = number of existing keys in the block (>= 1; rows beyond it hold finite padding).
+__device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&qf)[8][4], uint32_t k_addr,
+                                               uint32_t v_addr, int valid, float scale_log2, int tq) {
+  float sc[4][4];
+#pragma unroll
+  for (int n = 0; n < 4; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) {
+    uint32_t k0[4], k1[4];
+    ldmatrix_x4(k0, k_addr + kk * 32);
+    ldmatrix_x4(k1, k_addr + 16 * kPitch + kk * 32);
+    mma_bf16(sc[0], qf[kk], k0[0], k0[1]);
+    mma_bf16(sc[1], qf[kk], k0[2], k0[3]);
+    mma_bf16(sc[2], qf[kk], k1[0], k1[1]);
+    mma_bf16(sc[3], qf[kk], k1[2], k1[3]);
+  }
+#pragma unroll
+  for (int n = 0; n < 4; ++n)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int key = n * 8 + tq * 2 + (i & 1);
+      sc[n][i] = (key < valid) ? sc[n][i] * scale_log2 : -INFINITY;
+    }
+  float mx0 = fmaxf(fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])),
+                    fmaxf(fmaxf(sc[2][0], sc[2][1]), fmaxf(sc[3][0], sc[3][1])));
+  float mx1 = fmaxf(fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3])),
+                    fmaxf(fmaxf(sc[2][2], sc[2][3]), fmaxf(sc[3][2], sc[3][3])));
+  mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+  mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+  mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+  mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+  const float mn0 = fmaxf(st.m0, mx0), mn1 = fmaxf(st.m1, mx1);
+  const float base0 = (mn0 == -INFINITY) ? 0.f : mn0;
+  const float base1 = (mn1 == -INFINITY) ? 0.f : mn1;
+  const float al0 = ex2(st.m0 - base0), al1 = ex2(st.m1 - base1);
+  st.m0 = mn0;
+  st.m1 = mn1;
+  float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+  for (int n = 0; n < 4; ++n) {
+    sc[n][0] = ex2(sc[n][0] - base0);
+    sc[n][1] = ex2(sc[n][1] - base0);
+    sc[n][2] = ex2(sc[n][2] - base1);
+    sc[n][3] = ex2(sc[n][3] - base1);
+    s0 += sc[n][0] + sc[n][1];
+    s1 += sc[n][2] + sc[n][3];
+  }
+  st.l0 = st.l0 * al0 + s0;
+  st.l1 = st.l1 * al1 + s1;
+  if (__any_sync(0xffffffffu, al0 != 1.f || al1 != 1.f)) {
+#pragma unroll
+    for (int n = 0; n < 16; ++n) {
+      st.acc[n][0] *= al0;
+      st.acc[n][1] *= al0;
+      st.acc[n][2] *= al1;
+      st.acc[n][3] *= al1;
+    }
+  }
+  // A-operand fragments of P for the two 16-key halves, each as a bf16 pair (hi, lo)
+  uint32_t phi[2][4], plo[2][4];
+#pragma unroll
+  for (int kb = 0; kb < 2; ++kb)
+#pragma unroll
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+      for (int hrow = 0; hrow < 2; ++hrow) {
+        const float x = sc[kb * 2 + n][hrow * 2], y = sc[kb * 2 + n][hrow * 2 + 1];
+        const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
+        __nv_bfloat162 hi2;
+        hi2.x = xh;
+        hi2.y = yh;
+        phi[kb][n * 2 + hrow] = *reinterpret_cast<uint32_t*>(&hi2);
+        plo[kb][n * 2 + hrow] = pack_bf16(x - __bfloat162float(xh), y - __bfloat162float(yh));
+      }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    uint32_t v0[4], v1[4];
+    ldmatrix_x4_trans(v0, v_addr + j * 32);
+    ldmatrix_x4_trans(v1, v_addr + 16 * kPitch + j * 32);
+    mma_bf16(st.acc[2 * j], phi[0], v0[0], v0[1]);
+    mma_bf16(st.acc[2 * j + 1], phi[0], v0[2], v0[3]);
+    mma_bf16(st.acc[2 * j], phi[1], v1[0], v1[1]);
+    mma_bf16(st.acc[2 * j + 1], phi[1], v1[2], v1[3]);
+    mma_bf16(st.acc[2 * j], plo[0], v0[0], v0[1]);
+    mma_bf16(st.acc[2 * j + 1], plo[0], v0[2], v0[3]);
+    mma_bf16(st.acc[2 * j], plo[1], v1[0], v1[1]);
+    mma_bf16(st.acc[2 * j + 1], plo[1], v1[2], v1[3]);
+  }
+}
+
+template <int MT, int WPM>
+__global__ void __launch_bounds__((MT * WPM + kProdWarps) * 32, 1)
 sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
-  using Sh = VShared<MT, KS>;
-  constexpr int NC = MT * KS;                  // consumer warps
+  using Sh = VShared<MT, WPM>;
+  constexpr int NC = MT * WPM;                 // consumer warps
   constexpr int NT = (NC + kProdWarps) * 32;   // threads
-  constexpr int KPW = kStageTok / KS;          // keys per consumer warp per stage
+  constexpr int NCS = MT * (WPM / 2);          // consumer warps that read any one stage
   extern __shared__ __align__(128) unsigned char smem_raw[];
   Sh& sh = *reinterpret_cast<Sh*>(smem_raw);
 
@@ -135,17 +236,15 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   const int warp = tid >> 5;
   const int U = P.B * P.Hkv;
 
-  // ---- set-up: zero the tiles (stale rows must stay finite), barriers, unit prefix ------------
+  // ---- set-up: barriers, zero padding rows of the query tile, unit prefix ---------------------
   {
-    uint4* z = reinterpret_cast<uint4*>(sh.kv);
-    for (int i = tid; i < static_cast<int>(sizeof(sh.kv) / 16); i += NT) z[i] = make_uint4(0u, 0u, 0u, 0u);
     uint4* zq = reinterpret_cast<uint4*>(sh.q);
     for (int i = tid; i < static_cast<int>(sizeof(sh.q) / 16); i += NT) zq[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&sh.full[s], 1);
-      mbar_init(&sh.empty[s], NC);
+      mbar_init(&sh.full[s], 32);   // one deferred arrival per producer lane
+      mbar_init(&sh.empty[s], NCS);
     }
     mbar_init(&sh.q_full, 1);
     mbar_init(&sh.q_empty, NC);
@@ -240,25 +339,43 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         const unsigned ph = (it / kStages) & 1u;
         if (!mbar_wait(&sh.empty[s], ph ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
         const int ntok = min(kStageTok, tok_hi - t0);
-        if (lane == 0) mbar_arrive_expect_tx(&sh.full[s], static_cast<uint32_t>(ntok) * 2u * kRowBytes);
-        __syncwarp();
+        // The tail of a segment is padded to a whole 32-key block with copies of its last
+        // token, so that every row a consumer multiplies by a zero weight holds finite data.
+        const int npad = (ntok + 31) & ~31;
+        // lane j resolves tokens j and j + 32 to the byte offset of their K row
+        long long off[2];
         bool bad = false;
 #pragma unroll
-        for (int jj = 0; jj < kStageTok / 32; ++jj) {
-          const int j = lane + jj * 32;
-          if (j < ntok) {
-            int pos = P.dense ? (t0 + j) : __ldg(list + t0 + j);
-            if (pos < 0 || pos >= kvlen_b) { bad = true; pos = 0; }
-            const int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
-            const int slot = pos - lp * P.page_size;
-            long long page = P.bt ? static_cast<long long>(__ldg(P.bt + b * P.bt_stride + lp))
-                                  : (b * P.bt_stride + lp);
-            if (page < 0 || (P.n_pages > 0 && page >= P.n_pages)) { bad = true; page = 0; }
-            const __nv_bfloat16* src = kv_head + page * P.s_page + static_cast<long long>(slot) * P.s_slot;
-            bulk_g2s(sh.kv[s][0] + j * kPitch, src, kRowBytes, &sh.full[s]);
-            bulk_g2s(sh.kv[s][1] + j * kPitch, src + P.s_kv, kRowBytes, &sh.full[s]);
+        for (int jj = 0; jj < 2; ++jj) {
+          const int jt = min(lane + jj * 32, ntok - 1);
+          int pos = P.dense ? (t0 + jt) : __ldg(list + t0 + jt);
+          if (pos < 0 || pos >= kvlen_b) { bad = true; pos = 0; }
+          const int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
+          const int slot = pos - lp * P.page_size;
+          long long page = P.bt ? static_cast<long long>(__ldg(P.bt + b * P.bt_stride + lp))
+                                : (b * P.bt_stride + lp);
+          if (page < 0 || (P.n_pages > 0 && page >= P.n_pages)) { bad = true; page = 0; }
+          off[jj] = (page * P.s_page + static_cast<long long>(slot) * P.s_slot) * 2;
+        }
+        // 16 lanes move one 256-byte row with 16-byte cp.async copies: a warp instruction
+        // fetches two rows (four full 128-byte lines)
+        const char* kbase = reinterpret_cast<const char*>(kv_head) + (lane & 15) * 16;
+        const long long v_delta = P.s_kv * 2;
+        const uint32_t k_dst = smem_u32(sh.kv[s][0]) + (lane >> 4) * kPitch + (lane & 15) * 16;
+        const uint32_t v_dst = smem_u32(sh.kv[s][1]) + (lane >> 4) * kPitch + (lane & 15) * 16;
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj) {
+#pragma unroll 4
+          for (int i = 0; i < 16; ++i) {
+            const int tok = jj * 32 + 2 * i + (lane >> 4);
+            const long long o = __shfl_sync(0xffffffffu, off[jj], 2 * i + (lane >> 4));
+            if (tok < npad) {
+              cp_async16(k_dst + (jj * 32 + 2 * i) * kPitch, kbase + o);
+              cp_async16(v_dst + (jj * 32 + 2 * i) * kPitch, kbase + o + v_delta);
+            }
           }
         }
+        cp_async_mbar_arrive_noinc(&sh.full[s]);
         if (bad && P.status) atomicOr(P.status + b, SPECATTN_ROW_BAD_INDEX);
         last_it = it;
       }
@@ -277,8 +394,9 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   }
 
   // =============================== consumer warps ===========================================
-  const int mt = warp / KS;   // 16-row slab of the query block
-  const int ks = warp % KS;   // share of each tile's keys
+  const int mt = warp / WPM;            // 16-row slab of the query block
+  const int wr = warp % WPM;            // role inside the slab
+  const int parity = (WPM == 4) ? (wr >> 1) : wr;   // which stages (it % 2) this warp reads
   const int g = lane >> 2, tq = lane & 3;
   const int lm = lane >> 3, lr = lane & 7;  // ldmatrix: matrix id, row within it
   const uint32_t q_addr = smem_u32(sh.q) + (mt * 16 + (lm & 1) * 8 + lr) * kPitch + (lm >> 1) * 16;
@@ -288,7 +406,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
 
   // A warp that meets a failed wait raises abort_flag and stops computing, but still walks
   // through the combine barriers of the segment it is in; every warp re-reads the flag right
-  // after those barriers, so a whole key-split group always leaves together.
+  // after those barriers, so a whole slab group always leaves together.
   int it = 0, seg = 0;
   int a = a0, u = u_first;
   bool ok = true;
@@ -308,108 +426,44 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     __syncwarp();
     if (ok && lane == 0) mbar_arrive(&sh.q_empty);
 
-    float acc[16][4];
+    WarpState st;
 #pragma unroll
-    for (int n = 0; n < 16; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    for (int n = 0; n < 16; ++n) st.acc[n][0] = st.acc[n][1] = st.acc[n][2] = st.acc[n][3] = 0.f;
+    st.m0 = st.m1 = -INFINITY;
+    st.l0 = st.l1 = 0.f;
 
     for (int t0 = tok_lo; ok && t0 < tok_hi; t0 += kStageTok, ++it) {
+      if ((it & 1) != parity) continue;
       const int s = it % kStages;
       const unsigned ph = (it / kStages) & 1u;
       if (!mbar_wait(&sh.full[s], ph, &sh.abort_flag)) { sh.abort_flag = 1; ok = false; break; }
       const int ntok = min(kStageTok, tok_hi - t0);
-      const uint32_t k_base = smem_u32(sh.kv[s][0]);
-      const uint32_t v_base = smem_u32(sh.kv[s][1]);
-#pragma unroll
-      for (int sub = 0; sub < KPW / 16; ++sub) {
-        const int key0 = ks * KPW + sub * 16;
-        if (key0 >= ntok) break;
-        const int valid = ntok - key0;  // keys of this 16-block that exist (may exceed 16)
-        float sc[2][4];
-#pragma unroll
-        for (int n = 0; n < 2; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          uint32_t kf[4];
-          ldmatrix_x4(kf, k_base + key0 * kPitch + k_off + kk * 32);
-          mma_bf16(sc[0], qf[kk], kf[0], kf[1]);
-          mma_bf16(sc[1], qf[kk], kf[2], kf[3]);
-        }
-#pragma unroll
-        for (int n = 0; n < 2; ++n)
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const int key = n * 8 + tq * 2 + (i & 1);
-            sc[n][i] = (key < valid) ? sc[n][i] * P.scale_log2 : -INFINITY;
-          }
-        float mx0 = fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1]));
-        float mx1 = fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3]));
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
-        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
-        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-        const float base0 = (mn0 == -INFINITY) ? 0.f : mn0;
-        const float base1 = (mn1 == -INFINITY) ? 0.f : mn1;
-        const float al0 = ex2(m0 - base0), al1 = ex2(m1 - base1);
-        m0 = mn0;
-        m1 = mn1;
-        float p[2][4];
-#pragma unroll
-        for (int n = 0; n < 2; ++n) {
-          p[n][0] = ex2(sc[n][0] - base0);
-          p[n][1] = ex2(sc[n][1] - base0);
-          p[n][2] = ex2(sc[n][2] - base1);
-          p[n][3] = ex2(sc[n][3] - base1);
-        }
-        l0 = l0 * al0 + (p[0][0] + p[0][1] + p[1][0] + p[1][1]);
-        l1 = l1 * al1 + (p[0][2] + p[0][3] + p[1][2] + p[1][3]);
-#pragma unroll
-        for (int n = 0; n < 16; ++n) {
-          acc[n][0] *= al0;
-          acc[n][1] *= al0;
-          acc[n][2] *= al1;
-          acc[n][3] *= al1;
-        }
-        // P = P_hi + P_lo, two bf16 terms
-        uint32_t phi[4], plo[4];
-#pragma unroll
-        for (int n = 0; n < 2; ++n) {
-#pragma unroll
-          for (int hrow = 0; hrow < 2; ++hrow) {
-            const float x = p[n][hrow * 2], y = p[n][hrow * 2 + 1];
-            const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
-            const float xr = x - __bfloat162float(xh), yr = y - __bfloat162float(yh);
-            __nv_bfloat162 hi2;
-            hi2.x = xh;
-            hi2.y = yh;
-            phi[n * 2 + hrow] = *reinterpret_cast<uint32_t*>(&hi2);
-            plo[n * 2 + hrow] = pack_bf16(xr, yr);
-          }
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          uint32_t vf[4];
-          ldmatrix_x4_trans(vf, v_base + key0 * kPitch + v_off + j * 32);
-          mma_bf16(acc[2 * j], phi, vf[0], vf[1]);
-          mma_bf16(acc[2 * j + 1], phi, vf[2], vf[3]);
-          mma_bf16(acc[2 * j], plo, vf[0], vf[1]);
-          mma_bf16(acc[2 * j + 1], plo, vf[2], vf[3]);
-        }
+      const uint32_t k_base = smem_u32(sh.kv[s][0]) + k_off;
+      const uint32_t v_base = smem_u32(sh.kv[s][1]) + v_off;
+      if (WPM == 4) {
+        const int key0 = (wr & 1) * 32;
+        if (key0 < ntok)
+          attend_block32(st, qf, k_base + key0 * kPitch, v_base + key0 * kPitch, ntok - key0, P.scale_log2, tq);
+      } else {
+        attend_block32(st, qf, k_base, v_base, ntok, P.scale_log2, tq);
+        if (32 < ntok)
+          attend_block32(st, qf, k_base + 32 * kPitch, v_base + 32 * kPitch, ntok - 32, P.scale_log2, tq);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.empty[s]);
     }
 
-    // ---- end of the segment: row sums across the quad, then combine the key-split warps ------
+    // ---- end of the segment: row sums across the quad, then combine the slab's warps ---------
+    float m0 = st.m0, m1 = st.m1, l0 = st.l0, l1 = st.l1;
+    float (&acc)[16][4] = st.acc;
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
     l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
     l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
 #pragma unroll
-    for (int half = KS / 2; half >= 1; half >>= 1) {
-      if (ks >= half && ks < 2 * half) {
-        float* rec = sh.scratch[mt][ks - half];
+    for (int half = WPM / 2; half >= 1; half >>= 1) {
+      if (wr >= half && wr < 2 * half) {
+        float* rec = sh.scratch[mt][wr - half];
 #pragma unroll
         for (int n = 0; n < 16; ++n)
 #pragma unroll
@@ -419,9 +473,9 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         rec[66 * 32 + lane] = m1;
         rec[67 * 32 + lane] = l1;
       }
-      named_bar_sync(1 + mt, KS * 32);
-      if (ks < half) {
-        const float* rec = sh.scratch[mt][ks];
+      named_bar_sync(1 + mt, WPM * 32);
+      if (wr < half) {
+        const float* rec = sh.scratch[mt][wr];
         float mn, ao, ai;
         merge_scales(m0, rec[64 * 32 + lane], mn, ao, ai);
         l0 = l0 * ao + rec[65 * 32 + lane] * ai;
@@ -438,12 +492,11 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           acc[n][3] = acc[n][3] * ao1 + rec[(n * 4 + 3) * 32 + lane] * ai1;
         }
       }
-      named_bar_sync(1 + mt, KS * 32);
+      named_bar_sync(1 + mt, WPM * 32);
     }
-
     if (sh.abort_flag) { ok = false; break; }
 
-    if (ks == 0) {
+    if (wr == 0) {
       const bool whole = (a == us) && (seg_hi == ue);
       bool finish = whole;
       if (!whole) {
@@ -466,28 +519,33 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         if (old == static_cast<unsigned int>(i_hi - i_lo)) {
           finish = true;
           __threadfence();
-          // merge every contributor's record in CTA order (the own one included, from memory)
+          // Merge every contributor's record in CTA order (the own one included, read back
+          // from memory, so the result does not depend on who arrived last).  First the
+          // common maxima, then one scaled accumulation pass with independent loads.
           m0 = m1 = -INFINITY;
+          for (int i = i_lo; i <= i_hi; ++i) {
+            const float* r2 = P.partials +
+                (static_cast<size_t>(2 * i + (cta_first_atom(i, N, NP) >= us ? 0 : 1)) * MT + mt) * kRec;
+            m0 = fmaxf(m0, __ldcg(r2 + 64 * 32 + lane));
+            m1 = fmaxf(m1, __ldcg(r2 + 66 * 32 + lane));
+          }
+          const float base0 = (m0 == -INFINITY) ? 0.f : m0, base1 = (m1 == -INFINITY) ? 0.f : m1;
           l0 = l1 = 0.f;
 #pragma unroll
           for (int n = 0; n < 16; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
           for (int i = i_lo; i <= i_hi; ++i) {
-            const int first_atom = cta_first_atom(i, N, NP);
-            const float* r2 = P.partials + (static_cast<size_t>(2 * i + (first_atom >= us ? 0 : 1)) * MT + mt) * kRec;
-            float mn, ao, ai;
-            merge_scales(m0, __ldcg(r2 + 64 * 32 + lane), mn, ao, ai);
-            l0 = l0 * ao + __ldcg(r2 + 65 * 32 + lane) * ai;
-            m0 = mn;
-            float mn1, ao1, ai1;
-            merge_scales(m1, __ldcg(r2 + 66 * 32 + lane), mn1, ao1, ai1);
-            l1 = l1 * ao1 + __ldcg(r2 + 67 * 32 + lane) * ai1;
-            m1 = mn1;
+            const float* r2 = P.partials +
+                (static_cast<size_t>(2 * i + (cta_first_atom(i, N, NP) >= us ? 0 : 1)) * MT + mt) * kRec;
+            const float w0 = ex2(__ldcg(r2 + 64 * 32 + lane) - base0);
+            const float w1 = ex2(__ldcg(r2 + 66 * 32 + lane) - base1);
+            l0 += __ldcg(r2 + 65 * 32 + lane) * w0;
+            l1 += __ldcg(r2 + 67 * 32 + lane) * w1;
 #pragma unroll
             for (int n = 0; n < 16; ++n) {
-              acc[n][0] = acc[n][0] * ao + __ldcg(r2 + (n * 4 + 0) * 32 + lane) * ai;
-              acc[n][1] = acc[n][1] * ao + __ldcg(r2 + (n * 4 + 1) * 32 + lane) * ai;
-              acc[n][2] = acc[n][2] * ao1 + __ldcg(r2 + (n * 4 + 2) * 32 + lane) * ai1;
-              acc[n][3] = acc[n][3] * ao1 + __ldcg(r2 + (n * 4 + 3) * 32 + lane) * ai1;
+              acc[n][0] += __ldcg(r2 + (n * 4 + 0) * 32 + lane) * w0;
+              acc[n][1] += __ldcg(r2 + (n * 4 + 1) * 32 + lane) * w0;
+              acc[n][2] += __ldcg(r2 + (n * 4 + 2) * 32 + lane) * w1;
+              acc[n][3] += __ldcg(r2 + (n * 4 + 3) * 32 + lane) * w1;
             }
           }
           if (lane == 0) P.counters[u * kCountersPerUnit + mt] = 0u;  // ready for the next call
@@ -528,21 +586,21 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   if (!ok && P.status && lane == 0) atomicOr(P.status, SPECATTN_ROW_TIMEOUT);
 }
 
-template <int MT, int KS>
+template <int MT, int WPM>
 cudaError_t launch(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
-  const size_t smem = sizeof(VShared<MT, KS>) + 128;
+  const size_t smem = sizeof(VShared<MT, WPM>) + 128;
   static std::atomic<unsigned long long> done_mask{0};  // per device: shared-memory opt-in done
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   if (!((done_mask.load(std::memory_order_acquire) >> dev) & 1ull)) {
-    err = cudaFuncSetAttribute(sparse_verify_kernel<MT, KS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    err = cudaFuncSetAttribute(sparse_verify_kernel<MT, WPM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                static_cast<int>(smem));
     if (err != cudaSuccess) return err;
     done_mask.fetch_or(1ull << dev, std::memory_order_release);
   }
-  sparse_verify_kernel<MT, KS><<<n_ctas, (MT * KS + kProdWarps) * 32, smem, stream>>>(P);
+  sparse_verify_kernel<MT, WPM><<<n_ctas, (MT * WPM + kProdWarps) * 32, smem, stream>>>(P);
   return cudaGetLastError();
 }
 
