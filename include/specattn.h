@@ -148,6 +148,20 @@ int specattn_select_topp(const specattn_select_args* args, void* cuda_stream);
  * once with specattn_verify_workspace_init() and then reusable by consecutive calls on the
  * same stream; two calls that may overlap on the GPU need separate workspaces.
  * ======================================================================================== */
+/* flags for specattn_verify_args.flags
+ *
+ * SPECATTN_VERIFY_LISTS_STABLE: the caller promises that idx, counts, kv_len, block_table and
+ * the listed rows of kv_pages were produced at least two launches earlier in the stream, and
+ * that the launch right before this call is either another specattn_sparse_verify call or a
+ * kernel that does not signal programmatic launch completion early.  (True for every layer
+ * after the first of a step: the lists come from specattn_select_topp and the context's K/V
+ * rows are old.)  The verify kernel is always launched with programmatic stream
+ * serialization, i.e. it may begin while the preceding kernel is still running.  Without this
+ * flag it waits for that kernel to finish before reading anything, and lets its own successor
+ * start only after that wait; with it, it starts fetching K/V rows at once and waits only
+ * before reading q and before writing out, lse, status or the workspace. */
+#define SPECATTN_VERIFY_LISTS_STABLE 1u
+
 typedef struct specattn_verify_args {
   uint32_t struct_size;
   int32_t batch;
@@ -174,6 +188,7 @@ typedef struct specattn_verify_args {
   int32_t* status;       /* [batch] or NULL */
   void* workspace;
   size_t workspace_bytes;
+  uint32_t flags;        /* SPECATTN_VERIFY_* bits, 0 for none */
 } specattn_verify_args;
 
 /* Bytes of workspace specattn_sparse_verify needs for these shapes on the current device

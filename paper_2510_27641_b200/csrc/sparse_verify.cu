@@ -75,6 +75,7 @@ struct VerifyParams {
   int* status;
   unsigned int* counters;
   float* partials;
+  int lists_stable;  // SPECATTN_VERIFY_LISTS_STABLE
 };
 
 // WPM = consumer warps per 16-row slab: 4 -> (stage parity, 32-key half), 2 -> (stage parity).
@@ -236,6 +237,12 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   const int warp = tid >> 5;
   const int U = P.B * P.Hkv;
 
+  // Unless the caller vouched for the lists, nothing is read before the previous kernel is
+  // done.  Only then may the next kernel of the stream be scheduled: a successor that starts
+  // early therefore never overtakes the producer of the lists.
+  if (!P.lists_stable) pdl_wait();
+  pdl_launch_dependents();
+
   // ---- set-up: barriers, zero padding rows of the query tile, unit prefix ---------------------
   {
     uint4* zq = reinterpret_cast<uint4*>(sh.q);
@@ -275,19 +282,23 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   }
   __syncthreads();
 
-  // units with an empty list: out = 0, lse = -inf
-  for (int u = blockIdx.x; u < U; u += gridDim.x) {
-    if (sh.unit_cnt[u] != 0) continue;
-    const int b = u / P.Hkv, kvh = u % P.Hkv;
-    for (int e = tid; e < P.M * kD; e += NT) {
-      const int r = e / kD, t = r / P.grp, h = kvh * P.grp + r % P.grp;
-      P.out[((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD + e % kD] = 0.f;
-      if (e % kD == 0) P.lse[(static_cast<long long>(b) * P.T + t) * P.Hq + h] = -INFINITY;
-    }
-  }
-
   const long long N = sh.unit_start[U];
   const long long NP = (N < static_cast<long long>(gridDim.x)) ? N : static_cast<long long>(gridDim.x);
+  if (warp < NC) {
+    // consumers are the only writers of global memory: from here on the previous kernel's
+    // results (and its use of the shared workspace) are complete
+    if (P.lists_stable) pdl_wait();
+    // units with an empty list: out = 0, lse = -inf
+    for (int u = blockIdx.x; u < U; u += gridDim.x) {
+      if (sh.unit_cnt[u] != 0) continue;
+      const int b = u / P.Hkv, kvh = u % P.Hkv;
+      for (int e = tid; e < P.M * kD; e += NC * 32) {
+        const int r = e / kD, t = r / P.grp, h = kvh * P.grp + r % P.grp;
+        P.out[((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD + e % kD] = 0.f;
+        if (e % kD == 0) P.lse[(static_cast<long long>(b) * P.T + t) * P.Hq + h] = -INFINITY;
+      }
+    }
+  }
   if (static_cast<long long>(blockIdx.x) >= NP) return;
   const int a0 = cta_first_atom(blockIdx.x, N, NP);
   const int a1 = cta_first_atom(blockIdx.x + 1, N, NP);
@@ -321,10 +332,13 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       const int* list = P.dense ? nullptr
                                 : P.idx + (static_cast<long long>(b) * P.G + ((P.G == 1) ? 0 : kvh)) * P.idx_stride;
       const __nv_bfloat16* kv_head = P.kv + static_cast<long long>(kvh) * P.s_head;
-      if (pw == 0) {
-        // The query block of this unit: M rows of 256 bytes.  Always the same warp, walking
-        // the segments in order, so its parity wait can never be satisfied by a stale phase.
-        if (!mbar_wait(&sh.q_empty, (seg & 1u) ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
+      // The query block of this unit (M rows of 256 bytes) is always fetched by producer warp
+      // 0, walking the segments in order, so its parity wait can never be satisfied by a
+      // stale phase.  For the first segment it goes out after the warp's first tile, so that
+      // K/V prefetch is already in flight while the warp waits for the previous kernel.
+      auto load_q = [&]() -> bool {
+        if (seg == 0 && P.lists_stable) pdl_wait();
+        if (!mbar_wait(&sh.q_empty, (seg & 1u) ^ 1u, &sh.abort_flag)) return false;
         if (lane == 0) mbar_arrive_expect_tx(&sh.q_full, static_cast<uint32_t>(P.M) * kRowBytes);
         __syncwarp();
         for (int r = lane; r < P.M; r += 32) {
@@ -332,6 +346,12 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           bulk_g2s(sh.q + r * kPitch, P.q + ((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD,
                    kRowBytes, &sh.q_full);
         }
+        return true;
+      };
+      bool q_pending = (pw == 0);
+      if (q_pending && seg > 0) {
+        q_pending = false;
+        if (!load_q()) { sh.abort_flag = 1; dead = true; break; }
       }
       for (int t0 = tok_lo; t0 < tok_hi; t0 += kStageTok, ++it) {
         if ((it % kProdWarps) != pw) continue;
@@ -376,6 +396,10 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           }
         }
         cp_async_mbar_arrive_noinc(&sh.full[s]);
+        if (q_pending) {
+          q_pending = false;
+          if (!load_q()) { sh.abort_flag = 1; dead = true; break; }
+        }
         if (bad && P.status) atomicOr(P.status + b, SPECATTN_ROW_BAD_INDEX);
         last_it = it;
       }
@@ -600,8 +624,20 @@ cudaError_t launch(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
     if (err != cudaSuccess) return err;
     done_mask.fetch_or(1ull << dev, std::memory_order_release);
   }
-  sparse_verify_kernel<MT, WPM><<<n_ctas, (MT * WPM + kProdWarps) * 32, smem, stream>>>(P);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(static_cast<unsigned>(n_ctas), 1, 1);
+  cfg.blockDim = dim3((MT * WPM + kProdWarps) * 32, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  err = cudaLaunchKernelEx(&cfg, sparse_verify_kernel<MT, WPM>, P);
+  if (err != cudaSuccess) cudaGetLastError();
+  return err;
 }
 
 int m_tiles(const specattn_verify_args& A) {
@@ -699,6 +735,7 @@ extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cu
   P.lse = A.lse;
   P.status = A.status;
   P.counters = static_cast<unsigned int*>(A.workspace);
+  P.lists_stable = (A.flags & SPECATTN_VERIFY_LISTS_STABLE) ? 1 : 0;
   P.partials = reinterpret_cast<float*>(static_cast<unsigned char*>(A.workspace) + specattn::kCounterBytes);
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -10,7 +10,7 @@ from typing import Sequence
 
 import torch
 
-from . import (SelectArgs, VerifyArgs, SpecAttnError, lib, make_select_args, make_verify_args,
+from . import (SelectArgs, VerifyArgs, SpecAttnError, VERIFY_LISTS_STABLE, lib, make_select_args, make_verify_args,
                verify_step_host, verify_workspace, _stream_ptr)
 
 __all__ = ["VerifyStep"]
@@ -55,7 +55,10 @@ class VerifyStep:
                                  pages_per_seq=pages_per_seq,
                                  idx=None if u < 0 else self.idx[u], counts=None if u < 0 else self.counts[u],
                                  n_groups=n_groups, dense=u < 0, sm_scale=sm_scale, out=self.out[j],
-                                 lse=self.lse[j], status=self.status[j])
+                                 lse=self.lse[j], status=self.status[j],
+                                 # after the first layer the lists (written by select) and the
+                                 # context's K/V rows predate the preceding launch
+                                 flags=VERIFY_LISTS_STABLE if j > 0 else 0)
             if self.workspace is None:
                 self.workspace = verify_workspace(a, dev)
             a.workspace, a.workspace_bytes = self.workspace.data_ptr(), self.workspace.numel()
