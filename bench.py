@@ -39,8 +39,8 @@ UNIT = "us/step"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per sparse_verify launch on this workload, from
-# the ncu capture summarised in profiles/sparse_verify_cfg1.md (None until captured).
-NCU_VERIFY_TRAFFIC_BYTES = None
+# the ncu capture summarised in profiles/sparse_verify_cfg1.md.
+NCU_VERIFY_TRAFFIC_BYTES = 40.85e6
 
 
 # ----------------------------------------------------------------------------------------------

@@ -53,6 +53,8 @@ constexpr int kAtom = 16;
 constexpr int kMaxUnits = SPECATTN_MAX_VERIFY_UNITS;
 constexpr int kRec = 68 * 32;  // floats of one warp's (acc[64], m0, l0, m1, l1) record, lane-major
 constexpr int kCountersPerUnit = 4;
+constexpr int kAlignedMaxUnits = 256;  // the unit-aligned partition is tried up to this many units
+constexpr int kCandidates = 8;         // candidate target shares tried for it
 constexpr size_t kCounterBytes = static_cast<size_t>(kMaxUnits) * kCountersPerUnit * sizeof(unsigned int);
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -89,6 +91,10 @@ struct VShared {
   unsigned long long q_full, q_empty;
   int unit_start[kMaxUnits + 1];
   int unit_cnt[kMaxUnits];
+  int part_start[kAlignedMaxUnits + 1];  // aligned partition: first CTA of each unit
+  int cand_parts[kCandidates];           // per candidate share: total parts, largest part
+  int cand_max[kCandidates];
+  int aligned;                           // 1: unit-aligned partition, 0: contiguous atoms
   volatile int abort_flag;
 };
 
@@ -282,8 +288,73 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   }
   __syncthreads();
 
+  // ---- work partition ----------------------------------------------------------------------
+  // Two ways of dealing the N atoms to the CTAs.  "Aligned": every unit is cut into k_u equal
+  // parts, k_u = round(atoms_u / share), one part per CTA -- each CTA then touches one unit
+  // only and a unit is merged from k_u records; chosen when the parts fit in one wave and the
+  // largest exceeds the ideal share by no more than 24 atoms.  Otherwise "contiguous": the atoms of all units
+  // laid end to end and cut into gridDim equal ranges, which balances any mix of list lengths
+  // at the price of CTAs that straddle unit boundaries.
   const long long N = sh.unit_start[U];
-  const long long NP = (N < static_cast<long long>(gridDim.x)) ? N : static_cast<long long>(gridDim.x);
+  const int G = static_cast<int>(gridDim.x);
+  if (tid < kCandidates) { sh.cand_parts[tid] = 0; sh.cand_max[tid] = 0; }
+  if (tid == 0) sh.aligned = 0;
+  __syncthreads();
+  const bool try_aligned = (U <= kAlignedMaxUnits) && (N > 0);
+  if (try_aligned && tid < U) {
+    const int atoms = sh.unit_start[tid + 1] - sh.unit_start[tid];
+    if (atoms > 0) {
+#pragma unroll
+      for (int c = 0; c < kCandidates; ++c) {
+        // share_c = (N / G) * (1 + c / 16)
+        const long long num = static_cast<long long>(atoms) * G * 16;
+        const long long den = N * (16 + c);
+        int k = static_cast<int>((2 * num + den) / (2 * den));  // round to nearest
+        if (k < 1) k = 1;
+        if (k > atoms) k = atoms;
+        atomicAdd(&sh.cand_parts[c], k);
+        atomicMax(&sh.cand_max[c], (atoms + k - 1) / k);
+      }
+    }
+  }
+  __syncthreads();
+  int cand = -1;
+  if (try_aligned) {
+    for (int c = 0; c < kCandidates; ++c)
+      if (sh.cand_parts[c] <= G) { cand = c; break; }
+    // worth it only while the parts stay close to the ideal share: a straddling CTA costs a
+    // fixed few microseconds of extra merging, an oversized part costs time per atom
+    if (cand >= 0 && static_cast<long long>(sh.cand_max[cand]) * G > N + 24ll * G) cand = -1;
+  }
+  const bool aligned = cand >= 0;
+  if (aligned && warp == 0) {  // first CTA of every unit: exclusive scan of k_u
+    int carry = 0;
+    for (int base = 0; base < U; base += 32) {
+      const int u = base + lane;
+      int k = 0;
+      if (u < U) {
+        const int atoms = sh.unit_start[u + 1] - sh.unit_start[u];
+        if (atoms > 0) {
+          const long long num = static_cast<long long>(atoms) * G * 16;
+          const long long den = N * (16 + cand);
+          k = static_cast<int>((2 * num + den) / (2 * den));
+          if (k < 1) k = 1;
+          if (k > atoms) k = atoms;
+        }
+      }
+      int v = k;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += n;
+      }
+      if (u < U) sh.part_start[u + 1] = v + carry;
+      if (base == 0 && lane == 0) sh.part_start[0] = 0;
+      carry += __shfl_sync(0xffffffffu, v, 31);
+    }
+  }
+  __syncthreads();
+  const long long NP = aligned ? sh.part_start[U] : ((N < G) ? N : static_cast<long long>(G));
   if (warp < NC) {
     // consumers are the only writers of global memory: from here on the previous kernel's
     // results (and its use of the shared workspace) are complete
@@ -300,8 +371,22 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     }
   }
   if (static_cast<long long>(blockIdx.x) >= NP) return;
-  const int a0 = cta_first_atom(blockIdx.x, N, NP);
-  const int a1 = cta_first_atom(blockIdx.x + 1, N, NP);
+  int a0, a1;
+  if (aligned) {
+    int lo = 0, hi = U - 1;  // unit whose CTA range holds this CTA
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (sh.part_start[mid] <= static_cast<int>(blockIdx.x)) lo = mid; else hi = mid - 1;
+    }
+    const int k = sh.part_start[lo + 1] - sh.part_start[lo];
+    const int j = static_cast<int>(blockIdx.x) - sh.part_start[lo];
+    const long long atoms = sh.unit_start[lo + 1] - sh.unit_start[lo];
+    a0 = sh.unit_start[lo] + static_cast<int>(j * atoms / k);
+    a1 = sh.unit_start[lo] + static_cast<int>((j + 1) * atoms / k);
+  } else {
+    a0 = cta_first_atom(blockIdx.x, N, NP);
+    a1 = cta_first_atom(blockIdx.x + 1, N, NP);
+  }
 
   // unit holding atom a0
   int u_first;
@@ -536,7 +621,8 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         __stcg(rec + 67 * 32 + lane, l1);
         __threadfence();
         __syncwarp();
-        const int i_lo = cta_of_atom(us, N, NP), i_hi = cta_of_atom(ue - 1, N, NP);
+        const int i_lo = aligned ? sh.part_start[u] : cta_of_atom(us, N, NP);
+        const int i_hi = aligned ? sh.part_start[u + 1] - 1 : cta_of_atom(ue - 1, N, NP);
         unsigned int old = 0;
         if (lane == 0) old = atomicAdd(P.counters + u * kCountersPerUnit + mt, 1u);
         old = __shfl_sync(0xffffffffu, old, 0);
@@ -549,7 +635,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           m0 = m1 = -INFINITY;
           for (int i = i_lo; i <= i_hi; ++i) {
             const float* r2 = P.partials +
-                (static_cast<size_t>(2 * i + (cta_first_atom(i, N, NP) >= us ? 0 : 1)) * MT + mt) * kRec;
+                (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * MT + mt) * kRec;
             m0 = fmaxf(m0, __ldcg(r2 + 64 * 32 + lane));
             m1 = fmaxf(m1, __ldcg(r2 + 66 * 32 + lane));
           }
@@ -559,7 +645,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           for (int n = 0; n < 16; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
           for (int i = i_lo; i <= i_hi; ++i) {
             const float* r2 = P.partials +
-                (static_cast<size_t>(2 * i + (cta_first_atom(i, N, NP) >= us ? 0 : 1)) * MT + mt) * kRec;
+                (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * MT + mt) * kRec;
             const float w0 = ex2(__ldcg(r2 + 64 * 32 + lane) - base0);
             const float w1 = ex2(__ldcg(r2 + 66 * 32 + lane) - base1);
             l0 += __ldcg(r2 + 65 * 32 + lane) * w0;
