@@ -41,6 +41,7 @@ extern "C" {
 #define SPECATTN_ERR_WORKSPACE (-5)   /* workspace missing or smaller than *_workspace_bytes() */
 #define SPECATTN_ERR_UNSUPPORTED (-6) /* shape outside what the kernels are built for */
 #define SPECATTN_ERR_CUDA (-7)        /* the CUDA runtime refused the launch */
+#define SPECATTN_ERR_STATIC_SCRATCH (-8) /* shape needs more scratch than the built-in buffer has */
 
 /* ---- device-side per-list / per-sequence status flags ---------------------------------- */
 #define SPECATTN_ROW_OK 0
@@ -200,6 +201,38 @@ size_t specattn_verify_workspace_bytes(const specattn_verify_args* args);
 int specattn_verify_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 int specattn_sparse_verify(const specattn_verify_args* args, void* cuda_stream);
+
+/* ========================================================================================
+ * specattn_sparse_verify_static -- specattn_sparse_verify for callers that cannot allocate.
+ *
+ * (No counterpart in the paper: this entry point exists only for integration.)
+ *
+ * Some callers have no way to obtain the scratch buffer specattn_sparse_verify wants: code
+ * running as a custom call inside another runtime's compiled graph is handed its input and
+ * output buffers and nothing else; a serving engine may have reserved all device memory in
+ * its own pool, so that a cudaMalloc from a plug-in fails or stalls the whole device; and
+ * an allocation in the middle of a latency-critical decode loop synchronises the GPU.
+ * For them this variant keeps the scratch inside the library: a file-scope
+ * `static __device__` array of SPECATTN_STATIC_SCRATCH_BYTES bytes that every GPU loading the
+ * library holds from load until the process exits.  The call allocates and frees nothing
+ * (no cudaMalloc, cudaFree or allocating library routine).
+ *
+ * Same arguments, results and status codes as specattn_sparse_verify, except:
+ *   - args->workspace and args->workspace_bytes are ignored;
+ *   - a shape whose scratch need (specattn_verify_workspace_bytes) exceeds
+ *     SPECATTN_STATIC_SCRATCH_BYTES is rejected with SPECATTN_ERR_STATIC_SCRATCH and nothing
+ *     is launched.  The buffer covers up to 32 query rows per KV head (n_q * group <= 32) on
+ *     GPUs with up to 160 SMs;
+ *   - the first call on each device looks up the device address of the array (with that
+ *     device current); make that first call outside any stream capture;
+ *   - all calls on a device share the one array, which still holds what the previous call left
+ *     there: the arrival counters are cleared on the stream at the start of every call, and
+ *     two calls that may overlap on the GPU (different streams, or concurrent graph branches)
+ *     race on it -- serialise them or use specattn_sparse_verify with separate workspaces.
+ * ======================================================================================== */
+#define SPECATTN_STATIC_SCRATCH_BYTES (6u << 20)
+
+int specattn_sparse_verify_static(const specattn_verify_args* args, void* cuda_stream);
 
 /* ========================================================================================
  * specattn_verify_step_host -- one whole verification step from HOST buffers.

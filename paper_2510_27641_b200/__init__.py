@@ -12,7 +12,7 @@ from typing import Sequence
 
 import torch
 
-__all__ = ["select_topp", "sparse_verify", "verify_workspace", "verify_workspace_bytes",
+__all__ = ["select_topp", "sparse_verify", "sparse_verify_static", "verify_workspace", "verify_workspace_bytes",
            "verify_step_host", "status_string", "kernel_launch_count", "library_path",
            "SelectArgs", "VerifyArgs", "StepHostArgs", "lib", "SpecAttnError",
            "ROW_OK", "ROW_INVALID_PROB", "ROW_OVERFLOW", "ROW_BAD_INDEX", "ROW_TIMEOUT",
@@ -81,6 +81,8 @@ def lib() -> C.CDLL:
         L.specattn_verify_workspace_bytes.restype = C.c_size_t
         L.specattn_verify_workspace_init.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
         L.specattn_verify_workspace_init.restype = C.c_int
+        L.specattn_sparse_verify_static.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
+        L.specattn_sparse_verify_static.restype = C.c_int
         L.specattn_verify_step_host.argtypes = [C.POINTER(StepHostArgs), C.c_void_p]
         L.specattn_verify_step_host.restype = C.c_int
         L.specattn_status_string.argtypes = [C.c_int]
@@ -256,6 +258,17 @@ def sparse_verify(q: torch.Tensor, kv_pages: torch.Tensor, kv_len: torch.Tensor,
     if rc != 0:
         raise SpecAttnError(rc, "specattn_sparse_verify")
     return out, lse, status
+
+
+def sparse_verify_static(args: VerifyArgs, stream=None) -> None:
+    """specattn_sparse_verify_static: the same attention call for code that may not allocate
+    device memory (plug-ins handed only their inputs and outputs, engines whose pool owns the
+    whole GPU).  ``args`` is a filled VerifyArgs; its workspace fields are ignored because the
+    scratch is a fixed array inside the library.  Calls on one device share that array, so
+    they must not overlap on the GPU."""
+    rc = lib().specattn_sparse_verify_static(C.byref(args), _stream_ptr(stream))
+    if rc != 0:
+        raise SpecAttnError(rc, "specattn_sparse_verify_static")
 
 
 def verify_step_host(select_args: SelectArgs, draft_probs_host: Sequence[torch.Tensor | None],

@@ -48,6 +48,8 @@ extern "C" const char* specattn_status_string(int code) {
     case SPECATTN_ERR_WORKSPACE: return "workspace missing or too small";
     case SPECATTN_ERR_UNSUPPORTED: return "shape outside what the kernels support";
     case SPECATTN_ERR_CUDA: return "the CUDA runtime reported an error";
+    case SPECATTN_ERR_STATIC_SCRATCH:
+      return "the shape needs more scratch than the library's built-in static buffer holds";
     default: return "unknown status code";
   }
 }

@@ -836,3 +836,52 @@ extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cu
   specattn::g_launch_count.fetch_add(1, std::memory_order_relaxed);
   return SPECATTN_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// The variant for callers that cannot allocate: scratch lives in this library image.
+namespace specattn {
+namespace {
+// One copy per GPU that loads the library, held until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[SPECATTN_STATIC_SCRATCH_BYTES];
+}  // namespace
+}  // namespace specattn
+
+extern "C" int specattn_sparse_verify_static(const specattn_verify_args* args, void* cuda_stream) {
+  const int v = specattn::validate(args);
+  if (v != SPECATTN_OK) return v;
+  if (args->batch == 0) return SPECATTN_OK;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return SPECATTN_ERR_CUDA;
+  }
+  // In host code the array's name is only a handle; the kernel needs its device address,
+  // looked up once per device with that device current.
+  static void* device_addr[64] = {nullptr};
+  static std::atomic<unsigned long long> looked_up{0};
+  if (!((looked_up.load(std::memory_order_acquire) >> dev) & 1ull)) {
+    void* p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, specattn::g_static_scratch);
+    if (e != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return SPECATTN_ERR_CUDA;
+    }
+    device_addr[dev] = p;
+    looked_up.fetch_or(1ull << dev, std::memory_order_release);
+  }
+  void* scratch = device_addr[dev];
+  const int n_ctas = specattn::device_sm_count();
+  if (n_ctas <= 0) return SPECATTN_ERR_CUDA;
+  if (specattn::workspace_bytes_for(*args, n_ctas) > SPECATTN_STATIC_SCRATCH_BYTES)
+    return SPECATTN_ERR_STATIC_SCRATCH;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  // the array keeps the previous call's contents: the arrival counters must start at zero
+  if (cudaMemsetAsync(scratch, 0, specattn::kCounterBytes, stream) != cudaSuccess) {
+    cudaGetLastError();
+    return SPECATTN_ERR_CUDA;
+  }
+  specattn_verify_args a = *args;
+  a.workspace = scratch;
+  a.workspace_bytes = SPECATTN_STATIC_SCRATCH_BYTES;
+  return specattn_sparse_verify(&a, cuda_stream);
+}

@@ -1,0 +1,66 @@
+"""specattn_sparse_verify_static: the attention entry point for callers that cannot allocate
+device memory (a custom call inside another runtime's graph gets only its inputs and outputs;
+a serving engine's pool may own the whole GPU).  Its scratch is a fixed array inside the
+library, so the test checks that two calls in a row -- the second one meeting whatever the
+first left in that array -- both reproduce the regular entry point's results."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import workloads as wl
+from gpu_util import LSE_TOL, OUT_TOL, bf16_to_dev, dev, lse_err, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(seed, B, T, Hq, Hkv, lens, counts):
+    rng = np.random.default_rng(seed)
+    page = 16
+    pps = (max(lens) + page - 1) // page
+    kv = wl.kv_pool(seed, 0, B * pps, page, Hkv, 128, device=dev())
+    bt = to_dev(wl.block_table(seed, B, pps))
+    q = bf16_to_dev(wl.queries(seed, 0, B, T, Hq, 128))
+    idx = np.zeros((B, 1, max(lens)), np.int32)
+    for b in range(B):
+        idx[b, 0, :counts[b]] = np.sort(rng.choice(lens[b], size=counts[b], replace=False))
+    return q, kv, bt, to_dev(np.asarray(lens, np.int32)), to_dev(idx), to_dev(np.asarray(counts, np.int32).reshape(B, 1))
+
+
+def test_static_scratch_entry_point_matches_the_regular_one_twice_in_a_row():
+    import paper_2510_27641_b200 as sa
+    cases = [_case(41, 3, 6, 32, 8, [5000, 300, 40], [3100, 300, 0]),      # units split across CTAs
+             _case(42, 2, 5, 32, 8, [900, 2000], [17, 1999])]
+    for q, kv, bt, kv_len, idx, cnt in cases:
+        ref_out, ref_lse, ref_status = sa.sparse_verify(q, kv, kv_len, block_table=bt, idx=idx, counts=cnt)
+        torch.cuda.synchronize()
+        for call in range(2):
+            out = torch.full_like(ref_out, float("nan"))
+            lse = torch.full_like(ref_lse, float("nan"))
+            status = torch.zeros_like(ref_status)
+            args = sa.make_verify_args(q, kv, kv_len, block_table=bt, idx=idx, counts=cnt, out=out, lse=lse,
+                                       status=status)          # no workspace: none is needed
+            before = torch.cuda.memory_allocated()
+            sa.sparse_verify_static(args)
+            torch.cuda.synchronize()
+            assert torch.cuda.memory_allocated() == before
+            assert float((out - ref_out).abs().max()) <= OUT_TOL, f"call {call}"
+            assert lse_err(lse.cpu().numpy().astype(np.float64), ref_lse.cpu().numpy().astype(np.float64)) <= LSE_TOL
+            assert torch.equal(status, ref_status)
+
+
+def test_static_scratch_entry_point_rejects_shapes_beyond_its_buffer():
+    import paper_2510_27641_b200 as sa
+    # 8 queries x group of 8 = 64 query rows per KV head: four 16-row slabs need ~10 MB of scratch
+    q, kv, bt, kv_len, idx, cnt = _case(43, 1, 8, 64, 8, [64], [10])
+    out = torch.empty((1, 8, 64, 128), dtype=torch.float32, device=dev())
+    lse = torch.empty((1, 8, 64), dtype=torch.float32, device=dev())
+    args = sa.make_verify_args(q, kv, kv_len, block_table=bt, idx=idx, counts=cnt, out=out, lse=lse)
+    assert sa.verify_workspace_bytes(args) > (6 << 20)
+    n0 = sa.kernel_launch_count()
+    with pytest.raises(sa.SpecAttnError) as e:
+        sa.sparse_verify_static(args)
+    assert e.value.code == -8 and "static" in str(e.value)
+    assert sa.kernel_launch_count() == n0
+    assert sa.lib().specattn_sparse_verify_static(None, None) == -1
