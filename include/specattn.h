@@ -183,7 +183,7 @@ typedef struct specattn_verify_args {
   const int32_t* idx;
   int64_t idx_stride;
   const int32_t* counts;
-  float sm_scale;        /* 0 => 1/sqrt(head_dim) */
+  float sm_scale;        /* > 0, or 0 => 1/sqrt(head_dim); negative or NaN is rejected */
   float* out;            /* binary32 [batch, n_q, n_q_heads, head_dim] */
   float* lse;            /* binary32 [batch, n_q, n_q_heads] */
   int32_t* status;       /* [batch] or NULL */

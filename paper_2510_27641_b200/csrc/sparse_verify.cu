@@ -96,6 +96,9 @@ struct VShared {
   int cand_max[kCandidates];
   int aligned;                           // 1: unit-aligned partition, 0: contiguous atoms
   volatile int abort_flag;
+  // cluster merge (two CTAs per unit): the odd CTA's records land here, in the even CTA
+  unsigned long long peer_full;
+  float peer_rec[(MT <= 2) ? MT : 1][(MT <= 2) ? kRec : 1];
 };
 
 __device__ __forceinline__ int unit_count(const VerifyParams& P, int u) {
@@ -154,13 +157,16 @@ __device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&q
     mma_bf16(sc[2], qf[kk], k1[0], k1[1]);
     mma_bf16(sc[3], qf[kk], k1[2], k1[3]);
   }
+  // raw scores stay unscaled: exp2(s * c - m * c) is one fused multiply-add per element
+  if (valid < 32) {  // only the last block of a segment has missing keys
 #pragma unroll
-  for (int n = 0; n < 4; ++n)
+    for (int n = 0; n < 4; ++n)
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int key = n * 8 + tq * 2 + (i & 1);
-      sc[n][i] = (key < valid) ? sc[n][i] * scale_log2 : -INFINITY;
-    }
+      for (int i = 0; i < 4; ++i) {
+        const int key = n * 8 + tq * 2 + (i & 1);
+        if (key >= valid) sc[n][i] = -INFINITY;
+      }
+  }
   float mx0 = fmaxf(fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])),
                     fmaxf(fmaxf(sc[2][0], sc[2][1]), fmaxf(sc[3][0], sc[3][1])));
   float mx1 = fmaxf(fmaxf(fmaxf(sc[0][2], sc[0][3]), fmaxf(sc[1][2], sc[1][3])),
@@ -169,7 +175,8 @@ __device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&q
   mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
   mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
   mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-  const float mn0 = fmaxf(st.m0, mx0), mn1 = fmaxf(st.m1, mx1);
+  // running maxima are kept in the scaled log2 domain (scale_log2 > 0 keeps the order)
+  const float mn0 = fmaxf(st.m0, mx0 * scale_log2), mn1 = fmaxf(st.m1, mx1 * scale_log2);
   const float base0 = (mn0 == -INFINITY) ? 0.f : mn0;
   const float base1 = (mn1 == -INFINITY) ? 0.f : mn1;
   const float al0 = ex2(st.m0 - base0), al1 = ex2(st.m1 - base1);
@@ -178,10 +185,10 @@ __device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&q
   float s0 = 0.f, s1 = 0.f;
 #pragma unroll
   for (int n = 0; n < 4; ++n) {
-    sc[n][0] = ex2(sc[n][0] - base0);
-    sc[n][1] = ex2(sc[n][1] - base0);
-    sc[n][2] = ex2(sc[n][2] - base1);
-    sc[n][3] = ex2(sc[n][3] - base1);
+    sc[n][0] = ex2(fmaf(sc[n][0], scale_log2, -base0));
+    sc[n][1] = ex2(fmaf(sc[n][1], scale_log2, -base0));
+    sc[n][2] = ex2(fmaf(sc[n][2], scale_log2, -base1));
+    sc[n][3] = ex2(fmaf(sc[n][3], scale_log2, -base1));
     s0 += sc[n][0] + sc[n][1];
     s1 += sc[n][2] + sc[n][3];
   }
@@ -196,7 +203,8 @@ __device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&q
       st.acc[n][3] *= al1;
     }
   }
-  // A-operand fragments of P for the two 16-key halves, each as a bf16 pair (hi, lo)
+  // A-operand fragments of P for the two 16-key halves, each as a bf16 pair (hi, lo):
+  // hi = bf16x2(x, y); the residuals x - hi.x, y - hi.y are exact in fp32 and rounded once more
   uint32_t phi[2][4], plo[2][4];
 #pragma unroll
   for (int kb = 0; kb < 2; ++kb)
@@ -205,12 +213,9 @@ __device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&q
 #pragma unroll
       for (int hrow = 0; hrow < 2; ++hrow) {
         const float x = sc[kb * 2 + n][hrow * 2], y = sc[kb * 2 + n][hrow * 2 + 1];
-        const __nv_bfloat16 xh = __float2bfloat16_rn(x), yh = __float2bfloat16_rn(y);
-        __nv_bfloat162 hi2;
-        hi2.x = xh;
-        hi2.y = yh;
-        phi[kb][n * 2 + hrow] = *reinterpret_cast<uint32_t*>(&hi2);
-        plo[kb][n * 2 + hrow] = pack_bf16(x - __bfloat162float(xh), y - __bfloat162float(yh));
+        const uint32_t h = pack_bf16(x, y);
+        phi[kb][n * 2 + hrow] = h;
+        plo[kb][n * 2 + hrow] = pack_bf16(x - __uint_as_float(h << 16), y - __uint_as_float(h & 0xffff0000u));
       }
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
@@ -261,6 +266,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     }
     mbar_init(&sh.q_full, 1);
     mbar_init(&sh.q_empty, NC);
+    mbar_init(&sh.peer_full, MT);
     mbar_fence_init();
     sh.abort_flag = 0;
     sh.unit_start[0] = 0;
@@ -272,6 +278,9 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   }
   fence_proxy_async();
   __syncthreads();
+  // launched as CTA pairs: the peer's barrier must exist before anyone can arrive on it
+  const bool paired = (MT <= 2) && (cluster_num_ctas() == 2);
+  if (paired) cluster_sync_all();
   if (warp == 0) {  // inclusive scan of the atom counts, 32 at a time
     int carry = 0;
     for (int base = 0; base < U; base += 32) {
@@ -438,17 +447,10 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         q_pending = false;
         if (!load_q()) { sh.abort_flag = 1; dead = true; break; }
       }
-      for (int t0 = tok_lo; t0 < tok_hi; t0 += kStageTok, ++it) {
-        if ((it % kProdWarps) != pw) continue;
-        const int s = it % kStages;
-        const unsigned ph = (it / kStages) & 1u;
-        if (!mbar_wait(&sh.empty[s], ph ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
+      // lane j resolves tokens j and j + 32 of a tile to the byte offset of their K row:
+      // list -> position -> block table -> page, two dependent loads
+      auto resolve = [&](int t0, long long (&off)[2]) -> bool {
         const int ntok = min(kStageTok, tok_hi - t0);
-        // The tail of a segment is padded to a whole 32-key block with copies of its last
-        // token, so that every row a consumer multiplies by a zero weight holds finite data.
-        const int npad = (ntok + 31) & ~31;
-        // lane j resolves tokens j and j + 32 to the byte offset of their K row
-        long long off[2];
         bool bad = false;
 #pragma unroll
         for (int jj = 0; jj < 2; ++jj) {
@@ -462,6 +464,34 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           if (page < 0 || (P.n_pages > 0 && page >= P.n_pages)) { bad = true; page = 0; }
           off[jj] = (page * P.s_page + static_cast<long long>(slot) * P.s_slot) * 2;
         }
+        return bad;
+      };
+      long long off_next[2] = {0, 0};
+      bool bad_next = false;
+      int t0_next = -1;  // tile whose offsets are already resolved
+      for (int t0 = tok_lo; t0 < tok_hi; t0 += kStageTok, ++it) {
+        if ((it % kProdWarps) != pw) continue;
+        const int s = it % kStages;
+        const unsigned ph = (it / kStages) & 1u;
+        long long off[2];
+        bool bad;
+        if (t0_next == t0) {
+          off[0] = off_next[0];
+          off[1] = off_next[1];
+          bad = bad_next;
+        } else {
+          bad = resolve(t0, off);
+        }
+        // Resolve this warp's next tile of the segment now, so that its two dependent loads
+        // are in flight while the warp waits for the slot: the slot's turnaround then holds
+        // only the copy itself.
+        t0_next = t0 + kProdWarps * kStageTok;
+        if (t0_next < tok_hi) bad_next = resolve(t0_next, off_next); else t0_next = -1;
+        if (!mbar_wait(&sh.empty[s], ph ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
+        const int ntok = min(kStageTok, tok_hi - t0);
+        // The tail of a segment is padded to a whole 32-key block with copies of its last
+        // token, so that every row a consumer multiplies by a zero weight holds finite data.
+        const int npad = (ntok + 31) & ~31;
         // 16 lanes move one 256-byte row with 16-byte cp.async copies: a warp instruction
         // fetches two rows (four full 128-byte lines)
         const char* kbase = reinterpret_cast<const char*>(kv_head) + (lane & 15) * 16;
@@ -608,7 +638,44 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     if (wr == 0) {
       const bool whole = (a == us) && (seg_hi == ue);
       bool finish = whole;
-      if (!whole) {
+      // A unit cut in exactly two parts whose CTAs form one cluster is merged through the even
+      // CTA's shared memory: the odd CTA stores its record there and arrives on a barrier.
+      const bool pair_merge = paired && aligned && !whole && (sh.part_start[u + 1] - sh.part_start[u] == 2) &&
+                              ((sh.part_start[u] & 1) == 0);
+      if (pair_merge) {
+        if (cluster_cta_rank() == 1) {
+          const uint32_t dst = map_to_cta(smem_u32(sh.peer_rec[mt]), 0) + lane * 4;
+#pragma unroll
+          for (int n = 0; n < 16; ++n)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) st_cluster_f32(dst + (n * 4 + i) * 128, acc[n][i]);
+          st_cluster_f32(dst + 64 * 128, m0);
+          st_cluster_f32(dst + 65 * 128, l0);
+          st_cluster_f32(dst + 66 * 128, m1);
+          st_cluster_f32(dst + 67 * 128, l1);
+          __syncwarp();
+          if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&sh.peer_full), 0));
+        } else {
+          if (!mbar_wait_cluster(&sh.peer_full, 0u, &sh.abort_flag)) { sh.abort_flag = 1; ok = false; break; }
+          const float* rec = sh.peer_rec[mt];
+          float mn, ao, ai;
+          merge_scales(m0, rec[64 * 32 + lane], mn, ao, ai);
+          l0 = l0 * ao + rec[65 * 32 + lane] * ai;
+          m0 = mn;
+          float mn1, ao1, ai1;
+          merge_scales(m1, rec[66 * 32 + lane], mn1, ao1, ai1);
+          l1 = l1 * ao1 + rec[67 * 32 + lane] * ai1;
+          m1 = mn1;
+#pragma unroll
+          for (int n = 0; n < 16; ++n) {
+            acc[n][0] = acc[n][0] * ao + rec[(n * 4 + 0) * 32 + lane] * ai;
+            acc[n][1] = acc[n][1] * ao + rec[(n * 4 + 1) * 32 + lane] * ai;
+            acc[n][2] = acc[n][2] * ao1 + rec[(n * 4 + 2) * 32 + lane] * ai1;
+            acc[n][3] = acc[n][3] * ao1 + rec[(n * 4 + 3) * 32 + lane] * ai1;
+          }
+          finish = true;
+        }
+      } else if (!whole) {
         // publish this CTA's share of the unit, then see whether it was the last to arrive
         float* rec = P.partials + (static_cast<size_t>(2 * blockIdx.x + (a == a0 ? 0 : 1)) * MT + mt) * kRec;
 #pragma unroll
@@ -716,11 +783,18 @@ cudaError_t launch(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
   cfg.blockDim = dim3((MT * WPM + kProdWarps) * 32, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (MT <= 2 && n_ctas % 2 == 0) {  // CTA pairs: short units are merged through peer shared memory
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
   err = cudaLaunchKernelEx(&cfg, sparse_verify_kernel<MT, WPM>, P);
   if (err != cudaSuccess) cudaGetLastError();
   return err;
@@ -739,6 +813,7 @@ int validate(const specattn_verify_args* args) {
     return SPECATTN_ERR_RANGE;
   if (A.n_q_heads % A.n_kv_heads != 0) return SPECATTN_ERR_RANGE;
   if (A.n_groups != 1 && A.n_groups != A.n_kv_heads) return SPECATTN_ERR_RANGE;
+  if (!(A.sm_scale >= 0.f)) return SPECATTN_ERR_RANGE;  // negative or NaN
   if (A.head_dim != kD) return SPECATTN_ERR_UNSUPPORTED;
   if (A.n_q * (A.n_q_heads / A.n_kv_heads) > SPECATTN_MAX_QUERY_ROWS) return SPECATTN_ERR_UNSUPPORTED;
   if (static_cast<long long>(A.batch) * A.n_kv_heads > kMaxUnits) return SPECATTN_ERR_UNSUPPORTED;
