@@ -45,7 +45,8 @@ extern "C" {
 
 /* ---- device-side per-list / per-sequence status flags ---------------------------------- */
 #define SPECATTN_ROW_OK 0
-#define SPECATTN_ROW_INVALID_PROB 1 /* a contributing probability was negative, NaN or Inf */
+#define SPECATTN_ROW_INVALID_PROB 1 /* a contributing probability was negative, NaN or Inf (or the
+                                       binary32 sum of a position overflowed) */
 #define SPECATTN_ROW_OVERFLOW 2     /* the list has more entries than idx_stride; truncated */
 #define SPECATTN_ROW_BAD_INDEX 4    /* verify met a position or page id out of range */
 #define SPECATTN_ROW_TIMEOUT 8      /* a bounded device-side wait ran out; outputs invalid */
@@ -54,7 +55,7 @@ extern "C" {
 #define SPECATTN_MAX_DRAFT_LAYERS 64
 #define SPECATTN_MAX_DRAFT_HEADS 256
 #define SPECATTN_MAX_ROWS_PER_LIST 1024  /* contributing (head, query) rows per list */
-#define SPECATTN_MAX_KV_LEN 327680       /* positions per sequence for select (8 x 40960) */
+#define SPECATTN_MAX_KV_LEN 262144       /* positions per sequence for select (8 x 32768) */
 #define SPECATTN_MAX_VERIFY_UNITS 2048   /* batch * n_kv_heads for verify */
 #define SPECATTN_MAX_QUERY_ROWS 64       /* n_q * (n_q_heads / n_kv_heads) for verify */
 

@@ -81,7 +81,8 @@ int specattn_oracle_num_threads(void) {
 //   a_bar      [L] output
 // Order of the binary32 additions: start from +0, heads ascending, inside a
 // head the speculated queries ascending.  Returns ORACLE_INVALID_PROB if any
-// contributing input is negative, NaN or infinite (the row is still written).
+// contributing input is negative, NaN or infinite, or if the binary32 chain
+// itself overflows (impossible for probabilities) -- the row is still written.
 // [Sec. 3.4 item 1; Alg. 1 "Sparse Attention Mask Creation"]
 // ---------------------------------------------------------------------------
 int specattn_oracle_aggregate(const float* A, int n_heads, int gamma, int64_t L_stride, int L,
@@ -97,6 +98,7 @@ int specattn_oracle_aggregate(const float* A, int n_heads, int gamma, int64_t L_
         acc = acc + x;
       }
     }
+    if (!(acc <= FLT_MAX)) status = ORACLE_INVALID_PROB;  // the binary32 chain overflowed
     a_bar[i] = acc;
   }
   return status;

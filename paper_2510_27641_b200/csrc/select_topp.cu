@@ -8,9 +8,13 @@
 // histogram of (count, mass) per bin, and the row never leaves the chip between passes.
 //
 // Mapping to the GPU: one thread-block cluster (1, 2, 4 or 8 CTAs) per index list.  Each CTA
-//   1. streams its slice of positions of all contributing (head, query) rows from HBM with
-//      128-bit loads, adds them in the fixed order that defines the aggregated row, and keeps
-//      the aggregated slice in shared memory (it is never written to global memory);
+//   1. streams its slice of positions of all contributing (head, query) rows from HBM in 8 KB
+//      row pieces: every thread copies the two float4 columns it will add itself with 16-byte
+//      cp.async into its own shared-memory ring slots, eight pieces ahead (64 KB in flight per
+//      CTA, no registers held, no barrier needed), adds them in the fixed order that defines
+//      the aggregated row and keeps the aggregated slice in shared memory (it is never written
+//      to global memory).  (A 1-D bulk-copy ring fed by a producer warp was measured first:
+//      like the gather in the verify kernel it stalled near 25 GB/s per SM.)
 //   2. builds the level histogram in shared memory (64-bit packed count|mantissa-sum atomics;
 //      all values of a bin share one exponent, so the mantissa sum is an exact integer and
 //      the result does not depend on the order of the atomics);
@@ -26,6 +30,7 @@
 
 #include <atomic>
 
+#include "ptx.cuh"
 #include "specattn.h"
 
 namespace cg = cooperative_groups;
@@ -36,16 +41,19 @@ extern std::atomic<long long> g_launch_count;
 
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;            // worker threads
 constexpr int kWarps = kThreads / 32;
+constexpr int kBlock = kThreads;
+constexpr int kChunk = 2048;             // positions per staged row piece (8 KB)
+constexpr int kDepth = 8;                // row pieces in flight per thread (ring of 8 x 8 KB)
 constexpr int kL1Bins = 2048;        // sign(0) + 8 exponent bits + 3 mantissa bits
 constexpr int kL23Bins = 1024;       // 10 mantissa bits per later level
-constexpr int kHistSlots = kL1Bins + 8;  // slot kL1Bins counts invalid inputs
+constexpr int kHistSlots = kL1Bins + 8;  // slot kL1Bins counts invalid inputs, the next one timeouts
 constexpr int kInvalidSlot = kL1Bins;
+constexpr int kTimeoutSlot = kL1Bins + 1;
 constexpr int kGroup = 32;           // bins per scan group
 constexpr int kMaxGroups = kL1Bins / kGroup;
-constexpr int kSliceCap = 40960;     // positions per CTA
-constexpr int kUnroll = 8;           // rows in flight per thread
+constexpr int kSliceCap = 32768;     // positions per CTA
 constexpr unsigned long long kOne = 1ull << 44;  // count field of a packed bin
 constexpr unsigned long long kMantMask = kOne - 1;
 
@@ -68,9 +76,9 @@ struct SelectParams {
 
 struct Shared {
   unsigned long long hist[kHistSlots];
-  double mass[kL1Bins];
-  unsigned int cnt[kL1Bins];
-  int rows[SPECATTN_MAX_ROWS_PER_LIST];
+  double* mass;        // [kL1Bins] reduced bin masses  } both alias the staging ring, which is
+  unsigned int* cnt;   // [kL1Bins] reduced bin counts  } idle once the slice is aggregated
+  long long row_off[SPECATTN_MAX_ROWS_PER_LIST];  // element offset of each contributing row, in add order
   double grp_mass[kMaxGroups];
   double suf_mass[kMaxGroups + 1];
   unsigned int grp_cnt[kMaxGroups];
@@ -123,20 +131,22 @@ __device__ void reduce_hist(cg::cluster_group& cluster, Shared& sh, int nbins, E
   const unsigned cs = cluster.num_blocks();
   const unsigned rank = cluster.block_rank();
   const int per = nbins / static_cast<int>(cs);
+  double* const mass = sh.mass;
+  unsigned int* const cnt = sh.cnt;
   cluster.sync();  // every CTA's histogram is complete
   const int lo = static_cast<int>(rank) * per;
-  for (int bin = lo + threadIdx.x; bin < lo + per; bin += kThreads) {
+  for (int bin = lo + threadIdx.x; bin < lo + per && threadIdx.x < kThreads; bin += kThreads) {
     unsigned long long s = 0;
     for (unsigned r = 0; r < cs; ++r) s += *cluster.map_shared_rank(&sh.hist[bin], r);
-    sh.cnt[bin] = static_cast<unsigned int>(s >> 44);
-    sh.mass[bin] = static_cast<double>(s & kMantMask) * pow2_double(exp_of_bin(bin));
+    cnt[bin] = static_cast<unsigned int>(s >> 44);
+    mass[bin] = static_cast<double>(s & kMantMask) * pow2_double(exp_of_bin(bin));
   }
   cluster.sync();  // every owner's part is reduced; remote histograms are no longer read
-  for (int bin = threadIdx.x; bin < nbins; bin += kThreads) {
+  for (int bin = threadIdx.x; bin < nbins && threadIdx.x < kThreads; bin += kThreads) {
     const unsigned owner = static_cast<unsigned>(bin / per);
     if (owner != rank) {
-      sh.cnt[bin] = *cluster.map_shared_rank(&sh.cnt[bin], owner);
-      sh.mass[bin] = *cluster.map_shared_rank(&sh.mass[bin], owner);
+      cnt[bin] = *cluster.map_shared_rank(&cnt[bin], owner);
+      mass[bin] = *cluster.map_shared_rank(&mass[bin], owner);
     }
   }
   __syncthreads();
@@ -151,12 +161,14 @@ __device__ double scan_bins(Shared& sh, int nbins, double carry_mass, unsigned i
                             double target, bool target_is_fraction, float p) {
   const int groups = nbins / kGroup;
   const int tid = threadIdx.x;
+  const double* const mass = sh.mass;
+  const unsigned int* const cnt = sh.cnt;
   if (tid < groups) {
     double s = 0.0;
     unsigned int c = 0;
     for (int b = kGroup - 1; b >= 0; --b) {
-      s += sh.mass[tid * kGroup + b];
-      c += sh.cnt[tid * kGroup + b];
+      s += mass[tid * kGroup + b];
+      c += cnt[tid * kGroup + b];
     }
     sh.grp_mass[tid] = s;
     sh.grp_cnt[tid] = c;
@@ -195,11 +207,11 @@ __device__ double scan_bins(Shared& sh, int nbins, double carry_mass, unsigned i
     int last_bin = -1;
     for (int b = kGroup - 1; b >= 0; --b) {
       const int bin = j * kGroup + b;
-      const unsigned int cb = sh.cnt[bin];
+      const unsigned int cb = cnt[bin];
       if (cb == 0) continue;
       prev = s;
       cprev = c;
-      s += sh.mass[bin];
+      s += mass[bin];
       c += cb;
       last_bin = bin;
       if (target <= s) {
@@ -223,10 +235,10 @@ __device__ double scan_bins(Shared& sh, int nbins, double carry_mass, unsigned i
   return all;
 }
 
-__global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_constant__ SelectParams P) {
+__global__ void __launch_bounds__(kBlock, 2) select_topp_kernel(const __grid_constant__ SelectParams P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
-  float* a = reinterpret_cast<float*>(smem_raw + ((sizeof(Shared) + 15) / 16) * 16);
+  float* a = reinterpret_cast<float*>(smem_raw + ((sizeof(Shared) + 127) / 128) * 128);
 
   cg::cluster_group cluster = cg::this_cluster();
   const int cs = static_cast<int>(cluster.num_blocks());
@@ -234,6 +246,7 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int warp = tid >> 5;
+  const bool worker = tid < kThreads;
 
   const int list = blockIdx.y;  // (used slot, sequence, group)
   const int g = list % P.G;
@@ -256,62 +269,111 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
     int n = 0;
     for (int h = 0; h < P.H; ++h) {
       if (P.has_groups && P.head_group[h] != g) continue;
-      for (int s = 0; s < P.gamma; ++s) sh.rows[n++] = h * P.gamma + s;
+      for (int s = 0; s < P.gamma; ++s) sh.row_off[n++] = static_cast<long long>(h * P.gamma + s) * P.L_stride;
     }
     sh.n_rows = n;
   }
-  for (int i = tid; i < kHistSlots; i += kThreads) sh.hist[i] = 0ull;
+  for (int i = tid; i < kHistSlots; i += kBlock) sh.hist[i] = 0ull;
   __syncthreads();
   const int R = sh.n_rows;
 
   // ---- 1+2: aggregate the slice and build the level-1 histogram ------------------------------
   const float* A = P.probs[slot] + static_cast<long long>(b) * P.H * P.gamma * P.L_stride + lo;
   const int n4 = (n_loc + 3) >> 2;
+  const int n_pos4 = n4 * 4;                       // slice length rounded up to whole float4s
+  const int n_chunks = (n_pos4 + kChunk - 1) / kChunk;
+  // ring buffers follow the aggregated slice (whose capacity is fixed by the launch)
+  const int slice_cap4 = ((((P.L_stride + cs - 1) / cs + 3) & ~3ll) + 31) & ~31ll;
+  float* ring = a + slice_cap4;
+  if (tid == 0) {
+    sh.mass = reinterpret_cast<double*>(ring);
+    sh.cnt = reinterpret_cast<unsigned int*>(ring + 2 * kL1Bins);
+  }
   bool bad = false;
-  for (int base = 0; base < n4; base += kThreads) {
-    const int i4 = base + tid;
-    const bool act = i4 < n4;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (act) {
-      const float* col = A + 4 * i4;
-      const int left = n_loc - 4 * i4;  // valid positions in this group of four (>= 1)
-      for (int r0 = 0; r0 < R; r0 += kUnroll) {
-        float4 v[kUnroll];
+  // Pieces are numbered q = chunk * R + row, i.e. in the order the adds must happen.  Every
+  // thread copies exactly the two float4 columns of a piece that it will add itself, with
+  // 16-byte cp.async into its own ring slots, kDepth pieces ahead: completion is tracked per
+  // thread (commit / wait groups), so the pipeline needs no barrier at all and holds
+  // kDepth x 8 KB of reads in flight per CTA without occupying registers.
+  {
+    const uint32_t ring_addr = smem_u32(ring) + tid * 16;
+    const float* src0 = A + 4 * tid;
+    int ic = 0, ir = 0, islot = 0;  // chunk, row and ring slot of the next piece to request
+    auto issue = [&]() {
+      if (ic < n_chunks) {
+        const int len4 = min(kChunk, n_pos4 - ic * kChunk) >> 2;
+        const float* src = src0 + sh.row_off[ir] + ic * kChunk;
+        const uint32_t dst = ring_addr + islot * (kChunk * 4);
 #pragma unroll
-        for (int j = 0; j < kUnroll; ++j) {
-          if (r0 + j < R)
-            v[j] = __ldcs(reinterpret_cast<const float4*>(col + static_cast<long long>(sh.rows[r0 + j]) * P.L_stride));
-        }
+        for (int k = 0; k < 2; ++k)
+          if (tid + k * kThreads < len4) cp_async16(dst + k * kThreads * 16, src + k * kThreads * 4);
+        if (++ir == R) { ir = 0; ++ic; }
+        islot = (islot + 1) & (kDepth - 1);
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    for (int q = 0; q < kDepth - 1; ++q) issue();
+    // Validity of the inputs is tracked with a running minimum (a negative input, the only
+    // invalid value a sum can hide) -- NaN and Inf survive into the aggregated value itself.
+    float4 acc[2], mn[2];
+    acc[0] = acc[1] = mn[0] = mn[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+    int slot = 0;
+    for (int c = 0; c < n_chunks; ++c) {
+      const int len4 = min(kChunk, n_pos4 - c * kChunk) >> 2;
+      // positions of this thread's two float4s that lie beyond the slice (last float4 only)
+      int cut[2];
 #pragma unroll
-        for (int j = 0; j < kUnroll; ++j) {
-          if (r0 + j < R) {
-            const float4 x = v[j];
-            bad |= !(x.x >= 0.f && x.x <= FLT_MAX);
-            if (left > 1) bad |= !(x.y >= 0.f && x.y <= FLT_MAX);
-            if (left > 2) bad |= !(x.z >= 0.f && x.z <= FLT_MAX);
-            if (left > 3) bad |= !(x.w >= 0.f && x.w <= FLT_MAX);
-            acc.x = acc.x + x.x;
-            acc.y = acc.y + x.y;
-            acc.z = acc.z + x.z;
-            acc.w = acc.w + x.w;
+      for (int k = 0; k < 2; ++k) cut[k] = n_loc - (c * kChunk + 4 * (tid + k * kThreads));
+      for (int r = 0; r < R; ++r) {
+        issue();
+        asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
+        const float4* piece = reinterpret_cast<const float4*>(ring + slot * kChunk);
+        slot = (slot + 1) & (kDepth - 1);
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const int i4 = tid + k * kThreads;
+          if (i4 < len4) {
+            float4 x = piece[i4];
+            if (cut[k] < 4) {  // values beyond kv_len are not inputs
+              if (cut[k] < 4) x.w = 0.f;
+              if (cut[k] < 3) x.z = 0.f;
+              if (cut[k] < 2) x.y = 0.f;
+            }
+            mn[k].x = fminf(mn[k].x, x.x);
+            mn[k].y = fminf(mn[k].y, x.y);
+            mn[k].z = fminf(mn[k].z, x.z);
+            mn[k].w = fminf(mn[k].w, x.w);
+            acc[k].x = acc[k].x + x.x;
+            acc[k].y = acc[k].y + x.y;
+            acc[k].z = acc[k].z + x.z;
+            acc[k].w = acc[k].w + x.w;
           }
         }
       }
-      if (left < 4) acc.w = 0.f;
-      if (left < 3) acc.z = 0.f;
-      if (left < 2) acc.y = 0.f;
-      *reinterpret_cast<float4*>(a + 4 * i4) = acc;
-    }
-    {
-      const float vals[4] = {acc.x, acc.y, acc.z, acc.w};
+      // the chunk is complete: store it and feed the level-1 histogram
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const unsigned int key = __float_as_uint(vals[e]);
-        // zeros carry no mass and can never be the threshold of a row with positive total
-        const bool take = act && (4 * i4 + e < n_loc) && key != 0u && !(key >> 31);
-        hist_add(sh.hist, take, static_cast<int>(key >> 20), mantissa_of(key));
+      for (int k = 0; k < 2; ++k) {
+        const int i4 = tid + k * kThreads;
+        const bool act = i4 < len4;
+        const int pos = c * kChunk + 4 * i4;  // position inside the slice
+        const float4 v = acc[k];
+        if (act) {
+          *reinterpret_cast<float4*>(a + pos) = v;
+          bad |= (mn[k].x < 0.f) | (mn[k].y < 0.f) | (mn[k].z < 0.f) | (mn[k].w < 0.f);
+          bad |= !(v.x <= FLT_MAX) | !(v.y <= FLT_MAX) | !(v.z <= FLT_MAX) | !(v.w <= FLT_MAX);
+        }
+        const float vals[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const unsigned int key = __float_as_uint(vals[e]);
+          // zeros carry no mass and can never be the threshold of a row with positive total
+          const bool take = act && (pos + e < n_loc) && key != 0u && !(key >> 31);
+          hist_add(sh.hist, take, static_cast<int>(key >> 20), mantissa_of(key));
+        }
+        acc[k] = mn[k] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
   }
   if (bad) atomicAdd(&sh.hist[kInvalidSlot], 1ull);
   __syncthreads();
@@ -319,12 +381,15 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
   // ---- 3: threshold search --------------------------------------------------------------------
   // invalid inputs anywhere in the cluster?
   cluster.sync();
-  unsigned long long n_bad = 0;
-  for (int r = 0; r < cs; ++r) n_bad += *cluster.map_shared_rank(&sh.hist[kInvalidSlot], r);
+  unsigned long long n_bad = 0, n_timeout = 0;
+  for (int r = 0; r < cs; ++r) {
+    n_bad += *cluster.map_shared_rank(&sh.hist[kInvalidSlot], r);
+    n_timeout += *cluster.map_shared_rank(&sh.hist[kTimeoutSlot], r);
+  }
 
   unsigned int theta_key = 0u;  // keep everything with key >= theta_key
   double total = 0.0, target = 0.0, m_gt = 0.0, m_ge = 0.0;
-  bool invalid = n_bad != 0;
+  bool invalid = (n_bad != 0) || (n_timeout != 0);
   if (!invalid) {
     // level 1: bins = top 11 bits of the (non-negative) pattern
     reduce_hist(cluster, sh, kL1Bins, [](int bin) { return max(bin >> 3, 1) - 150; });
@@ -339,9 +404,9 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
       for (int level = 0; level < 2; ++level) {
         const int shift = (level == 0) ? 10 : 0;
         __syncthreads();
-        for (int i = tid; i < kL23Bins; i += kThreads) sh.hist[i] = 0ull;
+        for (int i = tid; i < kL23Bins; i += kBlock) sh.hist[i] = 0ull;
         __syncthreads();
-        for (int base = 0; base < n_loc; base += kThreads) {
+        for (int base = 0; base < n_loc && worker; base += kThreads) {
           const int i = base + tid;
           unsigned int key = 0u;
           bool take = false;
@@ -371,14 +436,14 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
   const int w_lo = min(n_loc, warp * chunk);
   const int w_hi = min(n_loc, w_lo + chunk);
   int wc = 0;
-  if (!invalid) {
+  if (!invalid && worker) {
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
       const int i = i0 + lane;
       const bool keep = i < w_hi && __float_as_uint(a[i]) >= theta_key;
       wc += __popc(__ballot_sync(0xffffffffu, keep));
     }
   }
-  if (lane == 0) sh.warp_cnt[warp] = wc;
+  if (lane == 0 && worker) sh.warp_cnt[warp] = wc;
   __syncthreads();
   if (tid == 0) {
     int s = 0;
@@ -396,7 +461,7 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
     if (r < rank) offset += c;
     count += c;
   }
-  if (!invalid) {
+  if (!invalid && worker) {
     int* out = P.idx + out_list * P.idx_stride;
     long long pos = offset + sh.warp_cnt[warp];
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
@@ -411,7 +476,7 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
   if (rank == 0 && tid == 0) {
     int st = SPECATTN_ROW_OK;
     if (invalid) {
-      st = SPECATTN_ROW_INVALID_PROB;
+      st = (n_bad != 0 ? SPECATTN_ROW_INVALID_PROB : 0) | (n_timeout != 0 ? SPECATTN_ROW_TIMEOUT : 0);
       count = 0;
     } else if (count > P.idx_stride) {
       st = SPECATTN_ROW_OVERFLOW;
@@ -504,20 +569,24 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   const int cs = specattn::pick_cluster(A.L_stride, n_lists);
   const long long slice = (((A.L_stride + cs - 1) / cs) + 3) / 4 * 4;
   if (slice > specattn::kSliceCap) return SPECATTN_ERR_UNSUPPORTED;
-  const size_t smem = ((sizeof(specattn::Shared) + 15) / 16) * 16 + static_cast<size_t>(slice) * sizeof(float) + 16;
+  // shared memory: fixed part, the aggregated slice, then the per-thread staging ring
+  // (kDepth pieces of 8 KB; it later hosts the reduced histogram).  Small slices leave room
+  // for two CTAs per SM.
+  const size_t fixed = ((sizeof(specattn::Shared) + 127) / 128) * 128;
+  const size_t slice_bytes = static_cast<size_t>((slice + 31) / 32 * 32) * sizeof(float);
+  const size_t smem = fixed + slice_bytes + static_cast<size_t>(specattn::kDepth) * specattn::kChunk * sizeof(float);
+  if (smem > 224 * 1024) return SPECATTN_ERR_UNSUPPORTED;
 
-  // Opt in to large dynamic shared memory once per device (the full slice capacity), so that
-  // later calls issue nothing but the launch.
+  // Opt in to large dynamic shared memory once per device, so that later calls issue nothing
+  // but the launch.
   cudaError_t err = cudaSuccess;
   {
     static std::atomic<unsigned long long> done_mask{0};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPECATTN_ERR_CUDA;
     if (!((done_mask.load(std::memory_order_acquire) >> dev) & 1ull)) {
-      const size_t max_smem = ((sizeof(specattn::Shared) + 15) / 16) * 16 +
-                              static_cast<size_t>(specattn::kSliceCap) * sizeof(float) + 16;
       err = cudaFuncSetAttribute(specattn::select_topp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(max_smem));
+                                 224 * 1024);
       if (err != cudaSuccess) {
         cudaGetLastError();
         return SPECATTN_ERR_CUDA;
@@ -529,7 +598,7 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(static_cast<unsigned>(cs), static_cast<unsigned>(n_lists), 1);
-  cfg.blockDim = dim3(specattn::kThreads, 1, 1);
+  cfg.blockDim = dim3(specattn::kBlock, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = static_cast<cudaStream_t>(cuda_stream);
   cudaLaunchAttribute attr[1];
