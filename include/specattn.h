@@ -55,7 +55,7 @@ extern "C" {
 #define SPECATTN_MAX_DRAFT_LAYERS 64
 #define SPECATTN_MAX_DRAFT_HEADS 256
 #define SPECATTN_MAX_ROWS_PER_LIST 1024  /* contributing (head, query) rows per list */
-#define SPECATTN_MAX_KV_LEN 262144       /* positions per sequence for select (8 x 32768) */
+#define SPECATTN_MAX_KV_LEN 196608       /* positions per sequence for select (8 x 24576) */
 #define SPECATTN_MAX_VERIFY_UNITS 2048   /* batch * n_kv_heads for verify */
 #define SPECATTN_MAX_QUERY_ROWS 64       /* n_q * (n_q_heads / n_kv_heads) for verify */
 

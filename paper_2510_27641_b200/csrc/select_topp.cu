@@ -15,11 +15,17 @@
 //      the aggregated row and keeps the aggregated slice in shared memory (it is never written
 //      to global memory).  (A 1-D bulk-copy ring fed by a producer warp was measured first:
 //      like the gather in the verify kernel it stalled near 25 GB/s per SM.)
-//   2. builds the level histogram in shared memory (64-bit packed count|mantissa-sum atomics;
-//      all values of a bin share one exponent, so the mantissa sum is an exact integer and
-//      the result does not depend on the order of the atomics);
-//   3. the cluster reduces the histograms through distributed shared memory, every CTA scans
-//      the reduced bins in binary64 in one fixed order and all arrive at the same bin;
+//   2. builds the level-1 histogram in shared memory with 32-bit atomics on three arrays
+//      (count, high and low half of the mantissa sum): all values of a bin share one
+//      exponent, so the mantissa sum is an exact integer and the result does not depend on
+//      the order of the atomics.  Warps whose lanes all hit one bin (ties, the common case
+//      for attention rows) pre-reduce with redux.sync and issue three atomics in total.
+//   3. the level-1 histograms are reduced across the cluster through distributed shared
+//      memory (each CTA owns a bin range, then all gather); for levels 2 and 3 the few
+//      elements inside the threshold bin are added with remote atomics straight into CTA 0's
+//      histogram, which every CTA then reads.  Every CTA scans the reduced bins with the same
+//      warp-shuffle suffix scan in binary64, so all arrive at the same bin without a
+//      broadcast.
 //   4. after three levels the threshold is known bit-exactly; each CTA compacts its kept
 //      positions in ascending order behind the counts of the lower-ranked CTAs.
 #include <cooperative_groups.h>
@@ -41,21 +47,15 @@ extern std::atomic<long long> g_launch_count;
 
 namespace {
 
-constexpr int kThreads = 256;            // worker threads
+constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kBlock = kThreads;
 constexpr int kChunk = 2048;             // positions per staged row piece (8 KB)
 constexpr int kDepth = 8;                // row pieces in flight per thread (ring of 8 x 8 KB)
-constexpr int kL1Bins = 2048;        // sign(0) + 8 exponent bits + 3 mantissa bits
-constexpr int kL23Bins = 1024;       // 10 mantissa bits per later level
-constexpr int kHistSlots = kL1Bins + 8;  // slot kL1Bins counts invalid inputs, the next one timeouts
-constexpr int kInvalidSlot = kL1Bins;
-constexpr int kTimeoutSlot = kL1Bins + 1;
-constexpr int kGroup = 32;           // bins per scan group
-constexpr int kMaxGroups = kL1Bins / kGroup;
-constexpr int kSliceCap = 32768;     // positions per CTA
-constexpr unsigned long long kOne = 1ull << 44;  // count field of a packed bin
-constexpr unsigned long long kMantMask = kOne - 1;
+constexpr int kL1Bins = 2048;            // sign(0) + 8 exponent bits + 3 mantissa bits
+constexpr int kL23Bins = 1024;           // 10 mantissa bits per later level
+constexpr int kGroup = 32;               // bins per scan group (one warp-wide scan)
+constexpr int kSliceCap = 24576;         // positions per CTA
+constexpr unsigned int kFull = 0xffffffffu;
 
 struct SelectParams {
   const float* probs[SPECATTN_MAX_DRAFT_LAYERS];  // per used slot
@@ -74,95 +74,86 @@ struct SelectParams {
   double* diag;
 };
 
+// A histogram: element count and the mantissa sum split into two 12-bit halves, so that every
+// update is a native 32-bit shared-memory atomic (slices hold at most 2^15 elements).
+struct Hist {
+  unsigned int* cnt;
+  unsigned int* hi;
+  unsigned int* lo;
+};
+
 struct Shared {
-  unsigned long long hist[kHistSlots];
-  double* mass;        // [kL1Bins] reduced bin masses  } both alias the staging ring, which is
-  unsigned int* cnt;   // [kL1Bins] reduced bin counts  } idle once the slice is aggregated
+  unsigned int h_cnt[kL1Bins];  // level-1 histogram of this CTA
+  unsigned int h_hi[kL1Bins];
+  unsigned int h_lo[kL1Bins];
   long long row_off[SPECATTN_MAX_ROWS_PER_LIST];  // element offset of each contributing row, in add order
-  double grp_mass[kMaxGroups];
-  double suf_mass[kMaxGroups + 1];
-  unsigned int grp_cnt[kMaxGroups];
-  unsigned int suf_cnt[kMaxGroups + 1];
+  double grp_mass[kL1Bins / kGroup];
+  unsigned int grp_cnt[kL1Bins / kGroup];
   int warp_cnt[kWarps];
   int n_rows;
-  int found_group;
+  int n_invalid;            // threads of this CTA that met an invalid input
+  int local_kept;           // read by the other CTAs of the cluster
+  // result of a scan (written by warp 0)
   int found_bin;
   unsigned int cnt_above;   // elements in bins strictly above the found bin (incl. carry)
-  unsigned int cnt_bin;     // elements in the found bin
   double mass_above;        // mass strictly above the found bin (incl. carry)
   double mass_ge;           // mass_above + mass of the found bin
-  int local_kept;           // read by the other CTAs of the cluster
+  double total;             // mass of everything at this level plus the carry
 };
+
+// Layout of the dynamic shared memory behind `Shared`: the aggregated slice, then the staging
+// ring.  Once the slice is aggregated the ring is idle and hosts
+//   [0, 16 KB)   reduced bin masses (binary64)      } level scans
+//   [16, 24 KB)  reduced bin counts                 }
+//   [24, 36 KB)  level-2 histogram of the cluster (only CTA 0's copy is used)
+//   [36, 48 KB)  level-3 histogram of the cluster (only CTA 0's copy is used)
+constexpr int kRingFloats = kDepth * kChunk;
+static_assert(kRingFloats * 4 >= 48 * 1024, "the ring must hold the scan arrays");
 
 __device__ __forceinline__ double pow2_double(int k) {  // 2^k, k in the normal range
   return __longlong_as_double(static_cast<long long>(k + 1023) << 52);
-}
-
-// Adds one aggregated value to a histogram bin.  When the whole warp hits the same bin the
-// packed values are summed with shuffles and one lane issues the atomic.
-__device__ __forceinline__ void hist_add(unsigned long long* hist, bool take, int bin,
-                                         unsigned int mant) {
-  const unsigned full = 0xffffffffu;
-  const unsigned takers = __ballot_sync(full, take);
-  if (takers == 0) return;
-  const int leader = __ffs(takers) - 1;
-  const int lead_bin = __shfl_sync(full, bin, leader);
-  const bool same = __all_sync(full, !take || bin == lead_bin);
-  if (same && __popc(takers) > 4) {
-    unsigned int m = take ? mant : 0u;
-    unsigned long long v = take ? (kOne | m) : 0ull;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(full, v, o);
-    if ((threadIdx.x & 31) == leader) atomicAdd(&hist[lead_bin], v);
-  } else if (take) {
-    atomicAdd(&hist[bin], kOne | mant);
-  }
 }
 
 __device__ __forceinline__ unsigned int mantissa_of(unsigned int key) {
   return (key >> 23) ? ((key & 0x7fffffu) | 0x800000u) : (key & 0x7fffffu);
 }
 
-// Cluster-wide reduction of the per-CTA histograms into (cnt, mass) for `nbins` bins, the
-// result replicated in every CTA.  `exp_of_bin(bin)` gives the binary exponent that scales the
-// integer mantissa sum of that bin.
-template <typename ExpFn>
-__device__ void reduce_hist(cg::cluster_group& cluster, Shared& sh, int nbins, ExpFn exp_of_bin) {
-  const unsigned cs = cluster.num_blocks();
-  const unsigned rank = cluster.block_rank();
-  const int per = nbins / static_cast<int>(cs);
-  double* const mass = sh.mass;
-  unsigned int* const cnt = sh.cnt;
-  cluster.sync();  // every CTA's histogram is complete
-  const int lo = static_cast<int>(rank) * per;
-  for (int bin = lo + threadIdx.x; bin < lo + per && threadIdx.x < kThreads; bin += kThreads) {
-    unsigned long long s = 0;
-    for (unsigned r = 0; r < cs; ++r) s += *cluster.map_shared_rank(&sh.hist[bin], r);
-    cnt[bin] = static_cast<unsigned int>(s >> 44);
-    mass[bin] = static_cast<double>(s & kMantMask) * pow2_double(exp_of_bin(bin));
-  }
-  cluster.sync();  // every owner's part is reduced; remote histograms are no longer read
-  for (int bin = threadIdx.x; bin < nbins && threadIdx.x < kThreads; bin += kThreads) {
-    const unsigned owner = static_cast<unsigned>(bin / per);
-    if (owner != rank) {
-      cnt[bin] = *cluster.map_shared_rank(&cnt[bin], owner);
-      mass[bin] = *cluster.map_shared_rank(&mass[bin], owner);
+// Adds one value to a histogram bin (all 32 lanes call this together).  When every taking
+// lane hits the same bin the warp pre-reduces and one lane issues the three atomics.
+__device__ __forceinline__ void hist_add(const Hist& h, bool take, int bin, unsigned int mant) {
+  const unsigned takers = __ballot_sync(kFull, take);
+  if (takers == 0) return;
+  const int leader = __ffs(takers) - 1;
+  const int lead_bin = __shfl_sync(kFull, bin, leader);
+  const bool same = __all_sync(kFull, !take || bin == lead_bin);
+  if (same && __popc(takers) > 2) {
+    const unsigned int shi = __reduce_add_sync(kFull, take ? (mant >> 12) : 0u);
+    const unsigned int slo = __reduce_add_sync(kFull, take ? (mant & 0xfffu) : 0u);
+    if ((threadIdx.x & 31) == leader) {
+      atomicAdd(&h.cnt[lead_bin], static_cast<unsigned int>(__popc(takers)));
+      atomicAdd(&h.hi[lead_bin], shi);
+      atomicAdd(&h.lo[lead_bin], slo);
     }
+  } else if (take) {
+    atomicAdd(&h.cnt[bin], 1u);
+    atomicAdd(&h.hi[bin], mant >> 12);
+    atomicAdd(&h.lo[bin], mant & 0xfffu);
   }
-  __syncthreads();
 }
 
-// Finds the highest bin at which the mass accumulated from the top (starting from
-// `carry_mass` / `carry_cnt` already above this level) reaches `target`.  All sums run in one
-// fixed order, so every CTA of a cluster gets the same answer.  Results go to sh.found_bin,
-// sh.mass_above, sh.mass_ge, sh.cnt_above, sh.cnt_bin.  Returns the mass of everything at
-// this level plus the carry (the row total at level 1).
-__device__ double scan_bins(Shared& sh, int nbins, double carry_mass, unsigned int carry_cnt,
-                            double target, bool target_is_fraction, float p) {
+__device__ __forceinline__ double shfl_down_f64(double v, int d) { return __shfl_down_sync(kFull, v, d); }
+
+// Scan of `nbins` reduced bins (nbins = 32 * groups, groups <= 64): finds the highest bin at
+// which the mass accumulated from the top -- starting from `carry_mass` / `carry_cnt` already
+// above this level -- reaches `target` (or p * everything when `target_is_fraction`).  All
+// sums run in one fixed order (per-group serial sums, then shuffle suffix scans in warp 0), so
+// every CTA of a cluster gets bit-identical results.  Results land in sh.found_bin,
+// sh.mass_above, sh.mass_ge, sh.cnt_above, sh.total.  Called by all threads.
+__device__ void scan_bins(Shared& sh, const double* mass, const unsigned int* cnt, int nbins, double carry_mass,
+                          unsigned int carry_cnt, double target, bool target_is_fraction, float p) {
   const int groups = nbins / kGroup;
   const int tid = threadIdx.x;
-  const double* const mass = sh.mass;
-  const unsigned int* const cnt = sh.cnt;
+  const int lane = tid & 31;
   if (tid < groups) {
     double s = 0.0;
     unsigned int c = 0;
@@ -174,68 +165,116 @@ __device__ double scan_bins(Shared& sh, int nbins, double carry_mass, unsigned i
     sh.grp_cnt[tid] = c;
   }
   __syncthreads();
-  if (tid == 0) {
-    double s = carry_mass;
-    unsigned int c = carry_cnt;
-    sh.suf_mass[groups] = s;
-    sh.suf_cnt[groups] = c;
-    for (int j = groups - 1; j >= 0; --j) {
-      s += sh.grp_mass[j];
-      c += sh.grp_cnt[j];
-      sh.suf_mass[j] = s;
-      sh.suf_cnt[j] = c;
-    }
-    sh.found_group = -1;
-  }
-  __syncthreads();
-  const double all = sh.suf_mass[0];
-  if (target_is_fraction) target = static_cast<double>(p) * all;
-  if (tid < groups && sh.suf_mass[tid + 1] < target && target <= sh.suf_mass[tid])
-    sh.found_group = tid;  // the suffix sums are monotone: at most one group qualifies
-  __syncthreads();
-  if (tid == 0) {
-    int j = sh.found_group;
-    if (j < 0) {  // only reachable through rounding at the very bottom: take the lowest group
-      j = 0;
-      while (j < groups - 1 && sh.grp_cnt[j] == 0) ++j;
-    }
-    double s = sh.suf_mass[j + 1];
-    unsigned int c = sh.suf_cnt[j + 1];
-    int found = -1;
-    double prev = s;
-    unsigned int cprev = c;
-    int last_bin = -1;
-    for (int b = kGroup - 1; b >= 0; --b) {
-      const int bin = j * kGroup + b;
-      const unsigned int cb = cnt[bin];
-      if (cb == 0) continue;
-      prev = s;
-      cprev = c;
-      s += mass[bin];
-      c += cb;
-      last_bin = bin;
-      if (target <= s) {
-        found = bin;
-        break;
+  if (tid < 32) {
+    // lane l owns groups 2l (low) and 2l+1 (high) when there are 64 groups, group l otherwise
+    const bool two = groups > 32;
+    const double g_hi = two ? sh.grp_mass[2 * lane + 1] : sh.grp_mass[lane];
+    const double g_lo = two ? sh.grp_mass[2 * lane] : 0.0;
+    const unsigned int c_hi = two ? sh.grp_cnt[2 * lane + 1] : sh.grp_cnt[lane];
+    const unsigned int c_lo = two ? sh.grp_cnt[2 * lane] : 0u;
+    // inclusive suffix sums over lanes (lane 31 holds the top groups)
+    double s = g_hi + g_lo;
+    unsigned int c = c_hi + c_lo;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const double sv = shfl_down_f64(s, d);
+      const unsigned int cv = __shfl_down_sync(kFull, c, d);
+      if (lane + d < 32) {
+        s += sv;
+        c += cv;
       }
     }
-    if (found < 0) found = last_bin;  // rounding between the two summation orders
-    if (found < 0) {                  // empty level (cannot happen with target > 0)
-      found = 0;
-      prev = s;
-      cprev = c;
+    // mass / count of everything strictly above this lane's groups, plus the carry
+    double above = shfl_down_f64(s, 1);
+    unsigned int cabove = __shfl_down_sync(kFull, c, 1);
+    if (lane == 31) {
+      above = 0.0;
+      cabove = 0u;
     }
-    sh.found_bin = found;
-    sh.mass_above = prev;
-    sh.mass_ge = s;
-    sh.cnt_above = cprev;
-    sh.cnt_bin = c - cprev;
+    above += carry_mass;
+    cabove += carry_cnt;
+    const double all = __shfl_sync(kFull, s, 0) + carry_mass;
+    if (target_is_fraction) target = static_cast<double>(p) * all;
+    // suffix mass including the high group, and including both
+    const double with_hi = above + g_hi;
+    const double with_lo = with_hi + g_lo;
+    // highest group whose inclusive suffix reaches the target
+    const bool hit_hi = (c_hi != 0u) && (with_hi >= target);
+    const bool hit_lo = two && (c_lo != 0u) && (with_lo >= target);
+    const unsigned hits = __ballot_sync(kFull, hit_hi || hit_lo);
+    int grp;            // chosen group
+    int src;            // lane that owns it
+    bool pick_hi;
+    if (hits != 0u) {
+      src = 31 - __clz(hits);
+      pick_hi = __shfl_sync(kFull, hit_hi ? 1 : 0, src) != 0;
+      grp = two ? (2 * src + (pick_hi ? 1 : 0)) : src;
+    } else {
+      // only reachable through rounding between two summation orders: take the lowest
+      // non-empty group, i.e. everything at this level is kept
+      const unsigned ne_lo = __ballot_sync(kFull, two ? (c_lo != 0u) : (c_hi != 0u));
+      const unsigned ne_hi = __ballot_sync(kFull, two && (c_hi != 0u));
+      int g0 = -1;
+      for (int l = 0; l < 32 && g0 < 0; ++l) {
+        if (two) {
+          if ((ne_lo >> l) & 1u) g0 = 2 * l;
+          else if ((ne_hi >> l) & 1u) g0 = 2 * l + 1;
+        } else if ((ne_lo >> l) & 1u) {
+          g0 = l;
+        }
+      }
+      if (g0 < 0) g0 = 0;
+      grp = g0;
+      src = two ? (g0 >> 1) : g0;
+      pick_hi = two ? ((g0 & 1) != 0) : true;
+    }
+    // mass / count strictly above the chosen group (incl. carry)
+    const double b_hi = __shfl_sync(kFull, above, src), b_lo = __shfl_sync(kFull, with_hi, src);
+    const unsigned int cb_hi = __shfl_sync(kFull, cabove, src), cb_lo = __shfl_sync(kFull, cabove + c_hi, src);
+    const double base = pick_hi ? b_hi : b_lo;
+    const unsigned int cbase = pick_hi ? cb_hi : cb_lo;
+    // inside the group: lane b <-> bin grp * 32 + b, inclusive suffix over lanes
+    const double m = mass[grp * kGroup + lane];
+    const unsigned int cb = cnt[grp * kGroup + lane];
+    double si = m;
+    unsigned int ci = cb;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const double sv = shfl_down_f64(si, d);
+      const unsigned int cv = __shfl_down_sync(kFull, ci, d);
+      if (lane + d < 32) {
+        si += sv;
+        ci += cv;
+      }
+    }
+    const double incl = base + si;  // mass of bins >= this one (incl. carry)
+    double ab = shfl_down_f64(si, 1);
+    unsigned int cab = __shfl_down_sync(kFull, ci, 1);
+    if (lane == 31) {
+      ab = 0.0;
+      cab = 0u;
+    }
+    const unsigned ok = __ballot_sync(kFull, cb != 0u && incl >= target);
+    const unsigned nonempty = __ballot_sync(kFull, cb != 0u);
+    int fb;
+    if (ok != 0u) fb = 31 - __clz(ok);
+    else if (nonempty != 0u) fb = __ffs(nonempty) - 1;  // rounding: keep the whole group
+    else fb = 0;
+    const double f_above = base + __shfl_sync(kFull, ab, fb);
+    const double f_ge = __shfl_sync(kFull, incl, fb);
+    const unsigned int f_cabove = cbase + __shfl_sync(kFull, cab, fb);
+    if (lane == 0) {
+      sh.found_bin = grp * kGroup + fb;
+      sh.mass_above = f_above;
+      sh.mass_ge = f_ge;
+      sh.cnt_above = f_cabove;
+      sh.total = all;
+    }
   }
   __syncthreads();
-  return all;
 }
 
-__global__ void __launch_bounds__(kBlock, 2) select_topp_kernel(const __grid_constant__ SelectParams P) {
+__global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_constant__ SelectParams P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
   float* a = reinterpret_cast<float*>(smem_raw + ((sizeof(Shared) + 127) / 128) * 128);
@@ -246,7 +285,6 @@ __global__ void __launch_bounds__(kBlock, 2) select_topp_kernel(const __grid_con
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int warp = tid >> 5;
-  const bool worker = tid < kThreads;
 
   const int list = blockIdx.y;  // (used slot, sequence, group)
   const int g = list % P.G;
@@ -272,23 +310,25 @@ __global__ void __launch_bounds__(kBlock, 2) select_topp_kernel(const __grid_con
       for (int s = 0; s < P.gamma; ++s) sh.row_off[n++] = static_cast<long long>(h * P.gamma + s) * P.L_stride;
     }
     sh.n_rows = n;
+    sh.n_invalid = 0;
   }
-  for (int i = tid; i < kHistSlots; i += kBlock) sh.hist[i] = 0ull;
+  for (int i = tid; i < kL1Bins; i += kThreads) sh.h_cnt[i] = sh.h_hi[i] = sh.h_lo[i] = 0u;
   __syncthreads();
   const int R = sh.n_rows;
+
+  // dynamic shared memory behind the fixed part
+  const int slice_cap = static_cast<int>(((((P.L_stride + cs - 1) / cs + 3) & ~3ll) + 31) & ~31ll);
+  float* ring = a + slice_cap;
+  double* const r_mass = reinterpret_cast<double*>(ring);
+  unsigned int* const r_cnt = reinterpret_cast<unsigned int*>(ring + 4096);
+  unsigned int* const lvl_base = reinterpret_cast<unsigned int*>(ring + 6144);  // 2 levels x 3 x 1024
+  const Hist h1 = {sh.h_cnt, sh.h_hi, sh.h_lo};
 
   // ---- 1+2: aggregate the slice and build the level-1 histogram ------------------------------
   const float* A = P.probs[slot] + static_cast<long long>(b) * P.H * P.gamma * P.L_stride + lo;
   const int n4 = (n_loc + 3) >> 2;
   const int n_pos4 = n4 * 4;                       // slice length rounded up to whole float4s
   const int n_chunks = (n_pos4 + kChunk - 1) / kChunk;
-  // ring buffers follow the aggregated slice (whose capacity is fixed by the launch)
-  const int slice_cap4 = ((((P.L_stride + cs - 1) / cs + 3) & ~3ll) + 31) & ~31ll;
-  float* ring = a + slice_cap4;
-  if (tid == 0) {
-    sh.mass = reinterpret_cast<double*>(ring);
-    sh.cnt = reinterpret_cast<unsigned int*>(ring + 2 * kL1Bins);
-  }
   bool bad = false;
   // Pieces are numbered q = chunk * R + row, i.e. in the order the adds must happen.  Every
   // thread copies exactly the two float4 columns of a piece that it will add itself, with
@@ -317,7 +357,7 @@ __global__ void __launch_bounds__(kBlock, 2) select_topp_kernel(const __grid_con
     // invalid value a sum can hide) -- NaN and Inf survive into the aggregated value itself.
     float4 acc[2], mn[2];
     acc[0] = acc[1] = mn[0] = mn[1] = make_float4(0.f, 0.f, 0.f, 0.f);
-    int slot = 0;
+    int slot_c = 0;
     for (int c = 0; c < n_chunks; ++c) {
       const int len4 = min(kChunk, n_pos4 - c * kChunk) >> 2;
       // positions of this thread's two float4s that lie beyond the slice (last float4 only)
@@ -327,15 +367,15 @@ __global__ void __launch_bounds__(kBlock, 2) select_topp_kernel(const __grid_con
       for (int r = 0; r < R; ++r) {
         issue();
         asm volatile("cp.async.wait_group %0;" ::"n"(kDepth - 1) : "memory");
-        const float4* piece = reinterpret_cast<const float4*>(ring + slot * kChunk);
-        slot = (slot + 1) & (kDepth - 1);
+        const float4* piece = reinterpret_cast<const float4*>(ring + slot_c * kChunk);
+        slot_c = (slot_c + 1) & (kDepth - 1);
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
           const int i4 = tid + k * kThreads;
           if (i4 < len4) {
             float4 x = piece[i4];
             if (cut[k] < 4) {  // values beyond kv_len are not inputs
-              if (cut[k] < 4) x.w = 0.f;
+              x.w = 0.f;
               if (cut[k] < 3) x.z = 0.f;
               if (cut[k] < 2) x.y = 0.f;
             }
@@ -368,66 +408,105 @@ __global__ void __launch_bounds__(kBlock, 2) select_topp_kernel(const __grid_con
           const unsigned int key = __float_as_uint(vals[e]);
           // zeros carry no mass and can never be the threshold of a row with positive total
           const bool take = act && (pos + e < n_loc) && key != 0u && !(key >> 31);
-          hist_add(sh.hist, take, static_cast<int>(key >> 20), mantissa_of(key));
+          hist_add(h1, take, static_cast<int>(key >> 20), mantissa_of(key));
         }
         acc[k] = mn[k] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
   }
-  if (bad) atomicAdd(&sh.hist[kInvalidSlot], 1ull);
+  if (bad) atomicAdd(&sh.n_invalid, 1);
   __syncthreads();
+  // the ring is idle from here on: CTA 0 zeroes the cluster's level-2 and level-3 histograms
+  if (rank == 0)
+    for (int i = tid; i < 2 * 3 * kL23Bins; i += kThreads) lvl_base[i] = 0u;
 
   // ---- 3: threshold search --------------------------------------------------------------------
-  // invalid inputs anywhere in the cluster?
-  cluster.sync();
-  unsigned long long n_bad = 0, n_timeout = 0;
-  for (int r = 0; r < cs; ++r) {
-    n_bad += *cluster.map_shared_rank(&sh.hist[kInvalidSlot], r);
-    n_timeout += *cluster.map_shared_rank(&sh.hist[kTimeoutSlot], r);
-  }
+  cluster.sync();  // every CTA's level-1 histogram and invalid count are complete
+  int n_bad = 0;
+  for (int r = 0; r < cs; ++r) n_bad += *cluster.map_shared_rank(&sh.n_invalid, r);
 
   unsigned int theta_key = 0u;  // keep everything with key >= theta_key
   double total = 0.0, target = 0.0, m_gt = 0.0, m_ge = 0.0;
-  bool invalid = (n_bad != 0) || (n_timeout != 0);
-  if (!invalid) {
-    // level 1: bins = top 11 bits of the (non-negative) pattern
-    reduce_hist(cluster, sh, kL1Bins, [](int bin) { return max(bin >> 3, 1) - 150; });
-    total = scan_bins(sh, kL1Bins, 0.0, 0u, 0.0, true, P.p);
-    target = static_cast<double>(P.p) * total;
-    if (target > 0.0 && !P.keep_all) {
-      const int b1 = sh.found_bin;
-      const int e1 = max(b1 >> 3, 1) - 150;
-      unsigned int prefix = static_cast<unsigned int>(b1);
-      double carry_m = sh.mass_above;
-      unsigned int carry_c = sh.cnt_above;
-      for (int level = 0; level < 2; ++level) {
-        const int shift = (level == 0) ? 10 : 0;
-        __syncthreads();
-        for (int i = tid; i < kL23Bins; i += kBlock) sh.hist[i] = 0ull;
-        __syncthreads();
-        for (int base = 0; base < n_loc && worker; base += kThreads) {
-          const int i = base + tid;
-          unsigned int key = 0u;
-          bool take = false;
-          if (i < n_loc) {
-            key = __float_as_uint(a[i]);
-            take = (key >> (shift + 10)) == prefix;
-          }
-          hist_add(sh.hist, take, static_cast<int>((key >> shift) & 1023u), mantissa_of(key));
-        }
-        reduce_hist(cluster, sh, kL23Bins, [e1](int) { return e1; });
-        scan_bins(sh, kL23Bins, carry_m, carry_c, target, false, P.p);
-        prefix = (prefix << 10) | static_cast<unsigned int>(sh.found_bin);
-        carry_m = sh.mass_above;
-        carry_c = sh.cnt_above;
+  const bool invalid = n_bad != 0;
+  bool searching = !invalid;
+  if (searching) {
+    // level 1: every CTA reduces its own range of bins over the cluster, then all gather
+    const int per_bins = kL1Bins / cs;
+    const int blo = rank * per_bins;
+    for (int bin = blo + tid; bin < blo + per_bins; bin += kThreads) {
+      unsigned long long c = 0, mh = 0, ml = 0;
+      for (int r = 0; r < cs; ++r) {
+        c += *cluster.map_shared_rank(&sh.h_cnt[bin], r);
+        mh += *cluster.map_shared_rank(&sh.h_hi[bin], r);
+        ml += *cluster.map_shared_rank(&sh.h_lo[bin], r);
       }
-      theta_key = prefix;
-      m_gt = sh.mass_above;
-      m_ge = sh.mass_ge;
-    } else {
-      m_ge = total;  // p >= 1, or an all-zero row where everything ties at zero: keep all
+      r_cnt[bin] = static_cast<unsigned int>(c);
+      r_mass[bin] = static_cast<double>((mh << 12) + ml) * pow2_double(max(bin >> 3, 1) - 150);
     }
+  }
+  cluster.sync();  // every owner's range is reduced
+  if (searching) {
+    const int per_bins = kL1Bins / cs;
+    for (int bin = tid; bin < kL1Bins; bin += kThreads) {
+      const int owner = bin / per_bins;
+      if (owner != rank) {
+        r_cnt[bin] = *cluster.map_shared_rank(&r_cnt[bin], owner);
+        r_mass[bin] = *cluster.map_shared_rank(&r_mass[bin], owner);
+      }
+    }
+    __syncthreads();
+    scan_bins(sh, r_mass, r_cnt, kL1Bins, 0.0, 0u, 0.0, true, P.p);
+    total = sh.total;
+    target = static_cast<double>(P.p) * total;
+    m_ge = total;
+    searching = (target > 0.0) && !P.keep_all;  // else: p >= 1 or an all-zero row -> keep all
+  }
+  // Levels 2 and 3 refine inside the found bin.  The cluster syncs are executed by every
+  // CTA whatever it decided (the decisions are identical across the cluster anyway).
+  unsigned int prefix = searching ? static_cast<unsigned int>(sh.found_bin) : 0u;
+  const int e1 = max(static_cast<int>(prefix >> 3), 1) - 150;
+  double carry_m = searching ? sh.mass_above : 0.0;
+  unsigned int carry_c = searching ? sh.cnt_above : 0u;
+  for (int level = 0; level < 2; ++level) {
+    const int shift = (level == 0) ? 10 : 0;
+    unsigned int* lb = lvl_base + level * 3 * kL23Bins;
+    if (searching) {
+      // the few elements inside the threshold bin go straight into CTA 0's histogram
+      const Hist hr = {cluster.map_shared_rank(lb, 0), cluster.map_shared_rank(lb + kL23Bins, 0),
+                       cluster.map_shared_rank(lb + 2 * kL23Bins, 0)};
+      for (int base = 0; base < n_loc; base += kThreads) {
+        const int i = base + tid;
+        unsigned int key = 0u;
+        bool take = false;
+        if (i < n_loc) {
+          key = __float_as_uint(a[i]);
+          take = (key >> (shift + 10)) == prefix;
+        }
+        hist_add(hr, take, static_cast<int>((key >> shift) & 1023u), mantissa_of(key));
+      }
+    }
+    cluster.sync();  // all remote atomics of this level have landed
+    if (searching) {
+      const unsigned int* src = cluster.map_shared_rank(lb, 0);
+      const double scale = pow2_double(e1);
+      __syncthreads();  // the previous scan no longer reads the arrays overwritten below
+      for (int bin = tid; bin < kL23Bins; bin += kThreads) {
+        const unsigned long long mh = src[kL23Bins + bin], ml = src[2 * kL23Bins + bin];
+        r_cnt[bin] = src[bin];
+        r_mass[bin] = static_cast<double>((mh << 12) + ml) * scale;
+      }
+      __syncthreads();
+      scan_bins(sh, r_mass, r_cnt, kL23Bins, carry_m, carry_c, target, false, P.p);
+      prefix = (prefix << 10) | static_cast<unsigned int>(sh.found_bin);
+      carry_m = sh.mass_above;
+      carry_c = sh.cnt_above;
+    }
+  }
+  if (searching) {
+    theta_key = prefix;
+    m_gt = sh.mass_above;
+    m_ge = sh.mass_ge;
   }
 
   // ---- 4: ordered compaction --------------------------------------------------------------------
@@ -436,14 +515,14 @@ __global__ void __launch_bounds__(kBlock, 2) select_topp_kernel(const __grid_con
   const int w_lo = min(n_loc, warp * chunk);
   const int w_hi = min(n_loc, w_lo + chunk);
   int wc = 0;
-  if (!invalid && worker) {
+  if (!invalid) {
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
       const int i = i0 + lane;
       const bool keep = i < w_hi && __float_as_uint(a[i]) >= theta_key;
-      wc += __popc(__ballot_sync(0xffffffffu, keep));
+      wc += __popc(__ballot_sync(kFull, keep));
     }
   }
-  if (lane == 0 && worker) sh.warp_cnt[warp] = wc;
+  if (lane == 0) sh.warp_cnt[warp] = wc;
   __syncthreads();
   if (tid == 0) {
     int s = 0;
@@ -461,13 +540,13 @@ __global__ void __launch_bounds__(kBlock, 2) select_topp_kernel(const __grid_con
     if (r < rank) offset += c;
     count += c;
   }
-  if (!invalid && worker) {
+  if (!invalid) {
     int* out = P.idx + out_list * P.idx_stride;
     long long pos = offset + sh.warp_cnt[warp];
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
       const int i = i0 + lane;
       const bool keep = i < w_hi && __float_as_uint(a[i]) >= theta_key;
-      const unsigned m = __ballot_sync(0xffffffffu, keep);
+      const unsigned m = __ballot_sync(kFull, keep);
       const long long my = pos + __popc(m & ((1u << lane) - 1u));
       if (keep && my < P.idx_stride) out[my] = lo + i;
       pos += __popc(m);
@@ -476,7 +555,7 @@ __global__ void __launch_bounds__(kBlock, 2) select_topp_kernel(const __grid_con
   if (rank == 0 && tid == 0) {
     int st = SPECATTN_ROW_OK;
     if (invalid) {
-      st = (n_bad != 0 ? SPECATTN_ROW_INVALID_PROB : 0) | (n_timeout != 0 ? SPECATTN_ROW_TIMEOUT : 0);
+      st = SPECATTN_ROW_INVALID_PROB;
       count = 0;
     } else if (count > P.idx_stride) {
       st = SPECATTN_ROW_OVERFLOW;
@@ -542,8 +621,8 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   if (A.head_group != nullptr) {
     for (int h = 0; h < A.n_draft_heads; ++h) {
       if (A.head_group[h] < 0 || A.head_group[h] >= A.n_groups) return SPECATTN_ERR_RANGE;
-      P.head_group[h] = static_cast<signed char>(A.head_group[h] & 0x7f);
       if (A.head_group[h] > 127) return SPECATTN_ERR_UNSUPPORTED;
+      P.head_group[h] = static_cast<signed char>(A.head_group[h]);
     }
     P.has_groups = 1;
   }
@@ -570,11 +649,11 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   const long long slice = (((A.L_stride + cs - 1) / cs) + 3) / 4 * 4;
   if (slice > specattn::kSliceCap) return SPECATTN_ERR_UNSUPPORTED;
   // shared memory: fixed part, the aggregated slice, then the per-thread staging ring
-  // (kDepth pieces of 8 KB; it later hosts the reduced histogram).  Small slices leave room
-  // for two CTAs per SM.
+  // (kDepth pieces of 8 KB; it later hosts the scan arrays).  Small slices leave room for two
+  // CTAs per SM.
   const size_t fixed = ((sizeof(specattn::Shared) + 127) / 128) * 128;
   const size_t slice_bytes = static_cast<size_t>((slice + 31) / 32 * 32) * sizeof(float);
-  const size_t smem = fixed + slice_bytes + static_cast<size_t>(specattn::kDepth) * specattn::kChunk * sizeof(float);
+  const size_t smem = fixed + slice_bytes + static_cast<size_t>(specattn::kRingFloats) * sizeof(float);
   if (smem > 224 * 1024) return SPECATTN_ERR_UNSUPPORTED;
 
   // Opt in to large dynamic shared memory once per device, so that later calls issue nothing
@@ -598,7 +677,7 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(static_cast<unsigned>(cs), static_cast<unsigned>(n_lists), 1);
-  cfg.blockDim = dim3(specattn::kBlock, 1, 1);
+  cfg.blockDim = dim3(specattn::kThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = static_cast<cudaStream_t>(cuda_stream);
   cudaLaunchAttribute attr[1];
