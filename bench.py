@@ -280,36 +280,41 @@ def run_reference(args, cfg):
 
 
 # ----------------------------------------------------------------------------------------------
-def topp_sweep(dev, reps=10):
-    """Selection micro-benchmark: 256 rows x n x p x family, rows/s per cell (R = 1)."""
+def topp_sweep(dev, reps=5):
+    """Selection micro-benchmark: 256 rows x n x p x family, rows/s per cell (R = 1).
+    Each cell is timed as a CUDA graph of launches over rotating copies of the rows (at least
+    256 MB in total, so every launch reads cold data), replayed `reps` times."""
+    import ctypes as C
     import torch
     import paper_2510_27641_b200 as sa
     import workloads as wl
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     out = {}
     for fam in wl.TOPP_FAMILIES:
         for n in wl.TOPP_SIZES:
-            rows = torch.from_numpy(wl.topp_rows(fam, 256, n, seed=2)).to(dev).view(256, 1, 1, n)
+            base = torch.from_numpy(wl.topp_rows(fam, 256, n, seed=2)).to(dev).view(256, 1, 1, n)
+            copies = max(2, min(64, (256 << 20) // (256 * n * 4)))
+            rows = [base.clone() for _ in range(copies)]
             kv = torch.full((256,), n, dtype=torch.int32, device=dev)
             idx = torch.empty((1, 256, 1, n), dtype=torch.int32, device=dev)
             cnt = torch.empty((1, 256, 1), dtype=torch.int32, device=dev)
             st = torch.empty((1, 256, 1), dtype=torch.int32, device=dev)
             for p in wl.TOPP_PS:
-                ts = []
-                for r in range(reps + 3):
-                    flush.zero_()
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                    sa.select_topp([rows], kv, [0], p, idx=idx, counts=cnt, row_status=st)
-                    e1.record()
-                    torch.cuda.synchronize()
-                    if r >= 3:
-                        ts.append(e0.elapsed_time(e1) * 1e3)
-                us = float(np.median(ts))
+                args = [sa.make_select_args([r], kv, [0], p, idx=idx, counts=cnt, row_status=st) for r in rows]
+
+                def launch_all():
+                    sp = sa._stream_ptr(None)
+                    for a, _keep in args:
+                        rc = sa.lib().specattn_select_topp(C.byref(a), sp)
+                        assert rc == 0, rc
+                launch_all()
+                torch.cuda.synchronize()
+                g, _ = capture(launch_all)
+                us = time_replays(g, reps, 2) / copies
                 out[f"{fam}/n={n}/p={p}"] = {"us": round(us, 2), "rows_per_s": round(256 / us * 1e6),
                                              "gbs": round(256 * n * 4 / us / 1e3, 1),
                                              "kept_mean": float(cnt.float().mean().item())}
-            del rows, idx
+                del g
+            del rows, idx, base
     return out
 
 

@@ -15,17 +15,18 @@
 //      the aggregated row and keeps the aggregated slice in shared memory (it is never written
 //      to global memory).  (A 1-D bulk-copy ring fed by a producer warp was measured first:
 //      like the gather in the verify kernel it stalled near 25 GB/s per SM.)
-//   2. builds the level-1 histogram in shared memory with 32-bit atomics on three arrays
-//      (count, high and low half of the mantissa sum): all values of a bin share one
-//      exponent, so the mantissa sum is an exact integer and the result does not depend on
-//      the order of the atomics.  Warps whose lanes all hit one bin (ties, the common case
-//      for attention rows) pre-reduce with redux.sync and issue three atomics in total.
-//   3. the level-1 histograms are reduced across the cluster through distributed shared
-//      memory (each CTA owns a bin range, then all gather); for levels 2 and 3 the few
-//      elements inside the threshold bin are added with remote atomics straight into CTA 0's
-//      histogram, which every CTA then reads.  Every CTA scans the reduced bins with the same
-//      warp-shuffle suffix scan in binary64, so all arrive at the same bin without a
-//      broadcast.
+//   2. builds the level-1 histogram of mantissa sums in shared memory: all values of a bin
+//      share one exponent, so the sum of their 24-bit mantissas is an exact integer and the
+//      result does not depend on the order of the updates.  The sum is kept as two 32-bit
+//      words (low 16 and high 8 mantissa bits), each updated with a fire-and-forget 32-bit
+//      reduction, so consecutive updates pipeline.  Warps whose lanes all hit one bin (ties,
+//      the common case for attention rows) pre-reduce with redux.sync first.
+//   3. the histograms are reduced across the cluster through distributed shared memory: at
+//      level 1 each CTA owns a bin range and all gather the result; at levels 2 and 3 (only
+//      the elements inside the threshold bin) every CTA reads all peers' histograms itself.
+//      Every CTA scans the reduced bins with the same warp-shuffle suffix scan in binary64,
+//      so all arrive at the same bin without a broadcast.  (Remote atomics into one CTA's
+//      histogram were measured first and cost ~11 us per level on tie-free rows.)
 //   4. after three levels the threshold is known bit-exactly; each CTA compacts its kept
 //      positions in ascending order behind the counts of the lower-ranked CTAs.
 #include <cooperative_groups.h>
@@ -74,28 +75,26 @@ struct SelectParams {
   double* diag;
 };
 
-// A histogram: element count and the mantissa sum split into two 12-bit halves, so that every
-// update is a native 32-bit shared-memory atomic (slices hold at most 2^15 elements).
+// A histogram of exact mantissa sums, kept as two 32-bit words: `lo` sums the low 16 mantissa
+// bits, `hi` the high 8 (a slice holds < 2^15 elements, so neither can wrap) and the total is
+// (hi << 16) + lo.  Updates never read a value back.  A bin is empty iff its sum is zero (zeros
+// are never entered, every other value has a non-zero mantissa).
 struct Hist {
-  unsigned int* cnt;
-  unsigned int* hi;
   unsigned int* lo;
+  unsigned int* hi;
 };
 
 struct Shared {
-  unsigned int h_cnt[kL1Bins];  // level-1 histogram of this CTA
+  unsigned int h_lo[kL1Bins];  // level-1 histogram of this CTA
   unsigned int h_hi[kL1Bins];
-  unsigned int h_lo[kL1Bins];
   long long row_off[SPECATTN_MAX_ROWS_PER_LIST];  // element offset of each contributing row, in add order
   double grp_mass[kL1Bins / kGroup];
-  unsigned int grp_cnt[kL1Bins / kGroup];
   int warp_cnt[kWarps];
   int n_rows;
   int n_invalid;            // threads of this CTA that met an invalid input
   int local_kept;           // read by the other CTAs of the cluster
   // result of a scan (written by warp 0)
   int found_bin;
-  unsigned int cnt_above;   // elements in bins strictly above the found bin (incl. carry)
   double mass_above;        // mass strictly above the found bin (incl. carry)
   double mass_ge;           // mass_above + mass of the found bin
   double total;             // mass of everything at this level plus the carry
@@ -103,12 +102,11 @@ struct Shared {
 
 // Layout of the dynamic shared memory behind `Shared`: the aggregated slice, then the staging
 // ring.  Once the slice is aggregated the ring is idle and hosts
-//   [0, 16 KB)   reduced bin masses (binary64)      } level scans
-//   [16, 24 KB)  reduced bin counts                 }
-//   [24, 36 KB)  level-2 histogram of the cluster (only CTA 0's copy is used)
-//   [36, 48 KB)  level-3 histogram of the cluster (only CTA 0's copy is used)
+//   [0, 16 KB)   reduced bin masses (binary64), read by the level scans
+//   [16, 24 KB)  level-2 histogram of this CTA (low and high words)
+//   [24, 32 KB)  level-3 histogram of this CTA
 constexpr int kRingFloats = kDepth * kChunk;
-static_assert(kRingFloats * 4 >= 48 * 1024, "the ring must hold the scan arrays");
+static_assert(kRingFloats * 4 >= 32 * 1024, "the ring must hold the scan arrays");
 
 __device__ __forceinline__ double pow2_double(int k) {  // 2^k, k in the normal range
   return __longlong_as_double(static_cast<long long>(k + 1023) << 52);
@@ -118,51 +116,45 @@ __device__ __forceinline__ unsigned int mantissa_of(unsigned int key) {
   return (key >> 23) ? ((key & 0x7fffffu) | 0x800000u) : (key & 0x7fffffu);
 }
 
+__device__ __forceinline__ void hist_bump(const Hist& h, int bin, unsigned int lo, unsigned int hi) {
+  atomicAdd(&h.lo[bin], lo);
+  atomicAdd(&h.hi[bin], hi);
+}
+
 // Adds one value to a histogram bin (all 32 lanes call this together).  When every taking
-// lane hits the same bin the warp pre-reduces and one lane issues the three atomics.
+// lane hits the same bin the warp pre-reduces and one lane issues the atomic.
 __device__ __forceinline__ void hist_add(const Hist& h, bool take, int bin, unsigned int mant) {
   const unsigned takers = __ballot_sync(kFull, take);
   if (takers == 0) return;
   const int leader = __ffs(takers) - 1;
   const int lead_bin = __shfl_sync(kFull, bin, leader);
   const bool same = __all_sync(kFull, !take || bin == lead_bin);
-  if (same && __popc(takers) > 2) {
-    const unsigned int shi = __reduce_add_sync(kFull, take ? (mant >> 12) : 0u);
-    const unsigned int slo = __reduce_add_sync(kFull, take ? (mant & 0xfffu) : 0u);
-    if ((threadIdx.x & 31) == leader) {
-      atomicAdd(&h.cnt[lead_bin], static_cast<unsigned int>(__popc(takers)));
-      atomicAdd(&h.hi[lead_bin], shi);
-      atomicAdd(&h.lo[lead_bin], slo);
-    }
+  if (same && __popc(takers) > 1) {
+    const unsigned int slo = __reduce_add_sync(kFull, take ? (mant & 0xffffu) : 0u);
+    const unsigned int shi = __reduce_add_sync(kFull, take ? (mant >> 16) : 0u);
+    if ((threadIdx.x & 31) == leader) hist_bump(h, lead_bin, slo, shi);
   } else if (take) {
-    atomicAdd(&h.cnt[bin], 1u);
-    atomicAdd(&h.hi[bin], mant >> 12);
-    atomicAdd(&h.lo[bin], mant & 0xfffu);
+    hist_bump(h, bin, mant & 0xffffu, mant >> 16);
   }
 }
 
 __device__ __forceinline__ double shfl_down_f64(double v, int d) { return __shfl_down_sync(kFull, v, d); }
 
 // Scan of `nbins` reduced bins (nbins = 32 * groups, groups <= 64): finds the highest bin at
-// which the mass accumulated from the top -- starting from `carry_mass` / `carry_cnt` already
-// above this level -- reaches `target` (or p * everything when `target_is_fraction`).  All
-// sums run in one fixed order (per-group serial sums, then shuffle suffix scans in warp 0), so
-// every CTA of a cluster gets bit-identical results.  Results land in sh.found_bin,
-// sh.mass_above, sh.mass_ge, sh.cnt_above, sh.total.  Called by all threads.
-__device__ void scan_bins(Shared& sh, const double* mass, const unsigned int* cnt, int nbins, double carry_mass,
-                          unsigned int carry_cnt, double target, bool target_is_fraction, float p) {
+// which the mass accumulated from the top -- starting from `carry_mass` already above this
+// level -- reaches `target` (or p * everything when `target_is_fraction`).  All sums run in
+// one fixed order (per-group serial sums, then shuffle suffix scans in warp 0), so every CTA
+// of a cluster gets bit-identical results.  Results land in sh.found_bin, sh.mass_above,
+// sh.mass_ge, sh.total.  Called by all threads.  An empty bin has mass exactly 0.
+__device__ void scan_bins(Shared& sh, const double* mass, int nbins, double carry_mass, double target,
+                          bool target_is_fraction, float p) {
   const int groups = nbins / kGroup;
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   if (tid < groups) {
     double s = 0.0;
-    unsigned int c = 0;
-    for (int b = kGroup - 1; b >= 0; --b) {
-      s += mass[tid * kGroup + b];
-      c += cnt[tid * kGroup + b];
-    }
+    for (int b = kGroup - 1; b >= 0; --b) s += mass[tid * kGroup + b];
     sh.grp_mass[tid] = s;
-    sh.grp_cnt[tid] = c;
   }
   __syncthreads();
   if (tid < 32) {
@@ -170,37 +162,25 @@ __device__ void scan_bins(Shared& sh, const double* mass, const unsigned int* cn
     const bool two = groups > 32;
     const double g_hi = two ? sh.grp_mass[2 * lane + 1] : sh.grp_mass[lane];
     const double g_lo = two ? sh.grp_mass[2 * lane] : 0.0;
-    const unsigned int c_hi = two ? sh.grp_cnt[2 * lane + 1] : sh.grp_cnt[lane];
-    const unsigned int c_lo = two ? sh.grp_cnt[2 * lane] : 0u;
     // inclusive suffix sums over lanes (lane 31 holds the top groups)
     double s = g_hi + g_lo;
-    unsigned int c = c_hi + c_lo;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
       const double sv = shfl_down_f64(s, d);
-      const unsigned int cv = __shfl_down_sync(kFull, c, d);
-      if (lane + d < 32) {
-        s += sv;
-        c += cv;
-      }
+      if (lane + d < 32) s += sv;
     }
-    // mass / count of everything strictly above this lane's groups, plus the carry
+    // mass of everything strictly above this lane's groups, plus the carry
     double above = shfl_down_f64(s, 1);
-    unsigned int cabove = __shfl_down_sync(kFull, c, 1);
-    if (lane == 31) {
-      above = 0.0;
-      cabove = 0u;
-    }
+    if (lane == 31) above = 0.0;
     above += carry_mass;
-    cabove += carry_cnt;
     const double all = __shfl_sync(kFull, s, 0) + carry_mass;
     if (target_is_fraction) target = static_cast<double>(p) * all;
     // suffix mass including the high group, and including both
     const double with_hi = above + g_hi;
     const double with_lo = with_hi + g_lo;
-    // highest group whose inclusive suffix reaches the target
-    const bool hit_hi = (c_hi != 0u) && (with_hi >= target);
-    const bool hit_lo = two && (c_lo != 0u) && (with_lo >= target);
+    // highest non-empty group whose inclusive suffix reaches the target
+    const bool hit_hi = (g_hi != 0.0) && (with_hi >= target);
+    const bool hit_lo = two && (g_lo != 0.0) && (with_lo >= target);
     const unsigned hits = __ballot_sync(kFull, hit_hi || hit_lo);
     int grp;            // chosen group
     int src;            // lane that owns it
@@ -212,8 +192,8 @@ __device__ void scan_bins(Shared& sh, const double* mass, const unsigned int* cn
     } else {
       // only reachable through rounding between two summation orders: take the lowest
       // non-empty group, i.e. everything at this level is kept
-      const unsigned ne_lo = __ballot_sync(kFull, two ? (c_lo != 0u) : (c_hi != 0u));
-      const unsigned ne_hi = __ballot_sync(kFull, two && (c_hi != 0u));
+      const unsigned ne_lo = __ballot_sync(kFull, two ? (g_lo != 0.0) : (g_hi != 0.0));
+      const unsigned ne_hi = __ballot_sync(kFull, two && (g_hi != 0.0));
       int g0 = -1;
       for (int l = 0; l < 32 && g0 < 0; ++l) {
         if (two) {
@@ -228,46 +208,32 @@ __device__ void scan_bins(Shared& sh, const double* mass, const unsigned int* cn
       src = two ? (g0 >> 1) : g0;
       pick_hi = two ? ((g0 & 1) != 0) : true;
     }
-    // mass / count strictly above the chosen group (incl. carry)
+    // mass strictly above the chosen group (incl. carry)
     const double b_hi = __shfl_sync(kFull, above, src), b_lo = __shfl_sync(kFull, with_hi, src);
-    const unsigned int cb_hi = __shfl_sync(kFull, cabove, src), cb_lo = __shfl_sync(kFull, cabove + c_hi, src);
     const double base = pick_hi ? b_hi : b_lo;
-    const unsigned int cbase = pick_hi ? cb_hi : cb_lo;
     // inside the group: lane b <-> bin grp * 32 + b, inclusive suffix over lanes
     const double m = mass[grp * kGroup + lane];
-    const unsigned int cb = cnt[grp * kGroup + lane];
     double si = m;
-    unsigned int ci = cb;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
       const double sv = shfl_down_f64(si, d);
-      const unsigned int cv = __shfl_down_sync(kFull, ci, d);
-      if (lane + d < 32) {
-        si += sv;
-        ci += cv;
-      }
+      if (lane + d < 32) si += sv;
     }
     const double incl = base + si;  // mass of bins >= this one (incl. carry)
     double ab = shfl_down_f64(si, 1);
-    unsigned int cab = __shfl_down_sync(kFull, ci, 1);
-    if (lane == 31) {
-      ab = 0.0;
-      cab = 0u;
-    }
-    const unsigned ok = __ballot_sync(kFull, cb != 0u && incl >= target);
-    const unsigned nonempty = __ballot_sync(kFull, cb != 0u);
+    if (lane == 31) ab = 0.0;
+    const unsigned ok = __ballot_sync(kFull, m != 0.0 && incl >= target);
+    const unsigned nonempty = __ballot_sync(kFull, m != 0.0);
     int fb;
     if (ok != 0u) fb = 31 - __clz(ok);
     else if (nonempty != 0u) fb = __ffs(nonempty) - 1;  // rounding: keep the whole group
     else fb = 0;
     const double f_above = base + __shfl_sync(kFull, ab, fb);
     const double f_ge = __shfl_sync(kFull, incl, fb);
-    const unsigned int f_cabove = cbase + __shfl_sync(kFull, cab, fb);
     if (lane == 0) {
       sh.found_bin = grp * kGroup + fb;
       sh.mass_above = f_above;
       sh.mass_ge = f_ge;
-      sh.cnt_above = f_cabove;
       sh.total = all;
     }
   }
@@ -312,7 +278,7 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
     sh.n_rows = n;
     sh.n_invalid = 0;
   }
-  for (int i = tid; i < kL1Bins; i += kThreads) sh.h_cnt[i] = sh.h_hi[i] = sh.h_lo[i] = 0u;
+  for (int i = tid; i < kL1Bins; i += kThreads) sh.h_hi[i] = sh.h_lo[i] = 0u;
   __syncthreads();
   const int R = sh.n_rows;
 
@@ -320,9 +286,8 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
   const int slice_cap = static_cast<int>(((((P.L_stride + cs - 1) / cs + 3) & ~3ll) + 31) & ~31ll);
   float* ring = a + slice_cap;
   double* const r_mass = reinterpret_cast<double*>(ring);
-  unsigned int* const r_cnt = reinterpret_cast<unsigned int*>(ring + 4096);
-  unsigned int* const lvl_base = reinterpret_cast<unsigned int*>(ring + 6144);  // 2 levels x 3 x 1024
-  const Hist h1 = {sh.h_cnt, sh.h_hi, sh.h_lo};
+  unsigned int* const lvl_base = reinterpret_cast<unsigned int*>(ring + 4096);  // 2 levels x (lo, hi) x 1024
+  const Hist h1 = {sh.h_lo, sh.h_hi};
 
   // ---- 1+2: aggregate the slice and build the level-1 histogram ------------------------------
   const float* A = P.probs[slot] + static_cast<long long>(b) * P.H * P.gamma * P.L_stride + lo;
@@ -417,9 +382,9 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
   }
   if (bad) atomicAdd(&sh.n_invalid, 1);
   __syncthreads();
-  // the ring is idle from here on: CTA 0 zeroes the cluster's level-2 and level-3 histograms
-  if (rank == 0)
-    for (int i = tid; i < 2 * 3 * kL23Bins; i += kThreads) lvl_base[i] = 0u;
+  // the ring is idle from here on: zero this CTA's level-2 and level-3 histograms
+  for (int i = tid; i < 2 * 2 * kL23Bins; i += kThreads) lvl_base[i] = 0u;
+  __syncthreads();
 
   // ---- 3: threshold search --------------------------------------------------------------------
   cluster.sync();  // every CTA's level-1 histogram and invalid count are complete
@@ -435,14 +400,12 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
     const int per_bins = kL1Bins / cs;
     const int blo = rank * per_bins;
     for (int bin = blo + tid; bin < blo + per_bins; bin += kThreads) {
-      unsigned long long c = 0, mh = 0, ml = 0;
+      unsigned long long mh = 0, ml = 0;
       for (int r = 0; r < cs; ++r) {
-        c += *cluster.map_shared_rank(&sh.h_cnt[bin], r);
         mh += *cluster.map_shared_rank(&sh.h_hi[bin], r);
         ml += *cluster.map_shared_rank(&sh.h_lo[bin], r);
       }
-      r_cnt[bin] = static_cast<unsigned int>(c);
-      r_mass[bin] = static_cast<double>((mh << 12) + ml) * pow2_double(max(bin >> 3, 1) - 150);
+      r_mass[bin] = static_cast<double>((mh << 16) + ml) * pow2_double(max(bin >> 3, 1) - 150);
     }
   }
   cluster.sync();  // every owner's range is reduced
@@ -450,13 +413,10 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
     const int per_bins = kL1Bins / cs;
     for (int bin = tid; bin < kL1Bins; bin += kThreads) {
       const int owner = bin / per_bins;
-      if (owner != rank) {
-        r_cnt[bin] = *cluster.map_shared_rank(&r_cnt[bin], owner);
-        r_mass[bin] = *cluster.map_shared_rank(&r_mass[bin], owner);
-      }
+      if (owner != rank) r_mass[bin] = *cluster.map_shared_rank(&r_mass[bin], owner);
     }
     __syncthreads();
-    scan_bins(sh, r_mass, r_cnt, kL1Bins, 0.0, 0u, 0.0, true, P.p);
+    scan_bins(sh, r_mass, kL1Bins, 0.0, 0.0, true, P.p);
     total = sh.total;
     target = static_cast<double>(P.p) * total;
     m_ge = total;
@@ -467,14 +427,12 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
   unsigned int prefix = searching ? static_cast<unsigned int>(sh.found_bin) : 0u;
   const int e1 = max(static_cast<int>(prefix >> 3), 1) - 150;
   double carry_m = searching ? sh.mass_above : 0.0;
-  unsigned int carry_c = searching ? sh.cnt_above : 0u;
   for (int level = 0; level < 2; ++level) {
     const int shift = (level == 0) ? 10 : 0;
-    unsigned int* lb = lvl_base + level * 3 * kL23Bins;
+    unsigned int* lb = lvl_base + level * 2 * kL23Bins;
     if (searching) {
-      // the few elements inside the threshold bin go straight into CTA 0's histogram
-      const Hist hr = {cluster.map_shared_rank(lb, 0), cluster.map_shared_rank(lb + kL23Bins, 0),
-                       cluster.map_shared_rank(lb + 2 * kL23Bins, 0)};
+      // only the elements inside the threshold bin take part
+      const Hist hr = {lb, lb + kL23Bins};
       for (int base = 0; base < n_loc; base += kThreads) {
         const int i = base + tid;
         unsigned int key = 0u;
@@ -486,21 +444,22 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
         hist_add(hr, take, static_cast<int>((key >> shift) & 1023u), mantissa_of(key));
       }
     }
-    cluster.sync();  // all remote atomics of this level have landed
+    cluster.sync();  // every CTA's histogram of this level is complete
     if (searching) {
-      const unsigned int* src = cluster.map_shared_rank(lb, 0);
       const double scale = pow2_double(e1);
-      __syncthreads();  // the previous scan no longer reads the arrays overwritten below
       for (int bin = tid; bin < kL23Bins; bin += kThreads) {
-        const unsigned long long mh = src[kL23Bins + bin], ml = src[2 * kL23Bins + bin];
-        r_cnt[bin] = src[bin];
-        r_mass[bin] = static_cast<double>((mh << 12) + ml) * scale;
+        unsigned long long ml = 0, mh = 0;
+        for (int r = 0; r < cs; ++r) {
+          const unsigned int* src = cluster.map_shared_rank(lb, r);
+          ml += src[bin];
+          mh += src[kL23Bins + bin];
+        }
+        r_mass[bin] = static_cast<double>((mh << 16) + ml) * scale;
       }
       __syncthreads();
-      scan_bins(sh, r_mass, r_cnt, kL23Bins, carry_m, carry_c, target, false, P.p);
+      scan_bins(sh, r_mass, kL23Bins, carry_m, target, false, P.p);
       prefix = (prefix << 10) | static_cast<unsigned int>(sh.found_bin);
       carry_m = sh.mass_above;
-      carry_c = sh.cnt_above;
     }
   }
   if (searching) {
