@@ -318,6 +318,54 @@ def topp_sweep(dev, reps=5):
     return out
 
 
+def verify_micro(dev, reps=10):
+    """sparse_verify alone on synthetic shapes: dense long context and sparse lists of several
+    lengths (shuffled block table, page 16).  Returns {case: {us, gbs}}; bytes = K/V rows read."""
+    import torch
+    import paper_2510_27641_b200 as sa
+    import workloads as wl
+    out = {}
+    cases = [("dense_b4_ctx131072_q6x32_kv8", 4, 131072, 6, 32, 8, None),
+             ("dense_b4_ctx131072_q5x64_kv8", 4, 131072, 5, 64, 8, None),
+             ("sparse1245_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, 1245),
+             ("sparse12450_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, 12450),
+             ("sparse1000_b4_ctx131072_q5x64_kv8", 4, 131072, 5, 64, 8, 1000)]
+    for name, B, L, T, Hq, Hkv, count in cases:
+        page = 16
+        pps = (L + page - 1) // page
+        kv = wl.kv_pool(9, 0, B * pps, page, Hkv, 128, device=dev)
+        bt = torch.from_numpy(wl.block_table(9, B, pps)).to(dev)
+        q = torch.randn((B, T, Hq, 128), device=dev).to(torch.bfloat16)
+        kv_len = torch.full((B,), L, dtype=torch.int32, device=dev)
+        o = torch.empty((B, T, Hq, 128), dtype=torch.float32, device=dev)
+        l = torch.empty((B, T, Hq), dtype=torch.float32, device=dev)
+        if count is None:
+            kw, c = dict(dense=True), L
+        else:
+            idx = torch.stack([torch.sort(torch.randperm(L, device=dev)[:count])[0] for _ in range(B)])
+            kw = dict(idx=idx.to(torch.int32).view(B, 1, count).contiguous(),
+                      counts=torch.full((B, 1), count, dtype=torch.int32, device=dev))
+            c = count
+        a = sa.make_verify_args(q, kv, kv_len, block_table=bt, out=o, lse=l, idx=kw.get("idx"),
+                                counts=kw.get("counts"), dense=kw.get("dense", False))
+        ws = sa.verify_workspace(a)
+        f = lambda: sa.sparse_verify(q, kv, kv_len, block_table=bt, out=o, lse=l, workspace=ws, **kw)
+        for _ in range(3):
+            f()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            f()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / reps
+        byts = B * c * Hkv * 512
+        out[name] = {"us": round(us, 1), "kv_mb": round(byts / 1e6, 1), "gbs": round(byts / us / 1e3)}
+        del kv
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -325,6 +373,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--topp-sweep", action="store_true", help="also run the 256-row selection micro-benchmark")
+    ap.add_argument("--verify-micro", action="store_true", help="only run the sparse_verify micro-benchmark")
     ap.add_argument("--layers", type=int, default=0, help="override the number of target layers (debug)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -349,6 +398,10 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
         barrier = lambda: (dist.barrier(), torch.cuda.synchronize())
+
+    if args.verify_micro:
+        print(json.dumps({"verify_micro": verify_micro(dev, reps=min(10, max(2, args.steps)))}))
+        return
 
     # every rank owns a batch of its own (batch sharding): same shapes, rank-specific seed
     cfg_r = cfg.scaled(seed=cfg.seed + 1000 * rank) if world > 1 else cfg
