@@ -60,6 +60,23 @@ def _measured_peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
+def rank_config(cfg, rank: int, world: int):
+    """The workload of one rank: with N > 1 every rank owns a batch of its own (sharding by
+    sequence, no collective on the data path) -- same shapes, rank-specific seed."""
+    return cfg.scaled(seed=cfg.seed + 1000 * rank) if world > 1 else cfg
+
+
+def reduce_max(values, world: int, device="cuda"):
+    """Element-wise MAX over ranks of a list of timings (identity for one rank)."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
 class ClockSampler:
     """Samples SM clock and clock-event reasons through NVML while the timed region runs."""
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
@@ -404,7 +421,7 @@ def main():
         return
 
     # every rank owns a batch of its own (batch sharding): same shapes, rank-specific seed
-    cfg_r = cfg.scaled(seed=cfg.seed + 1000 * rank) if world > 1 else cfg
+    cfg_r = rank_config(cfg, rank, world)
     si, pools, step, dp_host, q_host = build_step(cfg_r, dev)
     step.run()
     torch.cuda.synchronize()
@@ -459,10 +476,7 @@ def main():
     h2d = sum(t.numel() * 4 for t in dp_host if t is not None) + sum(t.numel() * 2 for t in q_host)
     d2h = sum(t.numel() * 4 for t in out_host) + sum(t.numel() * 4 for t in lse_host)
 
-    if world > 1:
-        t = torch.tensor([us_step, us_e2e, us_verify_all, us_select], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        us_step, us_e2e, us_verify_all, us_select = t.tolist()
+    us_step, us_e2e, us_verify_all, us_select = reduce_max([us_step, us_e2e, us_verify_all, us_select], world, dev)
 
     # ---- roofline of the dominant kernel (sparse verify) -------------------------------------
     per_layer = [verify_bytes(cfg_r, si, counts[int(u)]) for u in si.layer_map]
