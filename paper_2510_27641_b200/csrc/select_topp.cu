@@ -29,6 +29,10 @@
 //      histogram were measured first and cost ~11 us per level on tie-free rows.)
 //   4. after three levels the threshold is known bit-exactly; each CTA compacts its kept
 //      positions in ascending order behind the counts of the lower-ranked CTAs.
+// When a list has a single contributing row (one draft head, gamma = 1: the selection
+// micro-benchmark) of 32k positions or more there is nothing to aggregate and the row is not
+// copied to shared memory at all but re-read from global memory (L2) by the later passes,
+// which shrinks a CTA to ~57 KB of shared memory so that four of them share an SM.
 #include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <float.h>
@@ -73,6 +77,7 @@ struct SelectParams {
   int* counts;
   int* status;
   double* diag;
+  int single_row;  // every list has exactly one contributing row: read it in place
 };
 
 // A histogram of exact mantissa sums, kept as two 32-bit words: `lo` sums the low 16 mantissa
@@ -240,7 +245,8 @@ __device__ void scan_bins(Shared& sh, const double* mass, int nbins, double carr
   __syncthreads();
 }
 
-__global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_constant__ SelectParams P) {
+template <bool kInPlace>
+__global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel(const __grid_constant__ SelectParams P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
   float* a = reinterpret_cast<float*>(smem_raw + ((sizeof(Shared) + 127) / 128) * 128);
@@ -283,7 +289,7 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
   const int R = sh.n_rows;
 
   // dynamic shared memory behind the fixed part
-  const int slice_cap = static_cast<int>(((((P.L_stride + cs - 1) / cs + 3) & ~3ll) + 31) & ~31ll);
+  const int slice_cap = kInPlace ? 0 : static_cast<int>(((((P.L_stride + cs - 1) / cs + 3) & ~3ll) + 31) & ~31ll);
   float* ring = a + slice_cap;
   double* const r_mass = reinterpret_cast<double*>(ring);
   unsigned int* const lvl_base = reinterpret_cast<unsigned int*>(ring + 4096);  // 2 levels x (lo, hi) x 1024
@@ -291,10 +297,39 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
 
   // ---- 1+2: aggregate the slice and build the level-1 histogram ------------------------------
   const float* A = P.probs[slot] + static_cast<long long>(b) * P.H * P.gamma * P.L_stride + lo;
+  constexpr bool in_place = kInPlace;
+  // bit pattern of aggregated position i of the slice (-0.0 reads as +0.0)
+  auto key_at = [&](int i) -> unsigned int {
+    return in_place ? __float_as_uint(__ldg(A + i) + 0.f) : __float_as_uint(a[i]);
+  };
   const int n4 = (n_loc + 3) >> 2;
   const int n_pos4 = n4 * 4;                       // slice length rounded up to whole float4s
   const int n_chunks = (n_pos4 + kChunk - 1) / kChunk;
   bool bad = false;
+  if (in_place) {
+    // single contributing row: one pass over the slice for validity and the level-1 histogram
+    for (int base = 0; base < n4; base += kThreads) {
+      const int i4 = base + tid;
+      const bool act = i4 < n4;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (act) {
+        v = __ldg(reinterpret_cast<const float4*>(A) + i4);
+        const int left = n_loc - 4 * i4;
+        if (left < 4) v.w = 0.f;
+        if (left < 3) v.z = 0.f;
+        if (left < 2) v.y = 0.f;
+        bad |= !(v.x >= 0.f && v.x <= FLT_MAX) | !(v.y >= 0.f && v.y <= FLT_MAX) |
+               !(v.z >= 0.f && v.z <= FLT_MAX) | !(v.w >= 0.f && v.w <= FLT_MAX);
+      }
+      const float vals[4] = {v.x + 0.f, v.y + 0.f, v.z + 0.f, v.w + 0.f};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const unsigned int key = __float_as_uint(vals[e]);
+        const bool take = act && (4 * i4 + e < n_loc) && key != 0u && !(key >> 31);
+        hist_add(h1, take, static_cast<int>(key >> 20), mantissa_of(key));
+      }
+    }
+  } else
   // Pieces are numbered q = chunk * R + row, i.e. in the order the adds must happen.  Every
   // thread copies exactly the two float4 columns of a piece that it will add itself, with
   // 16-byte cp.async into its own ring slots, kDepth pieces ahead: completion is tracked per
@@ -438,7 +473,7 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
         unsigned int key = 0u;
         bool take = false;
         if (i < n_loc) {
-          key = __float_as_uint(a[i]);
+          key = key_at(i);
           take = (key >> (shift + 10)) == prefix;
         }
         hist_add(hr, take, static_cast<int>((key >> shift) & 1023u), mantissa_of(key));
@@ -477,7 +512,7 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
   if (!invalid) {
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
       const int i = i0 + lane;
-      const bool keep = i < w_hi && __float_as_uint(a[i]) >= theta_key;
+      const bool keep = i < w_hi && key_at(i) >= theta_key;
       wc += __popc(__ballot_sync(kFull, keep));
     }
   }
@@ -504,7 +539,7 @@ __global__ void __launch_bounds__(kThreads, 2) select_topp_kernel(const __grid_c
     long long pos = offset + sh.warp_cnt[warp];
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
       const int i = i0 + lane;
-      const bool keep = i < w_hi && __float_as_uint(a[i]) >= theta_key;
+      const bool keep = i < w_hi && key_at(i) >= theta_key;
       const unsigned m = __ballot_sync(kFull, keep);
       const long long my = pos + __popc(m & ((1u << lane) - 1u));
       if (keep && my < P.idx_stride) out[my] = lo + i;
@@ -604,15 +639,20 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   P.status = A.row_status;
   P.diag = A.diag;
 
+  // single-row lists are read in place once the rows are long enough for the extra CTAs per
+  // SM to pay for re-reading them from L2 (measured cross-over between 8k and 64k positions)
+  P.single_row = (static_cast<long long>(A.n_draft_heads) * A.gamma == 1 && A.L_stride >= 32768) ? 1 : 0;
   const int cs = specattn::pick_cluster(A.L_stride, n_lists);
-  const long long slice = (((A.L_stride + cs - 1) / cs) + 3) / 4 * 4;
+  const long long slice = P.single_row ? 0 : (((A.L_stride + cs - 1) / cs) + 3) / 4 * 4;
   if (slice > specattn::kSliceCap) return SPECATTN_ERR_UNSUPPORTED;
   // shared memory: fixed part, the aggregated slice, then the per-thread staging ring
   // (kDepth pieces of 8 KB; it later hosts the scan arrays).  Small slices leave room for two
   // CTAs per SM.
   const size_t fixed = ((sizeof(specattn::Shared) + 127) / 128) * 128;
   const size_t slice_bytes = static_cast<size_t>((slice + 31) / 32 * 32) * sizeof(float);
-  const size_t smem = fixed + slice_bytes + static_cast<size_t>(specattn::kRingFloats) * sizeof(float);
+  // (a single-row list keeps nothing but the 32 KB of scan arrays behind the fixed part)
+  const size_t smem = fixed + slice_bytes +
+                      (P.single_row ? static_cast<size_t>(32 * 1024) : static_cast<size_t>(specattn::kRingFloats) * sizeof(float));
   if (smem > 224 * 1024) return SPECATTN_ERR_UNSUPPORTED;
 
   // Opt in to large dynamic shared memory once per device, so that later calls issue nothing
@@ -623,8 +663,11 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPECATTN_ERR_CUDA;
     if (!((done_mask.load(std::memory_order_acquire) >> dev) & 1ull)) {
-      err = cudaFuncSetAttribute(specattn::select_topp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      err = cudaFuncSetAttribute(specattn::select_topp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  224 * 1024);
+      if (err == cudaSuccess)
+        err = cudaFuncSetAttribute(specattn::select_topp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   224 * 1024);
       if (err != cudaSuccess) {
         cudaGetLastError();
         return SPECATTN_ERR_CUDA;
@@ -646,7 +689,8 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  err = cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel, P);
+  err = P.single_row ? cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<true>, P)
+                     : cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<false>, P);
   if (err != cudaSuccess) {
     cudaGetLastError();
     return SPECATTN_ERR_CUDA;

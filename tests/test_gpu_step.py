@@ -140,15 +140,17 @@ def test_host_buffer_step_matches_device_resident_step():
         assert torch.equal(out_host[j], ref_out[j].cpu()) and torch.equal(lse_host[j], ref_lse[j].cpu())
 
 
-@pytest.mark.parametrize("which", ["cfg1", "cfg3"])
+@pytest.mark.parametrize("which", ["cfg1", "cfg3", "cfg4"])
 def test_full_size_sampled_outputs(which):
-    """Full batch / context of configs 1 and 3 (two target layers for config 1): every list is
+    """Full batch / context of configs 1, 3 and 4 (two target layers for 1 and 4): every list is
     compared; attention is checked on sampled (layer, sequence, kv head) units whose K/V rows
     are regenerated on the CPU from the hashed pool definition."""
     if which == "cfg1":
         cfg = wl.config1().scaled(n_target_layers=2)
-    else:
+    elif which == "cfg3":
         cfg = wl.config3()
+    else:
+        cfg = wl.config4(n_target_layers=2, p=0.9)   # 70B-shaped: 64 q / 8 kv heads, ctx 131072
     si, pools, step = _build(cfg)
     step.run()
     torch.cuda.synchronize()
