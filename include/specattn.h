@@ -140,6 +140,12 @@ int specattn_select_topp(const specattn_select_args* args, void* cuda_stream);
  * counts [batch, n_groups] (entries beyond idx_stride are ignored).  dense != 0 attends every
  * position below kv_len[b] and reads neither idx nor counts (both may be NULL).
  *
+ * tail_len > 0 adds the tokens being verified themselves (Alg. 1: the gamma+1 tokens go through
+ * the verifier in one pass): their K/V rows must already be in the cache at positions
+ * kv_len[b] + j, j < tail_len, and query t attends, after its list, the rows with
+ * j <= t + (tail_len - n_q) -- with tail_len == n_q token t sees tokens 0..t.  kv_len stays the
+ * context length without them.
+ *
  * Requirements: head_dim == 128; n_q * (n_q_heads / n_kv_heads) <= 64; batch * n_kv_heads
  * <= 2048; q, kv_pages 16-byte aligned and all four strides multiples of 8; out 16-byte
  * aligned.  status (int32 [batch], optional) receives SPECATTN_ROW_BAD_INDEX when a listed
@@ -191,6 +197,7 @@ typedef struct specattn_verify_args {
   void* workspace;
   size_t workspace_bytes;
   uint32_t flags;        /* SPECATTN_VERIFY_* bits, 0 for none */
+  int32_t tail_len;      /* in-flight tokens attended causally after the list, 0 <= tail_len <= 64 */
 } specattn_verify_args;
 
 /* Bytes of workspace specattn_sparse_verify needs for these shapes on the current device

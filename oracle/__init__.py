@@ -132,12 +132,13 @@ def attend_rows(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float | None
 
 
 def sparse_verify(q, kv_pages, kv_strides, block_table, kv_len, idx, counts, *, n_kv_heads,
-                  page_size, n_groups=1, dense=False, scale=0.0, pages_per_seq=None):
+                  page_size, n_groups=1, dense=False, scale=0.0, pages_per_seq=None, tail_len=0):
     """O3 over one target layer.
 
     q [B,T,H_q,d] uint16; kv_pages any-shaped uint16 buffer with element strides
     kv_strides = (page, kv, slot, head); block_table [B, max_pages] int32 or None
     (contiguous; pages_per_seq then required); idx [B,G,idx_stride], counts [B,G].
+    tail_len > 0: the in-flight tokens at positions kv_len[b] + j are attended causally.
     """
     q = _chk(q, np.uint16)
     B, T, Hq, d = q.shape
@@ -161,5 +162,5 @@ def sparse_verify(q, kv_pages, kv_strides, block_table, kv_len, idx, counts, *, 
                                         _p(kv_pages), C.c_int64(sp), C.c_int64(sk), C.c_int64(ss),
                                         C.c_int64(sh), _p(block_table), C.c_int64(bts), _p(kv_len),
                                         _p(idx_a), C.c_int64(istride), _p(cnt_a), int(bool(dense)),
-                                        C.c_double(scale), _p(out), _p(lse))
+                                        C.c_double(scale), int(tail_len), _p(out), _p(lse))
     return out, lse

@@ -280,6 +280,9 @@ void specattn_oracle_attend_rows(const uint16_t* q, int64_t q_stride, const uint
 //   idx/counts the lists of ONE draft layer: [B, G, idx_stride], [B, G];
 //              dense != 0: every position < kv_len[b] is attended, lists unread
 //   query head h uses kv head h / (H_q/H_kv) and list g = (G == 1 ? 0 : kv head)
+//   tail_len   the in-flight tokens: positions kv_len[b] + j, j < tail_len, already in the
+//              cache; query t additionally attends those with j <= t + (tail_len - T), i.e.
+//              causally among the tokens being verified (tail_len = T: token t sees itself)
 //   out [B, T, H_q, d] and lse [B, T, H_q] binary64.
 // All T queries and all heads of a group share one list.
 // [Alg. 1 "Verification with Sparse Attention": one mask per layer for the
@@ -290,8 +293,8 @@ void specattn_oracle_sparse_verify(int B, int T, int Hq, int Hkv, int d, int pag
                                    int64_t stride_kv, int64_t stride_slot, int64_t stride_head,
                                    const int32_t* block_table, int64_t bt_stride,
                                    const int32_t* kv_len, const int32_t* idx, int64_t idx_stride,
-                                   const int32_t* counts, int dense, double scale, double* out,
-                                   double* lse) {
+                                   const int32_t* counts, int dense, double scale, int tail_len,
+                                   double* out, double* lse) {
   const int grp = Hq / Hkv;
   if (scale == 0.0) scale = 1.0 / std::sqrt(static_cast<double>(d));
   const int64_t n_units = static_cast<int64_t>(B) * Hkv;
@@ -302,9 +305,10 @@ void specattn_oracle_sparse_verify(int B, int T, int Hq, int Hkv, int d, int pag
     const int g = (G == 1) ? 0 : hk;
     const int64_t li = static_cast<int64_t>(b) * G + g;
     const int64_t c = dense ? kv_len[b] : std::min<int64_t>(counts[li], idx_stride);
-    std::vector<uint16_t> Kr(std::max<int64_t>(c, 1) * d), Vr(std::max<int64_t>(c, 1) * d);
-    for (int64_t k = 0; k < c; ++k) {
-      const int64_t pos = dense ? k : idx[li * idx_stride + k];
+    const int64_t ct = c + tail_len;  // listed rows first, then the in-flight tokens
+    std::vector<uint16_t> Kr(std::max<int64_t>(ct, 1) * d), Vr(std::max<int64_t>(ct, 1) * d);
+    for (int64_t k = 0; k < ct; ++k) {
+      const int64_t pos = (k >= c) ? (kv_len[b] + (k - c)) : (dense ? k : idx[li * idx_stride + k]);
       const int64_t logical_page = pos / page_size;
       const int64_t page = block_table ? block_table[b * bt_stride + logical_page]
                                        : b * bt_stride + logical_page;
@@ -314,10 +318,13 @@ void specattn_oracle_sparse_verify(int B, int T, int Hq, int Hkv, int d, int pag
       std::memcpy(&Vr[k * d], base + stride_kv, sizeof(uint16_t) * d);
     }
     for (int t = 0; t < T; ++t) {
+      // query t sees the whole list and the first (t + tail_len - T + 1) in-flight tokens
+      int64_t n_tail = static_cast<int64_t>(t) + tail_len - T + 1;
+      n_tail = std::max<int64_t>(0, std::min<int64_t>(n_tail, tail_len));
       for (int hh = 0; hh < grp; ++hh) {
         const int h = hk * grp + hh;
         const int64_t row = (static_cast<int64_t>(b) * T + t) * Hq + h;
-        specattn_oracle_attend_rows(q + row * d, d, Kr.data(), d, Vr.data(), d, 1, c, d, scale,
+        specattn_oracle_attend_rows(q + row * d, d, Kr.data(), d, Vr.data(), d, 1, c + n_tail, d, scale,
                                     out + row * d, lse + row);
       }
     }

@@ -51,7 +51,8 @@ class VerifyArgs(C.Structure):
                 ("block_table_stride", C.c_int64), ("kv_len", C.c_void_p), ("idx", C.c_void_p),
                 ("idx_stride", C.c_int64), ("counts", C.c_void_p), ("sm_scale", C.c_float),
                 ("out", C.c_void_p), ("lse", C.c_void_p), ("status", C.c_void_p),
-                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("flags", C.c_uint32)]
+                ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("flags", C.c_uint32),
+                ("tail_len", C.c_int32)]
 
 
 class StepHostArgs(C.Structure):
@@ -181,7 +182,7 @@ def make_verify_args(q: torch.Tensor, kv_pages: torch.Tensor, kv_len: torch.Tens
                      idx: torch.Tensor | None, counts: torch.Tensor | None, n_groups: int = 1,
                      dense: bool = False, sm_scale: float = 0.0, out: torch.Tensor,
                      lse: torch.Tensor, status: torch.Tensor | None = None,
-                     workspace: torch.Tensor | None = None, flags: int = 0) -> VerifyArgs:
+                     workspace: torch.Tensor | None = None, flags: int = 0, tail_len: int = 0) -> VerifyArgs:
     """Fills a VerifyArgs from tensors.  kv_pages is [n_pages, 2, page_size, H_kv, d] bf16 (any
     strides with a unit innermost stride); idx [B, G, idx_stride] / counts [B, G] are the lists
     of ONE draft layer."""
@@ -209,6 +210,7 @@ def make_verify_args(q: torch.Tensor, kv_pages: torch.Tensor, kv_len: torch.Tens
         a.idx, a.idx_stride, a.counts = idx.data_ptr(), idx.shape[2], counts.data_ptr()
     a.sm_scale = float(sm_scale)
     a.flags = int(flags)
+    a.tail_len = int(tail_len)
     a.out, a.lse = out.data_ptr(), lse.data_ptr()
     a.status = None if status is None else status.data_ptr()
     if workspace is not None:
@@ -238,7 +240,7 @@ def sparse_verify(q: torch.Tensor, kv_pages: torch.Tensor, kv_len: torch.Tensor,
                   n_groups: int = 1, dense: bool = False, sm_scale: float = 0.0,
                   out: torch.Tensor | None = None, lse: torch.Tensor | None = None,
                   status: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
-                  flags: int = 0, stream=None):
+                  flags: int = 0, tail_len: int = 0, stream=None):
     """specattn_sparse_verify for one target layer.  Returns (out f32 [B,T,H_q,d], lse f32
     [B,T,H_q], status int32 [B])."""
     B, T, Hq, d = q.shape
@@ -250,7 +252,8 @@ def sparse_verify(q: torch.Tensor, kv_pages: torch.Tensor, kv_len: torch.Tensor,
         status = torch.zeros((B,), dtype=torch.int32, device=q.device)
     args = make_verify_args(q, kv_pages, kv_len, block_table=block_table, pages_per_seq=pages_per_seq,
                             idx=idx, counts=counts, n_groups=n_groups, dense=dense, sm_scale=sm_scale,
-                            out=out, lse=lse, status=status, workspace=workspace, flags=flags)
+                            out=out, lse=lse, status=status, workspace=workspace, flags=flags,
+                            tail_len=tail_len)
     if workspace is None:
         workspace = verify_workspace(args, q.device, stream)
         args.workspace, args.workspace_bytes = workspace.data_ptr(), workspace.numel()

@@ -78,6 +78,8 @@ struct VerifyParams {
   unsigned int* counters;
   float* partials;
   int lists_stable;  // SPECATTN_VERIFY_LISTS_STABLE
+  int tail;          // in-flight tokens appended to every unit, attended causally
+  int tail_off;      // tail - T: query t may see tail tokens j <= t + tail_off
 };
 
 // WPM = consumer warps per 16-row slab: 4 -> (stage parity, 32-key half), 2 -> (stage parity).
@@ -112,7 +114,7 @@ __device__ __forceinline__ int unit_count(const VerifyParams& P, int u) {
     if (c > P.idx_stride) c = P.idx_stride;
   }
   if (c < 0) c = 0;
-  return static_cast<int>(c);
+  return static_cast<int>(c) + P.tail;  // the in-flight tokens follow the list
 }
 
 // First atom of CTA i when n atoms are dealt to np CTAs.
@@ -142,8 +144,11 @@ struct WarpState {
 
 // One 32-key block: S = Q K^T (4 n-tiles), online softmax, O += P V with P = P_hi + P_lo.
 // `valid` = number of existing keys in the block (>= 1; rows beyond it hold finite padding).
+// `tail_begin` = index inside the block of the first in-flight token (>= 32: none); rows g and
+// g+8 of the slab may see in-flight tokens j <= lim0 / lim1 only (causal among themselves).
 __device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&qf)[8][4], uint32_t k_addr,
-                                               uint32_t v_addr, int valid, float scale_log2, int tq) {
+                                               uint32_t v_addr, int valid, float scale_log2, int tq,
+                                               int tail_begin, int lim0, int lim1) {
   float sc[4][4];
 #pragma unroll
   for (int n = 0; n < 4; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
@@ -165,6 +170,15 @@ __device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&q
       for (int i = 0; i < 4; ++i) {
         const int key = n * 8 + tq * 2 + (i & 1);
         if (key >= valid) sc[n][i] = -INFINITY;
+      }
+  }
+  if (tail_begin < 32) {  // the block holds in-flight tokens: causal mask per query row
+#pragma unroll
+    for (int n = 0; n < 4; ++n)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int j = n * 8 + tq * 2 + (i & 1) - tail_begin;
+        if (j >= 0 && j > ((i & 2) ? lim1 : lim0)) sc[n][i] = -INFINITY;  // j < 0: a listed row
       }
   }
   float mx0 = fmaxf(fmaxf(fmaxf(sc[0][0], sc[0][1]), fmaxf(sc[1][0], sc[1][1])),
@@ -423,6 +437,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       const int tok_lo = (a - us) * kAtom;
       const int tok_hi = min(sh.unit_cnt[u], (seg_hi - us) * kAtom);
       const int kvlen_b = P.kv_len[b];
+      const int c_list = sh.unit_cnt[u] - P.tail;
       const int* list = P.dense ? nullptr
                                 : P.idx + (static_cast<long long>(b) * P.G + ((P.G == 1) ? 0 : kvh)) * P.idx_stride;
       const __nv_bfloat16* kv_head = P.kv + static_cast<long long>(kvh) * P.s_head;
@@ -455,8 +470,9 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
 #pragma unroll
         for (int jj = 0; jj < 2; ++jj) {
           const int jt = min(lane + jj * 32, ntok - 1);
-          int pos = P.dense ? (t0 + jt) : __ldg(list + t0 + jt);
-          if (pos < 0 || pos >= kvlen_b) { bad = true; pos = 0; }
+          const int k = t0 + jt;  // token index inside the unit: the list first, then the tail
+          int pos = (k >= c_list) ? (kvlen_b + (k - c_list)) : (P.dense ? k : __ldg(list + k));
+          if (pos < 0 || pos >= kvlen_b + P.tail) { bad = true; pos = 0; }
           const int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
           const int slot = pos - lp * P.page_size;
           long long page = P.bt ? static_cast<long long>(__ldg(P.bt + b * P.bt_stride + lp))
@@ -555,6 +571,10 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     const int b = u / P.Hkv, kvh = u % P.Hkv;
     const int tok_lo = (a - us) * kAtom;
     const int tok_hi = min(sh.unit_cnt[u], (seg_hi - us) * kAtom);
+    const int c_list = sh.unit_cnt[u] - P.tail;
+    // in-flight tokens the two rows of this lane may see: row r belongs to query r / grp
+    const int lim0 = (mt * 16 + g) / P.grp + P.tail_off;
+    const int lim1 = (mt * 16 + g + 8) / P.grp + P.tail_off;
 
     // query fragments of this unit
     uint32_t qf[8][4];
@@ -579,14 +599,19 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       const int ntok = min(kStageTok, tok_hi - t0);
       const uint32_t k_base = smem_u32(sh.kv[s][0]) + k_off;
       const uint32_t v_base = smem_u32(sh.kv[s][1]) + v_off;
+      // index inside the tile of the first in-flight token (negative once the tile starts
+      // inside the tail; out of reach when the call has no tail)
+      const int tb = P.tail ? (c_list - t0) : (1 << 20);
       if (WPM == 4) {
         const int key0 = (wr & 1) * 32;
         if (key0 < ntok)
-          attend_block32(st, qf, k_base + key0 * kPitch, v_base + key0 * kPitch, ntok - key0, P.scale_log2, tq);
+          attend_block32(st, qf, k_base + key0 * kPitch, v_base + key0 * kPitch, ntok - key0, P.scale_log2, tq,
+                         tb - key0, lim0, lim1);
       } else {
-        attend_block32(st, qf, k_base, v_base, ntok, P.scale_log2, tq);
+        attend_block32(st, qf, k_base, v_base, ntok, P.scale_log2, tq, tb, lim0, lim1);
         if (32 < ntok)
-          attend_block32(st, qf, k_base + 32 * kPitch, v_base + 32 * kPitch, ntok - 32, P.scale_log2, tq);
+          attend_block32(st, qf, k_base + 32 * kPitch, v_base + 32 * kPitch, ntok - 32, P.scale_log2, tq,
+                         tb - 32, lim0, lim1);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.empty[s]);
@@ -814,6 +839,7 @@ int validate(const specattn_verify_args* args) {
   if (A.n_q_heads % A.n_kv_heads != 0) return SPECATTN_ERR_RANGE;
   if (A.n_groups != 1 && A.n_groups != A.n_kv_heads) return SPECATTN_ERR_RANGE;
   if (!(A.sm_scale >= 0.f)) return SPECATTN_ERR_RANGE;  // negative or NaN
+  if (A.tail_len < 0 || A.tail_len > 64) return SPECATTN_ERR_RANGE;
   if (A.head_dim != kD) return SPECATTN_ERR_UNSUPPORTED;
   if (A.n_q * (A.n_q_heads / A.n_kv_heads) > SPECATTN_MAX_QUERY_ROWS) return SPECATTN_ERR_UNSUPPORTED;
   if (static_cast<long long>(A.batch) * A.n_kv_heads > kMaxUnits) return SPECATTN_ERR_UNSUPPORTED;
@@ -897,6 +923,8 @@ extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cu
   P.status = A.status;
   P.counters = static_cast<unsigned int*>(A.workspace);
   P.lists_stable = (A.flags & SPECATTN_VERIFY_LISTS_STABLE) ? 1 : 0;
+  P.tail = A.tail_len;
+  P.tail_off = A.tail_len - A.n_q;
   P.partials = reinterpret_cast<float*>(static_cast<unsigned char*>(A.workspace) + specattn::kCounterBytes);
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -12,10 +12,10 @@ from workloads import bf16
 pytestmark = pytest.mark.gpu
 
 
-def _make_case(seed, B, T, Hq, Hkv, page, lens, G=1, counts=None, shuffle=True, d=128):
+def _make_case(seed, B, T, Hq, Hkv, page, lens, G=1, counts=None, shuffle=True, d=128, tail=0):
     rng = np.random.default_rng(seed)
     lens = np.asarray(lens, np.int32)
-    pages_per_seq = max(1, (int(lens.max()) + page - 1) // page)
+    pages_per_seq = max(1, (int(lens.max()) + tail + page - 1) // page)   # room for the in-flight tokens
     n_pages = B * pages_per_seq
     kv = wl.kv_pool(seed, 0, n_pages, page, Hkv, d)                      # torch bf16 on CPU
     bt = wl.block_table(seed, B, pages_per_seq, n_pages, shuffle=shuffle)
@@ -31,7 +31,7 @@ def _make_case(seed, B, T, Hq, Hkv, page, lens, G=1, counts=None, shuffle=True, 
             idx[b, g, :c] = sel
             cnt[b, g] = c
     return dict(q=q, kv=kv, bt=bt, lens=lens, idx=idx, cnt=cnt, page=page, Hkv=Hkv, G=G,
-                pages_per_seq=pages_per_seq)
+                pages_per_seq=pages_per_seq, tail=tail)
 
 
 def _run(case, dense=False, use_bt=True, sm_scale=0.0, workspace=None):
@@ -41,7 +41,7 @@ def _run(case, dense=False, use_bt=True, sm_scale=0.0, workspace=None):
         bf16_to_dev(case["q"]), kv_d, to_dev(case["lens"]),
         block_table=to_dev(case["bt"]) if use_bt else None, pages_per_seq=case["pages_per_seq"],
         idx=None if dense else to_dev(case["idx"]), counts=None if dense else to_dev(case["cnt"]),
-        n_groups=case["G"], dense=dense, sm_scale=sm_scale, workspace=workspace)
+        n_groups=case["G"], dense=dense, sm_scale=sm_scale, workspace=workspace, tail_len=case.get("tail", 0))
     torch.cuda.synchronize()
     return out, lse, status
 
@@ -52,7 +52,7 @@ def _oracle(case, dense=False, use_bt=True, scale=0.0):
     return oracle.sparse_verify(case["q"], kv_bits, wl.kv_strides(page, Hkv, 128),
                                 case["bt"] if use_bt else None, case["lens"], case["idx"], case["cnt"],
                                 n_kv_heads=Hkv, page_size=page, n_groups=case["G"], dense=dense,
-                                scale=scale, pages_per_seq=case["pages_per_seq"])
+                                scale=scale, pages_per_seq=case["pages_per_seq"], tail_len=case.get("tail", 0))
 
 
 @pytest.mark.parametrize("T,Hq,Hkv", [(5, 32, 8), (6, 32, 8), (5, 64, 8), (2, 8, 2), (8, 16, 2), (1, 4, 4)])
@@ -122,6 +122,24 @@ def test_per_kv_head_lists_page_sizes_and_scale():
         case = _make_case(24 + page, 2, 5, 16, 4, page, [900, 333], G=4)
         out, lse, _ = _run(case, sm_scale=0.05)
         check_attention(out, lse, *_oracle(case, scale=0.05))
+
+
+@pytest.mark.parametrize("T,tail", [(5, 5), (6, 6), (5, 2), (4, 7), (6, 1)])
+def test_causal_tail_of_in_flight_tokens(T, tail):
+    # list lengths chosen so that the tail starts at every offset of a 64-token tile, straddles
+    # tiles, follows an empty list, and follows lists cut between CTAs
+    lens = [300, 300, 300, 300, 300, 300, 3000, 5000]
+    counts = [[0], [1], [31], [60], [63], [64], [2999], [4097]]
+    case = _make_case(40 + T, 8, T, 32, 8, 16, lens, counts=counts, tail=tail)
+    out, lse, status = _run(case)
+    check_attention(out, lse, *_oracle(case))
+    assert int(status.abs().sum()) == 0
+    # dense context + tail = ordinary causal decode attention of the verified tokens
+    case_d = _make_case(50 + T, 2, T, 16, 2, 16, [130, 64], counts=[[130], [64]], tail=tail)
+    o_d, l_d, _ = _run(case_d, dense=True)
+    check_attention(o_d, l_d, *_oracle(case_d, dense=True))
+    o_f, l_f, _ = _run(case_d)
+    assert torch.equal(o_d, o_f) and torch.equal(l_d, l_f)
 
 
 def test_precision_when_few_tokens_dominate():

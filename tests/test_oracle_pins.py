@@ -406,3 +406,38 @@ def test_joint_error_bound_of_appendix_a():
         kept = dg["m_ge"] / dg["total"]
         assert err <= (1 - kept) * vmax * (1 + 1e-6) + 1e-9
         assert (1 - kept) <= (1 - p) + 1e-6
+
+
+def test_sparse_verify_causal_tail_matches_library_attention_per_query():
+    """The in-flight tokens (Alg. 1, "Verification with Sparse Attention": the gamma+1 tokens are
+    verified in one pass) are attended causally on top of the list: query t sees tail tokens
+    j <= t + tail_len - T.  Checked per query against a dense library softmax over that set."""
+    rng = np.random.default_rng(15)
+    B, T, Hq, Hkv, d, page = 2, 4, 4, 2, 128, 16
+    lens = [40, 23]
+    for tail in (4, 2, 6):
+        q, kv, bt, strides = _paged_case(rng, B, T, Hq, Hkv, d, page, [x + tail for x in lens])
+        kv_len = np.array(lens, np.int32)
+        idx = np.full((B, 1, 16), -1, np.int32)
+        counts = np.zeros((B, 1), np.int32)
+        for b in range(B):
+            sel = np.sort(rng.choice(lens[b], size=5 + 3 * b, replace=False))
+            idx[b, 0, :len(sel)] = sel
+            counts[b, 0] = len(sel)
+        out, lse = oracle.sparse_verify(q, kv, strides, bt, kv_len, idx, counts, n_kv_heads=Hkv,
+                                        page_size=page, tail_len=tail)
+        for b in range(B):
+            for t in range(T):
+                n_tail = max(0, min(tail, t + tail - T + 1))
+                pos = list(idx[b, 0, :counts[b, 0]]) + [lens[b] + j for j in range(n_tail)]
+                for h in range(Hq):
+                    hk = h // (Hq // Hkv)
+                    K = np.stack([kv[bt[b, i // page], 0, i % page, hk] for i in pos])
+                    V = np.stack([kv[bt[b, i // page], 1, i % page, hk] for i in pos])
+                    ro, rl = _torch_dense(q[b, t:t + 1, h], K, V)
+                    assert np.allclose(out[b, t, h], ro[0], rtol=1e-12, atol=1e-13)
+                    assert np.allclose(lse[b, t, h], rl[0], rtol=1e-12)
+    # tail_len = 0 is the plain call
+    o0, l0 = oracle.sparse_verify(q, kv, strides, bt, kv_len, idx, counts, n_kv_heads=Hkv, page_size=page)
+    o1, l1 = oracle.sparse_verify(q, kv, strides, bt, kv_len, idx, counts, n_kv_heads=Hkv, page_size=page, tail_len=0)
+    assert np.array_equal(o0, o1) and np.array_equal(l0, l1)
