@@ -167,8 +167,16 @@ int specattn_select_topp(const specattn_select_args* args, void* cuda_stream);
  * serialization, i.e. it may begin while the preceding kernel is still running.  Without this
  * flag it waits for that kernel to finish before reading anything, and lets its own successor
  * start only after that wait; with it, it starts fetching K/V rows at once and waits only
- * before reading q and before writing out, lse, status or the workspace. */
+ * before reading q and before writing out, lse, status or the workspace.
+ *
+ * SPECATTN_VERIFY_ENGINE_MMA_SYNC / SPECATTN_VERIFY_ENGINE_TCGEN05: force one of the two
+ * implementations of the same operation (warp-level mma.sync with register accumulators, or
+ * tcgen05.mma with accumulators in tensor memory).  With neither bit the library picks by
+ * problem shape; results agree within the tolerance of the operation either way.  Setting
+ * both bits is SPECATTN_ERR_RANGE. */
 #define SPECATTN_VERIFY_LISTS_STABLE 1u
+#define SPECATTN_VERIFY_ENGINE_MMA_SYNC 2u
+#define SPECATTN_VERIFY_ENGINE_TCGEN05 4u
 
 typedef struct specattn_verify_args {
   uint32_t struct_size;

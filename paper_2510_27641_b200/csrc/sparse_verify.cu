@@ -825,6 +825,8 @@ cudaError_t launch(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
   return err;
 }
 
+#include "sparse_verify_tc.cuh"
+
 int m_tiles(const specattn_verify_args& A) {
   const int grp = A.n_q_heads / A.n_kv_heads;
   return (A.n_q * grp + 15) / 16;
@@ -840,14 +842,29 @@ int validate(const specattn_verify_args* args) {
   if (A.n_groups != 1 && A.n_groups != A.n_kv_heads) return SPECATTN_ERR_RANGE;
   if (!(A.sm_scale >= 0.f)) return SPECATTN_ERR_RANGE;  // negative or NaN
   if (A.tail_len < 0 || A.tail_len > 64) return SPECATTN_ERR_RANGE;
+  if ((A.flags & SPECATTN_VERIFY_ENGINE_MMA_SYNC) && (A.flags & SPECATTN_VERIFY_ENGINE_TCGEN05))
+    return SPECATTN_ERR_RANGE;
   if (A.head_dim != kD) return SPECATTN_ERR_UNSUPPORTED;
   if (A.n_q * (A.n_q_heads / A.n_kv_heads) > SPECATTN_MAX_QUERY_ROWS) return SPECATTN_ERR_UNSUPPORTED;
   if (static_cast<long long>(A.batch) * A.n_kv_heads > kMaxUnits) return SPECATTN_ERR_UNSUPPORTED;
   return SPECATTN_OK;
 }
 
+// 32-row blocks of the query block (tcgen05 engine)
+int row_blocks(const specattn_verify_args& A) { return (m_tiles(A) + 1) / 2; }
+
+// Which engine runs a call: the caller's choice, else by shape.
+bool use_tcgen05(const specattn_verify_args& A) {
+  if (A.flags & SPECATTN_VERIFY_ENGINE_TCGEN05) return true;
+  if (A.flags & SPECATTN_VERIFY_ENGINE_MMA_SYNC) return false;
+  return false;
+}
+
+// Sized for either engine, so that the choice never depends on the workspace at hand.
 size_t workspace_bytes_for(const specattn_verify_args& A, int n_ctas) {
-  return kCounterBytes + static_cast<size_t>(2) * n_ctas * m_tiles(A) * kRec * sizeof(float);
+  const size_t a = static_cast<size_t>(m_tiles(A)) * kRec;
+  const size_t b = static_cast<size_t>(row_blocks(A)) * kTcRec;
+  return kCounterBytes + static_cast<size_t>(2) * n_ctas * (a > b ? a : b) * sizeof(float);
 }
 
 }  // namespace
@@ -929,11 +946,16 @@ extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cu
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t err;
-  switch (specattn::m_tiles(A)) {
-    case 1: err = specattn::launch<1, 4>(P, n_ctas, stream); break;
-    case 2: err = specattn::launch<2, 4>(P, n_ctas, stream); break;
-    case 3: err = specattn::launch<3, 2>(P, n_ctas, stream); break;
-    default: err = specattn::launch<4, 2>(P, n_ctas, stream); break;
+  if (specattn::use_tcgen05(A)) {
+    if (specattn::row_blocks(A) == 1) err = specattn::launch_tc<1, 4>(P, n_ctas, stream);
+    else err = specattn::launch_tc<2, 3>(P, n_ctas, stream);
+  } else {
+    switch (specattn::m_tiles(A)) {
+      case 1: err = specattn::launch<1, 4>(P, n_ctas, stream); break;
+      case 2: err = specattn::launch<2, 4>(P, n_ctas, stream); break;
+      case 3: err = specattn::launch<3, 2>(P, n_ctas, stream); break;
+      default: err = specattn::launch<4, 2>(P, n_ctas, stream); break;
+    }
   }
   if (err != cudaSuccess) return SPECATTN_ERR_CUDA;
   specattn::g_launch_count.fetch_add(1, std::memory_order_relaxed);

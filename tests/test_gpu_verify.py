@@ -11,6 +11,17 @@ from workloads import bf16
 
 pytestmark = pytest.mark.gpu
 
+_ENGINE = {"flags": 0}
+
+
+@pytest.fixture(params=["mma_sync", "tcgen05"], autouse=True)
+def engine(request):
+    """Every case runs once per implementation of the operation (forced through the flags)."""
+    import paper_2510_27641_b200 as sa
+    _ENGINE["flags"] = sa.VERIFY_ENGINE_MMA_SYNC if request.param == "mma_sync" else sa.VERIFY_ENGINE_TCGEN05
+    yield request.param
+    _ENGINE["flags"] = 0
+
 
 def _make_case(seed, B, T, Hq, Hkv, page, lens, G=1, counts=None, shuffle=True, d=128, tail=0):
     rng = np.random.default_rng(seed)
@@ -41,7 +52,8 @@ def _run(case, dense=False, use_bt=True, sm_scale=0.0, workspace=None):
         bf16_to_dev(case["q"]), kv_d, to_dev(case["lens"]),
         block_table=to_dev(case["bt"]) if use_bt else None, pages_per_seq=case["pages_per_seq"],
         idx=None if dense else to_dev(case["idx"]), counts=None if dense else to_dev(case["cnt"]),
-        n_groups=case["G"], dense=dense, sm_scale=sm_scale, workspace=workspace, tail_len=case.get("tail", 0))
+        n_groups=case["G"], dense=dense, sm_scale=sm_scale, workspace=workspace, tail_len=case.get("tail", 0),
+        flags=_ENGINE["flags"])
     torch.cuda.synchronize()
     return out, lse, status
 
@@ -100,7 +112,8 @@ def test_ragged_batch_with_shared_workspace_reuse():
     ws = sa.verify_workspace(args)
     for _ in range(3):
         o.fill_(float("nan"))
-        sa.sparse_verify(q_d, kv_d, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d, out=o, lse=l, workspace=ws)
+        sa.sparse_verify(q_d, kv_d, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d, out=o, lse=l, workspace=ws,
+                         flags=_ENGINE["flags"])
         torch.cuda.synchronize()
         assert torch.equal(o, out) and torch.equal(l, lse)
 
