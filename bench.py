@@ -134,7 +134,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------
-def build_step(cfg, dev):
+def build_step(cfg, dev, verify_flags=0):
     import torch
     import workloads as wl
     from paper_2510_27641_b200.step import VerifyStep
@@ -147,7 +147,7 @@ def build_step(cfg, dev):
                       n_q_heads=cfg.n_q_heads, p=cfg.p, kv_pools=pools,
                       kv_len=torch.from_numpy(si.kv_len).to(dev),
                       block_table=None if si.block_table is None else torch.from_numpy(si.block_table).to(dev),
-                      pages_per_seq=si.pages_per_seq)
+                      pages_per_seq=si.pages_per_seq, verify_flags=verify_flags)
     dp_host = [None if x is None else torch.from_numpy(x).pin_memory() for x in si.draft_probs]
     q_host = [bf16.bits_to_torch(q).pin_memory() for q in si.q]
     step.load_inputs(dp_host, q_host)
@@ -335,7 +335,7 @@ def topp_sweep(dev, reps=5):
     return out
 
 
-def verify_micro(dev, reps=10):
+def verify_micro(dev, reps=10, flags=0):
     """sparse_verify alone on synthetic shapes: dense long context and sparse lists of several
     lengths (shuffled block table, page 16).  Returns {case: {us, gbs}}; bytes = K/V rows read."""
     import torch
@@ -366,7 +366,7 @@ def verify_micro(dev, reps=10):
         a = sa.make_verify_args(q, kv, kv_len, block_table=bt, out=o, lse=l, idx=kw.get("idx"),
                                 counts=kw.get("counts"), dense=kw.get("dense", False))
         ws = sa.verify_workspace(a)
-        f = lambda: sa.sparse_verify(q, kv, kv_len, block_table=bt, out=o, lse=l, workspace=ws, **kw)
+        f = lambda: sa.sparse_verify(q, kv, kv_len, block_table=bt, out=o, lse=l, workspace=ws, flags=flags, **kw)
         for _ in range(3):
             f()
         torch.cuda.synchronize()
@@ -391,6 +391,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--topp-sweep", action="store_true", help="also run the 256-row selection micro-benchmark")
     ap.add_argument("--verify-micro", action="store_true", help="only run the sparse_verify micro-benchmark")
+    ap.add_argument("--verify-engine", default="auto", choices=["auto", "mma_sync", "tcgen05"],
+                    help="force one implementation of sparse_verify (default: the library picks by shape)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of target layers (debug)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -416,13 +418,15 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
         barrier = lambda: (dist.barrier(), torch.cuda.synchronize())
 
+    vflags = {"auto": 0, "mma_sync": sa.VERIFY_ENGINE_MMA_SYNC, "tcgen05": sa.VERIFY_ENGINE_TCGEN05}[args.verify_engine]
     if args.verify_micro:
-        print(json.dumps({"verify_micro": verify_micro(dev, reps=min(10, max(2, args.steps)))}))
+        print(json.dumps({"verify_micro": verify_micro(dev, reps=min(10, max(2, args.steps)), flags=vflags),
+                          "engine": args.verify_engine}))
         return
 
     # every rank owns a batch of its own (batch sharding): same shapes, rank-specific seed
     cfg_r = rank_config(cfg, rank, world)
-    si, pools, step, dp_host, q_host = build_step(cfg_r, dev)
+    si, pools, step, dp_host, q_host = build_step(cfg_r, dev, verify_flags=vflags)
     step.run()
     torch.cuda.synchronize()
     counts = step.counts.cpu().numpy()

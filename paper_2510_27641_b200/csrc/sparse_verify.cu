@@ -947,8 +947,12 @@ extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cu
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t err;
   if (specattn::use_tcgen05(A)) {
-    if (specattn::row_blocks(A) == 1) err = specattn::launch_tc<1, 4>(P, n_ctas, stream);
-    else err = specattn::launch_tc<2, 3>(P, n_ctas, stream);
+    switch (specattn::m_tiles(A)) {
+      case 1: err = specattn::launch_tc<1>(P, n_ctas, stream); break;
+      case 2: err = specattn::launch_tc<2>(P, n_ctas, stream); break;
+      case 3: err = specattn::launch_tc<3>(P, n_ctas, stream); break;
+      default: err = specattn::launch_tc<4>(P, n_ctas, stream); break;
+    }
   } else {
     switch (specattn::m_tiles(A)) {
       case 1: err = specattn::launch<1, 4>(P, n_ctas, stream); break;

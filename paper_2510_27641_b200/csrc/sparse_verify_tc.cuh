@@ -3,33 +3,41 @@
 // cross-CTA merge protocol with the mma.sync kernel there.
 //
 // Same operation (Eq. 1 over the listed rows, Sec. 3.5 / Alg. 1 "Verification with Sparse
-// Attention"), different engine for the two contractions of a 64-key tile:
-//   S[128 x 64]  = Q[128 x 128] K^T      one tcgen05.mma chain (8 x K=16), A and B from shared
-//                                         memory in the 128-byte-swizzled K-major layout
-//   O[128 x 128] += P[128 x 64] V        A = P as packed bf16 in TENSOR MEMORY (two terms,
-//                                         P = P_hi + P_lo), B = V from shared memory, MN-major
-// The query block ((gamma+1) x group <= 64 rows) sits in rows 0.. of the M = 128 operand, the
-// other rows are zero: the tensor pipe has throughput to spare, and in return every query row
-// lives in ONE thread of the softmax warps (TMEM lane = row), so max / sum / exp need no
-// shuffles and no shared memory at all.
+// Attention").  The query block of a unit has at most 64 rows, far fewer than the 128 rows a
+// tcgen05.mma produces, so both products are computed TRANSPOSED: the 128 KEYS of a tile (or
+// the 128 output dimensions) are the M side of the instruction, the N = 16..64 query rows its
+// N side:
+//   S^T[128 keys x N]  = K[128 x 128] Q^T          A = K tile, B = Q tile, both K-major in smem
+//   O^T[128 dims x N] += V^T[128 x 128 keys] P^T   A = V tile (MN-major), B = P^T (MN-major)
+// No tensor work is spent on padding rows, and -- because a TMEM lane is a key (or an output
+// dimension) -- the four softmax warps, one per lane quadrant and hence one per SM
+// sub-partition, each own 32 keys of every tile.  P = exp2(S - m) is written as two bf16
+// terms (P = P_hi + P_lo) into the shared-memory bytes of the K tile it was computed from,
+// which are dead once S^T is complete; the stage is released when the P V product has read it.
 //
-// Warp roles (9 warps): 4 producers gather K/V rows with 16-byte cp.async straight into the
-// swizzled tile layout (then fence.proxy.async, so the tensor core's async-proxy reads see them);
-// 1 warp issues all MMAs and tcgen05.commit arrivals; 2 x 2 softmax warps work on alternate
-// tiles, each parity with its own S / P / O columns in TMEM (512 columns in total), and are
-// combined at the end of a unit exactly like the key-split warps of the mma.sync kernel.
-// The running maximum is only raised when a tile exceeds it by 2^8 (P stays < 256 in bf16);
-// raising it rescales the O rows in TMEM (tcgen05.ld / st), which is rare.
+// The reference maximum m of a row is raised lazily: a tile whose scaled scores stay below
+// m + 8 (in the log2 domain) is exponentiated against the old m (P < 2^8, exact enough in two
+// bf16 terms and fp32 accumulation); only a tile that exceeds it takes the slow path (row
+// maxima over the 128 keys by warp butterflies and a small shared-memory exchange, then a
+// rescale of the O^T columns in tensor memory).  Whether a tile takes it is agreed per tile
+// through one named barrier of the four softmax warps.
+//
+// Warps: 0-3 softmax (TMEM lane quadrant = warp index), 4 = MMA issue (one thread),
+// 5-8 = producers: two warps per tile, 64 keys each, 16-byte cp.async straight into the
+// 128-byte-swizzled operand layout, then fence.proxy.async before the arrival.
 #pragma once
 
-constexpr int kTcTile = 64;                      // keys per tile
-constexpr int kTcTileBytes = kTcTile * 256;      // one K or V tile (16 KB)
-constexpr int kTcRecCols = 130;                  // 128 outputs, m, l of one row
-constexpr int kTcRec = kTcRecCols * 32;          // floats of a 32-row record, [column][row]
+constexpr int kTcTile = 128;                     // keys per tile
+constexpr int kTcTileBytes = kTcTile * 256;      // one K or V tile (32 KB)
+constexpr int kTcStages = 3;
+constexpr int kTcRec = 130 * 32;                 // floats of a record per 32 query rows
 constexpr float kTcRaise = 8.f;                  // raise the reference maximum beyond 2^8
+constexpr int kTcThreads = 9 * 32;
+constexpr int kTcMmaWarp = 4;
+constexpr int kTcSoftmaxThreads = 128;
 
-// byte offset of 16-byte chunk `c` (0..15) of row `r` in a tile of `rows` rows: two 128-byte
-// halves per row, chunks XOR-swizzled with the row index (UMMA 128-byte swizzle, K-major)
+// byte offset of 16-byte chunk `c` (0..15) of row `r` in a tile of `rows` rows of 256 bytes: two
+// 128-byte halves per row, chunks XOR-swizzled with the row index (UMMA 128-byte swizzle)
 __device__ __forceinline__ uint32_t tc_sw(int r, int c, int rows) {
   return static_cast<uint32_t>((c >> 3) * rows * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
@@ -55,13 +63,6 @@ __device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a, uint64_t 
       "l"(a), "l"(b), "r"(idesc), "r"(acc), "r"(0u)
       : "memory");
 }
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(b), "r"(idesc), "r"(acc), "r"(0u)
-      : "memory");
-}
 // arrival on an mbarrier once every tcgen05 operation issued so far by this thread has completed
 __device__ __forceinline__ void tc_commit(unsigned long long* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -72,58 +73,89 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// 32 lanes x 32 columns of 32 bits: thread t of the warp gets / provides TMEM lane (base + t)
-#define SPECATTN_TMEM_LD32(r, addr)                                                                             \
-  asm volatile(                                                                                                  \
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                                  \
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27," \
-      "%28,%29,%30,%31}, [%32];"                                                                                 \
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),          \
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),    \
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),  \
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])   \
-      : "r"(addr))
-#define SPECATTN_TMEM_ST32(addr, r)                                                                             \
-  asm volatile(                                                                                                  \
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "                                                            \
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28," \
-      "%29,%30,%31,%32};" ::"r"(addr),                                                                           \
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),         \
-      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), \
-      "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]),            \
-      "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])                                     \
-      : "memory")
+// 32 lanes x 16 columns of 32 bits: thread t of the warp gets / provides TMEM lane (base + t)
+__device__ __forceinline__ void tc_ld16(uint32_t (&r)[16], uint32_t addr) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(addr));
+}
+__device__ __forceinline__ void tc_st16(uint32_t addr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(
+          addr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+// named barrier that also ORs a predicate over its participants: everyone gets the same answer,
+// so a group that must leave together can decide to leave on it
+__device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %3, 0;\n\t"
+      "barrier.red.or.pred q, %1, %2, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+      : "=r"(r)
+      : "r"(id), "r"(nthreads), "r"(static_cast<uint32_t>(pred))
+      : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 
-// NB = 32-row blocks of the query block (1 or 2), NS = ring stages
-template <int NB, int NS>
+// Butterfly reduce-scatter over the 32 lanes of a warp: v[i] is this lane's value for row i;
+// afterwards lane r holds the reduction of row r (returned).  31 shuffles.
+template <bool kMax>
+__device__ __forceinline__ float tc_reduce_scatter(float (&v)[32], int lane) {
+#pragma unroll
+  for (int step = 16; step >= 1; step >>= 1) {
+    const bool upper = (lane & step) != 0;
+#pragma unroll
+    for (int i = 0; i < step; ++i) {
+      const float send = upper ? v[i] : v[i + step];
+      const float keep = upper ? v[i + step] : v[i];
+      const float recv = __shfl_xor_sync(0xffffffffu, send, step);
+      v[i] = kMax ? fmaxf(keep, recv) : (keep + recv);
+    }
+  }
+  return v[0];
+}
+
 struct TcShared {
-  alignas(1024) unsigned char kv[NS][2 * kTcTileBytes];  // per stage: K tile then V tile
-  alignas(1024) unsigned char q[128 * 256];
-  float scratch[NB][kTcRec];   // parity-1 group -> parity-0 group at the end of a unit
-  float peer_rec[NB][kTcRec];  // cluster-pair merge: the odd CTA's records land here
-  alignas(8) unsigned long long full[NS];
-  unsigned long long empty[NS];
+  alignas(1024) unsigned char kv[kTcStages][2 * kTcTileBytes];  // per stage: K tile (later P^T), V tile
+  alignas(1024) unsigned char q[64 * 256];
+  float m_ref[64];     // reference maximum of every query row (scaled log2 domain)
+  float alpha[64];     // rescale factors of the tile that raised it
+  float lsum[64];      // row sums at the end of a unit
+  float wred[4][64];   // per-warp row maxima / row sums
+  int row_off[64];     // query row r -> t * Hq + (r % grp): its output row inside (b, kv head)
+  int row_lim[64];     // last in-flight token row r may see
+  alignas(8) unsigned long long full[kTcStages];
+  unsigned long long empty[kTcStages];
   unsigned long long q_full, q_empty;
-  unsigned long long s_full[2], s_free[2], p_full[2], pv_done[2], o_free[2];
-  unsigned long long peer_full;
+  unsigned long long s_full[2], s_free[2], p_full, pv_done, o_free;
   uint32_t tmem_base;
+  int raise_tile[2];   // tile index + 1 of the last tile (per S buffer) that must raise m_ref
+  int last_arriver;
   int unit_start[kMaxUnits + 1];
-  int unit_cnt[kMaxUnits];
   int part_start[kAlignedMaxUnits + 1];
   int cand_parts[kCandidates];
   int cand_max[kCandidates];
   volatile int abort_flag;
 };
 
-constexpr int kTcThreads = 9 * 32;
-constexpr int kTcMmaWarp = 2;
-
-template <int NB, int NS>
+// NT = N / 16, N = query rows rounded up to a multiple of 16
+template <int NT>
 __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const __grid_constant__ VerifyParams P) {
-  using Sh = TcShared<NB, NS>;
+  constexpr int N = NT * 16;
+  constexpr int NS = kTcStages;
+  constexpr int NTH = kTcThreads;
+  constexpr int NBLK = (N + 31) / 32;
   extern __shared__ __align__(1024) unsigned char smem_raw_tc[];
-  Sh& sh = *reinterpret_cast<Sh*>((reinterpret_cast<uintptr_t>(smem_raw_tc) + 1023) & ~static_cast<uintptr_t>(1023));
-  constexpr int NT = kTcThreads;
+  TcShared& sh =
+      *reinterpret_cast<TcShared*>((reinterpret_cast<uintptr_t>(smem_raw_tc) + 1023) & ~static_cast<uintptr_t>(1023));
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int warp = tid >> 5;
@@ -135,36 +167,34 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   // ---- set-up ---------------------------------------------------------------------------------
   {
     uint4* zq = reinterpret_cast<uint4*>(sh.q);  // rows beyond the query block stay zero
-    for (int i = tid; i < static_cast<int>(sizeof(sh.q) / 16); i += NT) zq[i] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = tid; i < static_cast<int>(sizeof(sh.q) / 16); i += NTH) zq[i] = make_uint4(0u, 0u, 0u, 0u);
   }
   if (tid == 0) {
     for (int s = 0; s < NS; ++s) {
-      mbar_init(&sh.full[s], 1);
+      mbar_init(&sh.full[s], 2);   // two producer warps per tile
       mbar_init(&sh.empty[s], 1);
     }
     mbar_init(&sh.q_full, 1);
     mbar_init(&sh.q_empty, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sh.s_full[i], 1);
-      mbar_init(&sh.s_free[i], NB);
-      mbar_init(&sh.p_full[i], NB);
-      mbar_init(&sh.pv_done[i], 1);
-      mbar_init(&sh.o_free[i], NB);
+      mbar_init(&sh.s_free[i], 4);
     }
-    mbar_init(&sh.peer_full, NB);
+    mbar_init(&sh.p_full, 4);
+    mbar_init(&sh.pv_done, 1);
+    mbar_init(&sh.o_free, 4);
     mbar_fence_init();
     sh.abort_flag = 0;
+    sh.raise_tile[0] = sh.raise_tile[1] = 0;
     sh.unit_start[0] = 0;
   }
-  for (int u = tid; u < U; u += NT) {
-    const int c = unit_count(P, u);
-    sh.unit_cnt[u] = c;
-    sh.unit_start[u + 1] = (c + kAtom - 1) / kAtom;
+  if (tid < 64) {
+    sh.row_off[tid] = (tid / P.grp) * P.Hq + tid % P.grp;
+    sh.row_lim[tid] = tid / P.grp + P.tail_off;
   }
+  for (int u = tid; u < U; u += NTH) sh.unit_start[u + 1] = (unit_count(P, u) + kAtom - 1) / kAtom;
   fence_proxy_async();
   __syncthreads();
-  const bool paired = cluster_num_ctas() == 2;
-  if (paired) cluster_sync_all();
   if (warp == 0) {  // inclusive scan of the atom counts
     int carry = 0;
     for (int base = 0; base < U; base += 32) {
@@ -181,19 +211,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   }
   __syncthreads();
 
-  // ---- work partition (same two schemes as the mma.sync kernel) ---------------------------------
-  const long long N = sh.unit_start[U];
+  // ---- work partition (the two schemes of the mma.sync kernel) -----------------------------------
+  const long long NA = sh.unit_start[U];
   const int G = static_cast<int>(gridDim.x);
   if (tid < kCandidates) { sh.cand_parts[tid] = 0; sh.cand_max[tid] = 0; }
   __syncthreads();
-  const bool try_aligned = (U <= kAlignedMaxUnits) && (N > 0);
+  const bool try_aligned = (U <= kAlignedMaxUnits) && (NA > 0);
   if (try_aligned && tid < U) {
     const int atoms = sh.unit_start[tid + 1] - sh.unit_start[tid];
     if (atoms > 0) {
 #pragma unroll
       for (int c = 0; c < kCandidates; ++c) {
         const long long num = static_cast<long long>(atoms) * G * 16;
-        const long long den = N * (16 + c);
+        const long long den = NA * (16 + c);
         int k = static_cast<int>((2 * num + den) / (2 * den));
         if (k < 1) k = 1;
         if (k > atoms) k = atoms;
@@ -207,7 +237,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   if (try_aligned) {
     for (int c = 0; c < kCandidates; ++c)
       if (sh.cand_parts[c] <= G) { cand = c; break; }
-    if (cand >= 0 && static_cast<long long>(sh.cand_max[cand]) * G > N + 24ll * G) cand = -1;
+    if (cand >= 0 && static_cast<long long>(sh.cand_max[cand]) * G > NA + 24ll * G) cand = -1;
   }
   const bool aligned = cand >= 0;
   if (aligned && warp == 0) {
@@ -219,7 +249,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         const int atoms = sh.unit_start[u + 1] - sh.unit_start[u];
         if (atoms > 0) {
           const long long num = static_cast<long long>(atoms) * G * 16;
-          const long long den = N * (16 + cand);
+          const long long den = NA * (16 + cand);
           k = static_cast<int>((2 * num + den) / (2 * den));
           if (k < 1) k = 1;
           if (k > atoms) k = atoms;
@@ -237,21 +267,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
     }
   }
   __syncthreads();
-  const long long NP = aligned ? sh.part_start[U] : ((N < G) ? N : static_cast<long long>(G));
+  const long long NP = aligned ? sh.part_start[U] : ((NA < G) ? NA : static_cast<long long>(G));
 
-  const bool is_softmax = (warp == 0 || warp == 1 || warp == 4 || warp == 5);
+  const bool is_softmax = warp < 4;
   const bool is_mma = (warp == kTcMmaWarp);
-  if (is_softmax || is_mma) {
-    // the only warps that write global memory or consume q: the previous kernel is complete
-    if (P.lists_stable) pdl_wait();
-  }
   if (is_softmax) {
+    // the only warps that write global memory: the previous kernel is complete from here on
+    if (P.lists_stable) pdl_wait();
     // units with an empty list: out = 0, lse = -inf
     for (int u = blockIdx.x; u < U; u += gridDim.x) {
-      if (sh.unit_cnt[u] != 0) continue;
+      if (unit_count(P, u) != 0) continue;
       const int b = u / P.Hkv, kvh = u % P.Hkv;
-      const int st = ((warp & 1) + (warp >> 2) * 2) * 32 + lane;  // 0..127 over the four warps
-      for (int e = st; e < P.M * kD; e += 128) {
+      for (int e = tid; e < P.M * kD; e += kTcSoftmaxThreads) {
         const int r = e / kD, t = r / P.grp, h = kvh * P.grp + r % P.grp;
         P.out[((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD + e % kD] = 0.f;
         if (e % kD == 0) P.lse[(static_cast<long long>(b) * P.T + t) * P.Hq + h] = -INFINITY;
@@ -272,8 +299,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
     a0 = sh.unit_start[lo] + static_cast<int>(j * atoms / k);
     a1 = sh.unit_start[lo] + static_cast<int>((j + 1) * atoms / k);
   } else {
-    a0 = cta_first_atom(blockIdx.x, N, NP);
-    a1 = cta_first_atom(blockIdx.x + 1, N, NP);
+    a0 = cta_first_atom(blockIdx.x, NA, NP);
+    a1 = cta_first_atom(blockIdx.x + 1, NA, NP);
   }
   int u_first;
   {
@@ -286,10 +313,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
     while (sh.unit_start[u_first + 1] <= a0) ++u_first;
   }
 
-  // ---- tensor memory: 512 columns = S[2] (64 each), P_hi[2], P_lo[2] (32 each), O[2] (128 each) --
+  // ---- tensor memory: S^T double-buffered (N columns each), O^T (N columns) ---------------------
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)),
-                 "r"(512u)
+                 "r"(256u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -297,12 +324,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sh.tmem_base;
-  auto col_s = [&](int par) { return tmem + static_cast<uint32_t>(par * 64); };
-  auto col_phi = [&](int par) { return tmem + 128u + static_cast<uint32_t>(par * 32); };
-  auto col_plo = [&](int par) { return tmem + 192u + static_cast<uint32_t>(par * 32); };
-  auto col_o = [&](int par) { return tmem + 256u + static_cast<uint32_t>(par * 128); };
+  const uint32_t col_o = tmem + 2u * N;
 
-  // every role walks the same sequence of segments (unit, token range) and 64-key tiles
   auto next_unit = [&](int& a, int& u, int seg_hi, int ue) {
     a = seg_hi;
     if (a == ue) {
@@ -313,178 +336,171 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
 
   if (!is_softmax && !is_mma) {
     // =============================== producer warps ===============================================
-    const int pw = (warp == 3) ? 0 : (warp - 5);  // warps 3, 6, 7, 8 -> 0..3
-    if (pw < NS) {
-      int it = 0, seg = 0;
-      int a = a0, u = u_first;
-      bool dead = false;
-      while (a < a1 && !dead) {
-        const int us = sh.unit_start[u], ue = sh.unit_start[u + 1];
-        const int seg_hi = min(a1, ue);
-        const int b = u / P.Hkv, kvh = u % P.Hkv;
-        const int tok_lo = (a - us) * kAtom;
-        const int tok_hi = min(sh.unit_cnt[u], (seg_hi - us) * kAtom);
-        const int kvlen_b = P.kv_len[b];
-        const int c_list = sh.unit_cnt[u] - P.tail;
-        const int* list = P.dense ? nullptr
-                                  : P.idx + (static_cast<long long>(b) * P.G + ((P.G == 1) ? 0 : kvh)) * P.idx_stride;
-        const __nv_bfloat16* kv_head = P.kv + static_cast<long long>(kvh) * P.s_head;
-        // the query block of this unit, straight into the swizzled operand layout (warp 0 of
-        // the producers only; first segment: after the warp's first tile)
-        auto load_q = [&]() -> bool {
-          if (seg == 0 && P.lists_stable) pdl_wait();
-          if (!mbar_wait(&sh.q_empty, (seg & 1u) ^ 1u, &sh.abort_flag)) return false;
-          const uint32_t qb = smem_u32(sh.q);
-          for (int i = lane; i < P.M * 16; i += 32) {
-            const int r = i >> 4, c = i & 15;
-            const int t = r / P.grp, h = kvh * P.grp + r % P.grp;
-            cp_async16(qb + tc_sw(r, c, 128), P.q + ((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD + c * 8);
+    // tile i is filled by warps 2 (i & 1) and 2 (i & 1) + 1: keys 0..63 and 64..127 of the tile
+    const int pw = warp - 5;
+    const int tpar = pw >> 1, half = pw & 1;
+    int it = 0, seg = 0;
+    int a = a0, u = u_first;
+    bool dead = false;
+    while (a < a1 && !dead) {
+      const int us = sh.unit_start[u], ue = sh.unit_start[u + 1];
+      const int seg_hi = min(a1, ue);
+      const int b = u / P.Hkv, kvh = u % P.Hkv;
+      const int ucnt = unit_count(P, u);
+      const int tok_lo = (a - us) * kAtom;
+      const int tok_hi = min(ucnt, (seg_hi - us) * kAtom);
+      const int kvlen_b = P.kv_len[b];
+      const int c_list = ucnt - P.tail;
+      const int* list = P.dense ? nullptr
+                                : P.idx + (static_cast<long long>(b) * P.G + ((P.G == 1) ? 0 : kvh)) * P.idx_stride;
+      const __nv_bfloat16* kv_head = P.kv + static_cast<long long>(kvh) * P.s_head;
+      // The query block of this unit, straight into the swizzled operand layout; always by
+      // producer warp 0, walking the segments in order (for the first segment after the warp's
+      // first half tile, so that K/V prefetch is in flight while it waits for the previous kernel).
+      auto load_q = [&]() -> bool {
+        if (seg == 0 && P.lists_stable) pdl_wait();
+        if (!mbar_wait(&sh.q_empty, (seg & 1u) ^ 1u, &sh.abort_flag)) return false;
+        const uint32_t qb = smem_u32(sh.q);
+        for (int i = lane; i < P.M * 16; i += 32) {
+          const int r = i >> 4, c = i & 15;
+          const int t = r / P.grp, h = kvh * P.grp + r % P.grp;
+          cp_async16(qb + tc_sw(r, c, 64), P.q + ((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD + c * 8);
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.q_full);
+        return true;
+      };
+      bool q_pending = (pw == 0);
+      if (q_pending && seg > 0) {
+        q_pending = false;
+        if (!load_q()) { sh.abort_flag = 1; dead = true; break; }
+      }
+      // lane j resolves keys j and j + 32 of this warp's half tile to the byte offset of their K row
+      auto resolve = [&](int h0, long long (&off)[2]) -> bool {
+        const int ntok = min(64, tok_hi - h0);
+        bool bad = false;
+        if (ntok <= 0) return false;
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj) {
+          const int jt = min(lane + jj * 32, ntok - 1);
+          const int k = h0 + jt;  // token index inside the unit: the list first, then the tail
+          int pos = (k >= c_list) ? (kvlen_b + (k - c_list)) : (P.dense ? k : __ldg(list + k));
+          if (pos < 0 || pos >= kvlen_b + P.tail) { bad = true; pos = 0; }
+          const int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
+          const int slot = pos - lp * P.page_size;
+          long long page = P.bt ? static_cast<long long>(__ldg(P.bt + b * P.bt_stride + lp))
+                                : (b * P.bt_stride + lp);
+          if (page < 0 || (P.n_pages > 0 && page >= P.n_pages)) { bad = true; page = 0; }
+          off[jj] = (page * P.s_page + static_cast<long long>(slot) * P.s_slot) * 2;
+        }
+        return bad;
+      };
+      long long off_next[2] = {0, 0};
+      bool bad_next = false;
+      int t0_next = -1;
+      for (int t0 = tok_lo; t0 < tok_hi; t0 += kTcTile, ++it) {
+        if ((it & 1) != tpar) continue;
+        const int s = it % NS;
+        const unsigned ph = (it / NS) & 1u;
+        const int h0 = t0 + half * 64;
+        long long off[2] = {0, 0};
+        bool bad;
+        if (t0_next == t0) {
+          off[0] = off_next[0];
+          off[1] = off_next[1];
+          bad = bad_next;
+        } else {
+          bad = resolve(h0, off);
+        }
+        t0_next = t0 + 2 * kTcTile;
+        if (t0_next < tok_hi) bad_next = resolve(t0_next + half * 64, off_next); else t0_next = -1;
+        if (!mbar_wait(&sh.empty[s], ph ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
+        const int ntok = max(0, min(64, tok_hi - h0));
+        const int npad = (ntok + 15) & ~15;  // the P V product runs over whole 16-key steps
+        const char* kbase = reinterpret_cast<const char*>(kv_head) + (lane & 15) * 16;
+        const long long v_delta = P.s_kv * 2;
+        const uint32_t k_dst = smem_u32(sh.kv[s]);
+        const uint32_t v_dst = k_dst + kTcTileBytes;
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj) {
+#pragma unroll 4
+          for (int i = 0; i < 16; ++i) {
+            const int tok = jj * 32 + 2 * i + (lane >> 4);
+            const long long o = __shfl_sync(0xffffffffu, off[jj], 2 * i + (lane >> 4));
+            if (tok < npad) {
+              const uint32_t d = tc_sw(half * 64 + tok, lane & 15, kTcTile);
+              cp_async16(k_dst + d, kbase + o);
+              cp_async16(v_dst + d, kbase + o + v_delta);
+            }
           }
-          asm volatile("cp.async.wait_all;" ::: "memory");
-          fence_proxy_async();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sh.q_full);
-          return true;
-        };
-        bool q_pending = (pw == 0);
-        if (q_pending && seg > 0) {
+        }
+        asm volatile("cp.async.wait_all;" ::: "memory");
+        fence_proxy_async();  // generic-proxy writes -> visible to the tensor core's reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.full[s]);
+        if (bad && P.status) atomicOr(P.status + b, SPECATTN_ROW_BAD_INDEX);
+        if (q_pending) {
           q_pending = false;
           if (!load_q()) { sh.abort_flag = 1; dead = true; break; }
         }
-        auto resolve = [&](int t0, long long (&off)[2]) -> bool {
-          const int ntok = min(kTcTile, tok_hi - t0);
-          bool bad = false;
-#pragma unroll
-          for (int jj = 0; jj < 2; ++jj) {
-            const int jt = min(lane + jj * 32, ntok - 1);
-            const int k = t0 + jt;
-            int pos = (k >= c_list) ? (kvlen_b + (k - c_list)) : (P.dense ? k : __ldg(list + k));
-            if (pos < 0 || pos >= kvlen_b + P.tail) { bad = true; pos = 0; }
-            const int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
-            const int slot = pos - lp * P.page_size;
-            long long page = P.bt ? static_cast<long long>(__ldg(P.bt + b * P.bt_stride + lp))
-                                  : (b * P.bt_stride + lp);
-            if (page < 0 || (P.n_pages > 0 && page >= P.n_pages)) { bad = true; page = 0; }
-            off[jj] = (page * P.s_page + static_cast<long long>(slot) * P.s_slot) * 2;
-          }
-          return bad;
-        };
-        long long off_next[2] = {0, 0};
-        bool bad_next = false;
-        int t0_next = -1;
-        for (int t0 = tok_lo; t0 < tok_hi; t0 += kTcTile, ++it) {
-          if ((it % NS) != pw) continue;
-          const int s = it % NS;
-          const unsigned ph = (it / NS) & 1u;
-          long long off[2];
-          bool bad;
-          if (t0_next == t0) {
-            off[0] = off_next[0];
-            off[1] = off_next[1];
-            bad = bad_next;
-          } else {
-            bad = resolve(t0, off);
-          }
-          t0_next = t0 + NS * kTcTile;
-          if (t0_next < tok_hi) bad_next = resolve(t0_next, off_next); else t0_next = -1;
-          if (!mbar_wait(&sh.empty[s], ph ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
-          const int ntok = min(kTcTile, tok_hi - t0);
-          const int npad = (ntok + 15) & ~15;  // the P V product runs over whole 16-key steps
-          const char* kbase = reinterpret_cast<const char*>(kv_head) + (lane & 15) * 16;
-          const long long v_delta = P.s_kv * 2;
-          const uint32_t k_dst = smem_u32(sh.kv[s]);
-          const uint32_t v_dst = k_dst + kTcTileBytes;
-#pragma unroll
-          for (int jj = 0; jj < 2; ++jj) {
-#pragma unroll 4
-            for (int i = 0; i < 16; ++i) {
-              const int tok = jj * 32 + 2 * i + (lane >> 4);
-              const long long o = __shfl_sync(0xffffffffu, off[jj], 2 * i + (lane >> 4));
-              if (tok < npad) {
-                const uint32_t d = tc_sw(tok, lane & 15, kTcTile);
-                cp_async16(k_dst + d, kbase + o);
-                cp_async16(v_dst + d, kbase + o + v_delta);
-              }
-            }
-          }
-          asm volatile("cp.async.wait_all;" ::: "memory");
-          fence_proxy_async();  // generic-proxy writes -> visible to the tensor core's reads
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sh.full[s]);
-          if (bad && P.status) atomicOr(P.status + b, SPECATTN_ROW_BAD_INDEX);
-          if (q_pending) {
-            q_pending = false;
-            if (!load_q()) { sh.abort_flag = 1; dead = true; break; }
-          }
-        }
-        ++seg;
-        next_unit(a, u, seg_hi, ue);
       }
+      ++seg;
+      next_unit(a, u, seg_hi, ue);
     }
     return;
   }
 
-  bool ok = true;
   if (is_mma) {
     // =============================== MMA issue warp (one thread) =================================
     if (lane == 0) {
-      const uint32_t idesc_qk = tc_idesc(128, kTcTile, 0, 0);
-      const uint32_t idesc_pv = tc_idesc(128, kD, 0, 1);
+      const uint32_t idesc = tc_idesc(128, N, 0, 0);      // S^T = K Q^T: both operands K-major
+      const uint32_t idesc_pv = tc_idesc(128, N, 1, 1);   // O^T += V^T P^T: both MN-major
       const uint32_t q_base = smem_u32(sh.q);
+      bool ok = true;
       int it = 0, seg = 0;
-      int o_used[2] = {0, 0};  // segments so far in which each parity accumulated
       int a = a0, u = u_first;
-      auto issue_pv = [&](int j, int ntok, bool first) {
-        const int par = j & 1, s = j % NS;
-        const uint32_t v_base = smem_u32(sh.kv[s]) + kTcTileBytes;
-        const int ksteps = (ntok + 15) >> 4;
-        for (int kk = 0; kk < ksteps; ++kk)
-          tc_mma_ts(col_o(par), col_phi(par) + kk * 8, tc_desc(v_base + kk * 2048, 8192, 1024), idesc_pv,
-                    (first && kk == 0) ? 0u : 1u);
-        for (int kk = 0; kk < ksteps; ++kk)
-          tc_mma_ts(col_o(par), col_plo(par) + kk * 8, tc_desc(v_base + kk * 2048, 8192, 1024), idesc_pv, 1u);
-        tc_commit(&sh.empty[s]);
-        tc_commit(&sh.pv_done[par]);
-      };
       while (a < a1 && ok) {
         const int us = sh.unit_start[u], ue = sh.unit_start[u + 1];
         const int seg_hi = min(a1, ue);
         const int tok_lo = (a - us) * kAtom;
-        const int tok_hi = min(sh.unit_cnt[u], (seg_hi - us) * kAtom);
+        const int tok_hi = min(unit_count(P, u), (seg_hi - us) * kAtom);
         const int ntiles = (tok_hi - tok_lo + kTcTile - 1) / kTcTile;
         if (!mbar_wait(&sh.q_full, seg & 1u, &sh.abort_flag)) { ok = false; break; }
-        bool o_waited[2] = {false, false};
-        bool first_pv[2] = {true, true};
         for (int n = 0; n <= ntiles && ok; ++n) {
-          if (n < ntiles) {  // S = Q K^T of tile it + n
-            const int i = it + n, s = i % NS, par = i & 1;
+          if (n < ntiles) {  // S^T of tile it + n
+            const int i = it + n, s = i % NS, sb = i & 1;
             if (!mbar_wait(&sh.full[s], (i / NS) & 1u, &sh.abort_flag)) { ok = false; break; }
-            if (!mbar_wait(&sh.s_free[par], ((i >> 1) & 1u) ^ 1u, &sh.abort_flag)) { ok = false; break; }
+            if (!mbar_wait(&sh.s_free[sb], ((i >> 1) & 1u) ^ 1u, &sh.abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t k_base = smem_u32(sh.kv[s]);
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)
-              tc_mma_ss(col_s(par), tc_desc(q_base + (kk >> 2) * (128 * 128) + (kk & 3) * 32, 16, 1024),
-                        tc_desc(k_base + (kk >> 2) * (kTcTile * 128) + (kk & 3) * 32, 16, 1024), idesc_qk, kk > 0);
-            tc_commit(&sh.s_full[par]);
+              tc_mma_ss(tmem + sb * N, tc_desc(k_base + (kk >> 2) * (kTcTile * 128) + (kk & 3) * 32, 16, 1024),
+                        tc_desc(q_base + (kk >> 2) * (64 * 128) + (kk & 3) * 32, 16, 1024), idesc, kk > 0);
+            tc_commit(&sh.s_full[sb]);
             if (n == ntiles - 1) tc_commit(&sh.q_empty);  // the query tile may be replaced
           }
-          if (n > 0) {  // O += P V of tile it + n - 1
-            const int j = it + n - 1, par = j & 1;
-            if (!o_waited[par]) {  // this parity's O rows of its previous segment have been read out
-              if (!mbar_wait(&sh.o_free[par], (o_used[par] & 1u) ^ 1u, &sh.abort_flag)) { ok = false; break; }
-              o_waited[par] = true;
-            }
-            if (!mbar_wait(&sh.p_full[par], (j >> 1) & 1u, &sh.abort_flag)) { ok = false; break; }
+          if (n > 0) {  // O^T += V^T P^T of tile it + n - 1
+            const int j = it + n - 1, s = j % NS;
+            if (n == 1 && !mbar_wait(&sh.o_free, (seg & 1u) ^ 1u, &sh.abort_flag)) { ok = false; break; }
+            if (!mbar_wait(&sh.p_full, j & 1u, &sh.abort_flag)) { ok = false; break; }
             tc_fence_after();
-            issue_pv(j, min(kTcTile, tok_hi - (tok_lo + (n - 1) * kTcTile)), first_pv[par]);
-            first_pv[par] = false;
+            const int ntok = min(kTcTile, tok_hi - (tok_lo + (n - 1) * kTcTile));
+            const int ksteps = (ntok + 15) >> 4;
+            const uint32_t p_base = smem_u32(sh.kv[s]);          // P^T hi, then lo, in the K tile's bytes
+            const uint32_t v_base = p_base + kTcTileBytes;
+            for (int kk = 0; kk < ksteps; ++kk)
+              tc_mma_ss(col_o, tc_desc(v_base + kk * 2048, kTcTile * 128, 1024), tc_desc(p_base + kk * 2048, 0, 1024),
+                        idesc_pv, (n == 1 && kk == 0) ? 0u : 1u);
+            for (int kk = 0; kk < ksteps; ++kk)
+              tc_mma_ss(col_o, tc_desc(v_base + kk * 2048, kTcTile * 128, 1024),
+                        tc_desc(p_base + 16384 + kk * 2048, 0, 1024), idesc_pv, 1u);
+            tc_commit(&sh.empty[s]);
+            tc_commit(&sh.pv_done);
           }
         }
-        // o_free[par] completes one phase per segment in which that parity had a tile: a parity
-        // without one neither arrives nor is waited for, so no phase can ever be skipped
-        for (int par = 0; par < 2; ++par)
-          if (o_waited[par]) ++o_used[par];
         it += ntiles;
         ++seg;
         next_unit(a, u, seg_hi, ue);
@@ -494,247 +510,292 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
     __syncwarp();
   } else {
     // =============================== softmax warps ==============================================
-    const int par = warp >> 2;  // tiles with (tile index & 1) == par
-    const int rb = warp & 1;    // rows rb * 32 .. rb * 32 + 31 of the query block
-    const bool active = rb < NB;
-    const int row = rb * 32 + lane;
-    const uint32_t lane_sel = static_cast<uint32_t>(rb * 32) << 16;
-    const int t_row = row / P.grp;
-    const int lim = t_row + P.tail_off;  // last in-flight token this row may see
+    const int key_lane = tid;  // key of the tile / output dimension = TMEM lane
+    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
+    constexpr int kBar = 1;
+    bool fail = false;
     int it = 0, seg = 0;
+    int pv_next = 0;  // next phase of pv_done not yet waited for (every phase is waited, in order)
+    auto pv_catch_up = [&](int upto) {
+      while (pv_next <= upto) {
+        if (!mbar_wait(&sh.pv_done, pv_next & 1u, &sh.abort_flag)) { fail = true; return; }
+        ++pv_next;
+      }
+    };
     int a = a0, u = u_first;
-    while (active && a < a1) {
+    while (a < a1) {
       const int us = sh.unit_start[u], ue = sh.unit_start[u + 1];
       const int seg_hi = min(a1, ue);
       const int b = u / P.Hkv, kvh = u % P.Hkv;
+      const int ucnt = unit_count(P, u);
       const int tok_lo = (a - us) * kAtom;
-      const int tok_hi = min(sh.unit_cnt[u], (seg_hi - us) * kAtom);
-      const int c_list = sh.unit_cnt[u] - P.tail;
+      const int tok_hi = min(ucnt, (seg_hi - us) * kAtom);
+      const int c_list = ucnt - P.tail;
       const int ntiles = (tok_hi - tok_lo + kTcTile - 1) / kTcTile;
-      float m_ref = -INFINITY, l = 0.f;  // reference maximum (scaled log2 domain), row sum
-      bool has_acc = false;
-      int last_i = -1;
-      for (int n = 0; n < ntiles && ok; ++n) {
-        const int i = it + n;
-        if ((i & 1) != par) continue;
+      if (tid < N) sh.m_ref[tid] = -INFINITY;
+      float l_part[N];
+#pragma unroll
+      for (int r = 0; r < N; ++r) l_part[r] = 0.f;
+      if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
+
+      for (int n = 0; n < ntiles; ++n) {
+        const int i = it + n, s = i % NS, sb = i & 1;
         const int t0 = tok_lo + n * kTcTile;
         const int ntok = min(kTcTile, tok_hi - t0);
-        if (!mbar_wait(&sh.s_full[par], (i >> 1) & 1u, &sh.abort_flag)) { ok = false; break; }
+        const bool kvalid = key_lane < ntok;
+        // in-flight token index of this key (negative: a listed row, visible to every query)
+        const int jt = P.tail ? (key_lane - (c_list - t0)) : -1;
+        if (!fail && !mbar_wait(&sh.s_full[sb], (i >> 1) & 1u, &sh.abort_flag)) fail = true;
         tc_fence_after();
-        uint32_t s0[32], s1[32];
-        SPECATTN_TMEM_LD32(s0, col_s(par) + lane_sel);
-        SPECATTN_TMEM_LD32(s1, col_s(par) + lane_sel + 32);
-        tc_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.s_free[par]);
-        // mask keys that do not exist and in-flight tokens this row may not see yet
-        const int tb = P.tail ? (c_list - t0) : (1 << 20);
-        float tmax = -INFINITY;
+        // ---- pass 1: does any visible score exceed its row's reference maximum by 2^8? --------
+        bool exceed = false;
+        if (!__any_sync(0xffffffffu, fail)) {
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
-          float x = __uint_as_float(s0[k]), y = __uint_as_float(s1[k]);
-          if (k >= ntok || (k - tb >= 0 && k - tb > lim)) x = -INFINITY;
-          if (k + 32 >= ntok || (k + 32 - tb >= 0 && k + 32 - tb > lim)) y = -INFINITY;
-          s0[k] = __float_as_uint(x);
-          s1[k] = __float_as_uint(y);
-          tmax = fmaxf(tmax, fmaxf(x, y));
-        }
-        tmax *= P.scale_log2;
-        // P[par] and O[par] are quiet once the P V product of this parity's previous tile is done
-        if (!mbar_wait(&sh.pv_done[par], ((i >> 1) & 1u) ^ 1u, &sh.abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        const bool raise = (tmax > m_ref + kTcRaise) || (m_ref == -INFINITY && tmax > -INFINITY);
-        if (__any_sync(0xffffffffu, raise && has_acc)) {
-          // rescale this warp's O rows in tensor memory (rows that do not raise scale by 1)
-          const float alpha = (raise && has_acc) ? ex2(m_ref - tmax) : 1.f;
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            uint32_t o[32];
-            SPECATTN_TMEM_LD32(o, col_o(par) + lane_sel + c * 32);
+          for (int c = 0; c < NT; ++c) {
+            uint32_t sv[16];
+            tc_ld16(sv, tmem + sb * N + lane_sel + c * 16);
             tc_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * alpha);
-            SPECATTN_TMEM_ST32(col_o(par) + lane_sel + c * 32, o);
+            for (int j = 0; j < 16; ++j) {
+              const int r = c * 16 + j;
+              const bool vis = kvalid && !(jt >= 0 && jt > sh.row_lim[r]);
+              const float x = fmaf(__uint_as_float(sv[j]), P.scale_log2, -sh.m_ref[r]);
+              exceed |= vis && !(x <= kTcRaise);
+            }
           }
-          tc_wait_st();
         }
-        if (raise) {
-          l *= (m_ref == -INFINITY) ? 0.f : ex2(m_ref - tmax);
-          m_ref = tmax;
-        }
-        const float base = (m_ref == -INFINITY) ? 0.f : m_ref;
-        float sum = 0.f;
-        uint32_t phi[32], plo[32];
+        if (__any_sync(0xffffffffu, exceed) && lane == 0) sh.raise_tile[sb] = i + 1;
+        if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
+        if (sh.raise_tile[sb] == i + 1) {
+          // ---- slow path: new row maxima, rescale of the sums and of O^T ----------------------
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-          const float x0 = ex2(fmaf(__uint_as_float(s0[2 * k]), P.scale_log2, -base));
-          const float x1 = ex2(fmaf(__uint_as_float(s0[2 * k + 1]), P.scale_log2, -base));
-          const float y0 = ex2(fmaf(__uint_as_float(s1[2 * k]), P.scale_log2, -base));
-          const float y1 = ex2(fmaf(__uint_as_float(s1[2 * k + 1]), P.scale_log2, -base));
-          sum += (x0 + x1) + (y0 + y1);
-          const uint32_t hx = pack_bf16(x0, x1), hy = pack_bf16(y0, y1);
-          phi[k] = hx;
-          phi[16 + k] = hy;
-          plo[k] = pack_bf16(x0 - __uint_as_float(hx << 16), x1 - __uint_as_float(hx & 0xffff0000u));
-          plo[16 + k] = pack_bf16(y0 - __uint_as_float(hy << 16), y1 - __uint_as_float(hy & 0xffff0000u));
-        }
-        l += sum;
-        SPECATTN_TMEM_ST32(col_phi(par) + lane_sel, phi);
-        SPECATTN_TMEM_ST32(col_plo(par) + lane_sel, plo);
-        tc_wait_st();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.p_full[par]);
-        has_acc = true;
-        last_i = i;
-      }
-      // ---- end of the unit's share: read this parity's O rows, hand the columns back -----------
-      float acc[kD];
-      if (ok && has_acc) {
-        if (!mbar_wait(&sh.pv_done[par], (last_i >> 1) & 1u, &sh.abort_flag)) ok = false;
-        tc_fence_after();
-      }
-      if (ok && has_acc) {
+          for (int blk = 0; blk < NBLK; ++blk) {
+            float v[32];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t o[32];
-          SPECATTN_TMEM_LD32(o, col_o(par) + lane_sel + c * 32);
+            for (int c = 0; c < 2; ++c) {
+              if (blk * 2 + c < NT) {
+                uint32_t sv[16];
+                tc_ld16(sv, tmem + sb * N + lane_sel + (blk * 2 + c) * 16);
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  const int r = blk * 32 + c * 16 + j;
+                  const bool vis = kvalid && !(jt >= 0 && jt > sh.row_lim[r]);
+                  v[c * 16 + j] = vis ? __uint_as_float(sv[j]) * P.scale_log2 : -INFINITY;
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[c * 16 + j] = -INFINITY;
+              }
+            }
+            const float wm = tc_reduce_scatter<true>(v, lane);
+            if (blk * 32 + lane < N) sh.wred[warp][blk * 32 + lane] = wm;
+          }
+          if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
+          if (tid < N) {
+            const float mo = sh.m_ref[tid];
+            const float mn = fmaxf(fmaxf(mo, sh.wred[0][tid]),
+                                   fmaxf(sh.wred[1][tid], fmaxf(sh.wred[2][tid], sh.wred[3][tid])));
+            sh.alpha[tid] = (mo == -INFINITY) ? 0.f : ex2(mo - mn);
+            sh.m_ref[tid] = mn;
+          }
+          if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
+          if (n > 0) {  // O^T holds this unit's earlier tiles: quiet once their P V products are done
+            pv_catch_up(i - 1);
+            tc_fence_after();
+            if (!__any_sync(0xffffffffu, fail)) {
+#pragma unroll
+              for (int c = 0; c < NT; ++c) {
+                uint32_t ov[16];
+                tc_ld16(ov, col_o + lane_sel + c * 16);
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * sh.alpha[c * 16 + j]);
+                tc_st16(col_o + lane_sel + c * 16, ov);
+              }
+              tc_wait_st();
+            }
+          }
+#pragma unroll
+          for (int r = 0; r < N; ++r) l_part[r] *= sh.alpha[r];
+        }
+        // ---- pass 2: P = exp2(S - m) as two bf16 terms, into the dead K tile ------------------
+        if (!__any_sync(0xffffffffu, fail)) {
+          const uint32_t pb = smem_u32(sh.kv[s]) + (key_lane >> 3) * 1024 + (key_lane & 7) * 128;
+#pragma unroll
+          for (int c = 0; c < NT; ++c) {
+            uint32_t sv[16];
+            tc_ld16(sv, tmem + sb * N + lane_sel + c * 16);
+            tc_wait_ld();
+            if (c == NT - 1) {  // S^T buffer read for the last time
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&sh.s_free[sb]);
+            }
+            float p[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int r = c * 16 + j;
+              const bool vis = kvalid && !(jt >= 0 && jt > sh.row_lim[r]);
+              const float x = fmaf(__uint_as_float(sv[j]), P.scale_log2, -sh.m_ref[r]);
+              p[j] = vis ? ex2(x) : 0.f;
+              l_part[r] += p[j];
+            }
+#pragma unroll
+            for (int g8 = 0; g8 < 2; ++g8) {
+              uint32_t hi[4], lo[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float x0 = p[g8 * 8 + 2 * e], x1 = p[g8 * 8 + 2 * e + 1];
+                hi[e] = pack_bf16(x0, x1);
+                lo[e] = pack_bf16(x0 - __uint_as_float(hi[e] << 16), x1 - __uint_as_float(hi[e] & 0xffff0000u));
+              }
+              const uint32_t dst = pb + ((((c * 2 + g8) ^ (key_lane & 7))) << 4);
+              st_shared_v4(dst, hi[0], hi[1], hi[2], hi[3]);
+              st_shared_v4(dst + 16384, lo[0], lo[1], lo[2], lo[3]);
+            }
+          }
+          fence_proxy_async();  // P^T is read by the tensor core through the async proxy
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.p_full);
+        }
+        if (n > 0 && !fail) pv_catch_up(i - 1);
+      }
+      if (fail) sh.abort_flag = 1;
+
+      // ---- end of the unit's share: row sums over all keys, O^T out of tensor memory ------------
+#pragma unroll
+      for (int blk = 0; blk < NBLK; ++blk) {
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = (blk * 32 + j < N) ? l_part[(blk * 32 + j < N) ? blk * 32 + j : 0] : 0.f;
+        const float ws = tc_reduce_scatter<false>(v, lane);
+        if (blk * 32 + lane < N) sh.wred[warp][blk * 32 + lane] = ws;
+      }
+      if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
+      if (tid < N) sh.lsum[tid] = (sh.wred[0][tid] + sh.wred[1][tid]) + (sh.wred[2][tid] + sh.wred[3][tid]);
+      pv_catch_up(it + ntiles - 1);
+      tc_fence_after();
+      if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
+
+      const bool whole = (a == us) && (seg_hi == ue);
+      const long long obase = static_cast<long long>(b) * P.T * P.Hq + kvh * P.grp;
+      const int d = key_lane;  // this thread's output dimension
+      if (whole) {
+#pragma unroll
+        for (int c = 0; c < NT; ++c) {
+          uint32_t ov[16];
+          tc_ld16(ov, col_o + lane_sel + c * 16);
           tc_wait_ld();
 #pragma unroll
-          for (int k = 0; k < 32; ++k) acc[c * 32 + k] = __uint_as_float(o[k]);
+          for (int j = 0; j < 16; ++j) {
+            const int r = c * 16 + j;
+            if (r < P.M) {
+              const float l = sh.lsum[r];
+              P.out[(obase + sh.row_off[r]) * kD + d] = __uint_as_float(ov[j]) * ((l > 0.f) ? 1.f / l : 0.f);
+            }
+          }
+        }
+        if (tid < P.M) {
+          const float l = sh.lsum[tid];
+          P.lse[obase + sh.row_off[tid]] = (l > 0.f) ? (sh.m_ref[tid] + log2f(l)) * kLn2 : -INFINITY;
         }
       } else {
+        // publish this CTA's share ([row][dim] sums, then m, then l), then see who arrived last
+        float* rec = P.partials + static_cast<size_t>(2 * blockIdx.x + (a == a0 ? 0 : 1)) * NBLK * kTcRec;
 #pragma unroll
-        for (int k = 0; k < kD; ++k) acc[k] = 0.f;
+        for (int c = 0; c < NT; ++c) {
+          uint32_t ov[16];
+          tc_ld16(ov, col_o + lane_sel + c * 16);
+          tc_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 16; ++j) __stcg(rec + (c * 16 + j) * kD + d, __uint_as_float(ov[j]));
+        }
+        if (tid < N) {
+          __stcg(rec + N * kD + tid, sh.m_ref[tid]);
+          __stcg(rec + N * kD + N + tid, sh.lsum[tid]);
+        }
+        __threadfence();
+        if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
+        const int i_lo = aligned ? sh.part_start[u] : cta_of_atom(us, NA, NP);
+        const int i_hi = aligned ? sh.part_start[u + 1] - 1 : cta_of_atom(ue - 1, NA, NP);
+        if (tid == 0) {
+          const unsigned int old = atomicAdd(P.counters + u * kCountersPerUnit, 1u);
+          sh.last_arriver = (old == static_cast<unsigned int>(i_hi - i_lo)) ? 1 : 0;
+        }
+        if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
+        if (sh.last_arriver) {
+          __threadfence();
+          // merge every contributor's record in CTA order, 16 query rows at a time
+          auto rec_of = [&](int i) {
+            return P.partials + static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, NA, NP) >= us) ? 0 : 1)) *
+                                    NBLK * kTcRec;
+          };
+#pragma unroll 1
+          for (int c = 0; c < NT; ++c) {
+            float mx[16], acc[16], ls[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) { mx[j] = -INFINITY; acc[j] = 0.f; ls[j] = 0.f; }
+            for (int i = i_lo; i <= i_hi; ++i) {
+              const float* r2 = rec_of(i) + N * kD + c * 16;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) mx[j] = fmaxf(mx[j], __ldcg(r2 + j));
+            }
+            for (int i = i_lo; i <= i_hi; ++i) {
+              const float* r2 = rec_of(i);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const float base = (mx[j] == -INFINITY) ? 0.f : mx[j];
+                const float w = ex2(__ldcg(r2 + N * kD + c * 16 + j) - base);
+                ls[j] += __ldcg(r2 + N * kD + N + c * 16 + j) * w;
+                acc[j] += __ldcg(r2 + (c * 16 + j) * kD + d) * w;
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const int r = c * 16 + j;
+              if (r < P.M) {
+                P.out[(obase + sh.row_off[r]) * kD + d] = acc[j] * ((ls[j] > 0.f) ? 1.f / ls[j] : 0.f);
+                if (d == 0) P.lse[obase + sh.row_off[r]] = (ls[j] > 0.f) ? (mx[j] + log2f(ls[j])) * kLn2 : -INFINITY;
+              }
+            }
+          }
+          if (tid == 0) P.counters[u * kCountersPerUnit] = 0u;  // ready for the next call
+        }
       }
+      // O^T may be overwritten by the next unit
       tc_fence_before();
       __syncwarp();
-      if (has_acc && lane == 0) mbar_arrive(&sh.o_free[par]);
-      if (!ok) sh.abort_flag = 1;
-
-      // combine the two parities of this row block (warps w and w + 4) through shared memory
-      float m = m_ref;
-      if (par == 1) {
-        float* rec = sh.scratch[rb];
-#pragma unroll
-        for (int k = 0; k < kD; ++k) rec[k * 32 + lane] = acc[k];
-        rec[128 * 32 + lane] = m;
-        rec[129 * 32 + lane] = l;
-      }
-      named_bar_sync(1 + rb, 64);
-      if (par == 0) {
-        const float* rec = sh.scratch[rb];
-        float mn, ao, ai;
-        merge_scales(m, rec[128 * 32 + lane], mn, ao, ai);
-        l = l * ao + rec[129 * 32 + lane] * ai;
-        m = mn;
-#pragma unroll
-        for (int k = 0; k < kD; ++k) acc[k] = acc[k] * ao + rec[k * 32 + lane] * ai;
-      }
-      named_bar_sync(1 + rb, 64);
-      if (sh.abort_flag) { ok = false; break; }
-
-      if (par == 0) {
-        const bool whole = (a == us) && (seg_hi == ue);
-        bool finish = whole;
-        const bool pair_merge = paired && aligned && !whole && (sh.part_start[u + 1] - sh.part_start[u] == 2) &&
-                                ((sh.part_start[u] & 1) == 0);
-        if (pair_merge) {
-          if (cluster_cta_rank() == 1) {
-            const uint32_t dst = map_to_cta(smem_u32(sh.peer_rec[rb]), 0) + lane * 4;
-#pragma unroll
-            for (int k = 0; k < kD; ++k) st_cluster_f32(dst + k * 128, acc[k]);
-            st_cluster_f32(dst + 128 * 128, m);
-            st_cluster_f32(dst + 129 * 128, l);
-            __syncwarp();
-            if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&sh.peer_full), 0));
-          } else {
-            if (!mbar_wait_cluster(&sh.peer_full, 0u, &sh.abort_flag)) { sh.abort_flag = 1; ok = false; break; }
-            const float* rec = sh.peer_rec[rb];
-            float mn, ao, ai;
-            merge_scales(m, rec[128 * 32 + lane], mn, ao, ai);
-            l = l * ao + rec[129 * 32 + lane] * ai;
-            m = mn;
-#pragma unroll
-            for (int k = 0; k < kD; ++k) acc[k] = acc[k] * ao + rec[k * 32 + lane] * ai;
-            finish = true;
-          }
-        } else if (!whole) {
-          float* rec = P.partials + (static_cast<size_t>(2 * blockIdx.x + (a == a0 ? 0 : 1)) * NB + rb) * kTcRec;
-#pragma unroll
-          for (int k = 0; k < kD; ++k) __stcg(rec + k * 32 + lane, acc[k]);
-          __stcg(rec + 128 * 32 + lane, m);
-          __stcg(rec + 129 * 32 + lane, l);
-          __threadfence();
-          __syncwarp();
-          const int i_lo = aligned ? sh.part_start[u] : cta_of_atom(us, N, NP);
-          const int i_hi = aligned ? sh.part_start[u + 1] - 1 : cta_of_atom(ue - 1, N, NP);
-          unsigned int old = 0;
-          if (lane == 0) old = atomicAdd(P.counters + u * kCountersPerUnit + rb, 1u);
-          old = __shfl_sync(0xffffffffu, old, 0);
-          if (old == static_cast<unsigned int>(i_hi - i_lo)) {
-            finish = true;
-            __threadfence();
-            // merge every contributor's record in CTA order (the own one included, from memory)
-            m = -INFINITY;
-            for (int i = i_lo; i <= i_hi; ++i) {
-              const float* r2 = P.partials +
-                  (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * NB + rb) * kTcRec;
-              m = fmaxf(m, __ldcg(r2 + 128 * 32 + lane));
-            }
-            const float base = (m == -INFINITY) ? 0.f : m;
-            l = 0.f;
-#pragma unroll
-            for (int k = 0; k < kD; ++k) acc[k] = 0.f;
-            for (int i = i_lo; i <= i_hi; ++i) {
-              const float* r2 = P.partials +
-                  (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * NB + rb) * kTcRec;
-              const float w = ex2(__ldcg(r2 + 128 * 32 + lane) - base);
-              l += __ldcg(r2 + 129 * 32 + lane) * w;
-#pragma unroll
-              for (int k = 0; k < kD; ++k) acc[k] += __ldcg(r2 + k * 32 + lane) * w;
-            }
-            if (lane == 0) P.counters[u * kCountersPerUnit + rb] = 0u;
-          }
-        }
-        if (finish && row < P.M) {
-          const float inv = (l > 0.f) ? 1.f / l : 0.f;
-          const int h = kvh * P.grp + row % P.grp;
-          const long long orow = (static_cast<long long>(b) * P.T + t_row) * P.Hq + h;
-          float4* o = reinterpret_cast<float4*>(P.out + orow * kD);
-#pragma unroll
-          for (int k = 0; k < kD / 4; ++k)
-            o[k] = make_float4(acc[4 * k] * inv, acc[4 * k + 1] * inv, acc[4 * k + 2] * inv, acc[4 * k + 3] * inv);
-          P.lse[orow] = (l > 0.f) ? (m + log2f(l)) * kLn2 : -INFINITY;
-        }
-      }
+      if (lane == 0) mbar_arrive(&sh.o_free);
       it += ntiles;
       ++seg;
       next_unit(a, u, seg_hi, ue);
     }
-    if (!ok && P.status && lane == 0) atomicOr(P.status, SPECATTN_ROW_TIMEOUT);
+    if (fail) {
+      sh.abort_flag = 1;
+      if (P.status && lane == 0) atomicOr(P.status, SPECATTN_ROW_TIMEOUT);
+    }
   }
 
   // ---- release tensor memory once every warp that touches it is done -----------------------------
   tc_fence_before();
-  named_bar_sync(5, 5 * 32);  // warps 0, 1, 2, 4, 5
+  named_bar_sync(2, 5 * 32);  // warps 0..4
   if (warp == 0) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
   }
 }
 
-template <int NB, int NS>
+template <int NT>
 cudaError_t launch_tc(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
-  const size_t smem = sizeof(TcShared<NB, NS>) + 1024;
+  const size_t smem = sizeof(TcShared) + 1024;
   static std::atomic<unsigned long long> done_mask{0};
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   if (!((done_mask.load(std::memory_order_acquire) >> dev) & 1ull)) {
-    err = cudaFuncSetAttribute(sparse_verify_tc_kernel<NB, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    err = cudaFuncSetAttribute(sparse_verify_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                static_cast<int>(smem));
     if (err != cudaSuccess) return err;
     done_mask.fetch_or(1ull << dev, std::memory_order_release);
@@ -745,19 +806,12 @@ cudaError_t launch_tc(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
   cfg.blockDim = dim3(kTcThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[2];
+  cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (n_ctas % 2 == 0) {
-    attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = 2;
-    attr[1].val.clusterDim.y = 1;
-    attr[1].val.clusterDim.z = 1;
-    cfg.numAttrs = 2;
-  }
-  err = cudaLaunchKernelEx(&cfg, sparse_verify_tc_kernel<NB, NS>, P);
+  err = cudaLaunchKernelEx(&cfg, sparse_verify_tc_kernel<NT>, P);
   if (err != cudaSuccess) cudaGetLastError();
   return err;
 }

@@ -22,7 +22,7 @@ class VerifyStep:
                  kv_pools: Sequence[torch.Tensor], kv_len: torch.Tensor,
                  block_table: torch.Tensor | None, pages_per_seq: int | None = None,
                  n_groups: int = 1, head_group: Sequence[int] | None = None,
-                 idx_stride: int | None = None, sm_scale: float = 0.0, device=None):
+                 idx_stride: int | None = None, sm_scale: float = 0.0, verify_flags: int = 0, device=None):
         dev = device or kv_pools[0].device
         self.layer_map = [int(x) for x in layer_map]
         self.n_layers = len(self.layer_map)
@@ -58,7 +58,7 @@ class VerifyStep:
                                  lse=self.lse[j], status=self.status[j],
                                  # after the first layer the lists (written by select) and the
                                  # context's K/V rows predate the preceding launch
-                                 flags=VERIFY_LISTS_STABLE if j > 0 else 0)
+                                 flags=(VERIFY_LISTS_STABLE if j > 0 else 0) | int(verify_flags))
             if self.workspace is None:
                 self.workspace = verify_workspace(a, dev)
             a.workspace, a.workspace_bytes = self.workspace.data_ptr(), self.workspace.numel()
