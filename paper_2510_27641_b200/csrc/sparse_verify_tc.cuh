@@ -105,6 +105,21 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
   asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+__device__ __forceinline__ void tc_lds16(float (&d)[16], const float* p) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float4 v = reinterpret_cast<const float4*>(p)[i];
+    d[4 * i] = v.x; d[4 * i + 1] = v.y; d[4 * i + 2] = v.z; d[4 * i + 3] = v.w;
+  }
+}
+__device__ __forceinline__ void tc_lds16(int (&d)[16], const int* p) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int4 v = reinterpret_cast<const int4*>(p)[i];
+    d[4 * i] = v.x; d[4 * i + 1] = v.y; d[4 * i + 2] = v.z; d[4 * i + 3] = v.w;
+  }
+}
+
 // Butterfly reduce-scatter over the 32 lanes of a warp: v[i] is this lane's value for row i;
 // afterwards lane r holds the reduction of row r (returned).  31 shuffles.
 template <bool kMax>
@@ -126,12 +141,12 @@ __device__ __forceinline__ float tc_reduce_scatter(float (&v)[32], int lane) {
 struct TcShared {
   alignas(1024) unsigned char kv[kTcStages][2 * kTcTileBytes];  // per stage: K tile (later P^T), V tile
   alignas(1024) unsigned char q[64 * 256];
-  float m_ref[64];     // reference maximum of every query row (scaled log2 domain)
-  float alpha[64];     // rescale factors of the tile that raised it
-  float lsum[64];      // row sums at the end of a unit
+  alignas(16) float m_ref[64];     // reference maximum of every query row (scaled log2 domain)
+  alignas(16) float alpha[64];     // rescale factors of the tile that raised it
+  alignas(16) float lsum[64];      // row sums at the end of a unit
   float wred[4][64];   // per-warp row maxima / row sums
   int row_off[64];     // query row r -> t * Hq + (r % grp): its output row inside (b, kv head)
-  int row_lim[64];     // last in-flight token row r may see
+  alignas(16) int row_lim[64];     // last in-flight token row r may see
   alignas(8) unsigned long long full[kTcStages];
   unsigned long long empty[kTcStages];
   unsigned long long q_full, q_empty;
@@ -313,7 +328,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
     while (sh.unit_start[u_first + 1] <= a0) ++u_first;
   }
 
-  // ---- tensor memory: S^T double-buffered (N columns each), O^T (N columns) ---------------------
+  // ---- tensor memory: S^T double-buffered (N columns each), O^T (2 N: P_hi and P_lo parts) ------
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)),
                  "r"(256u)
@@ -324,7 +339,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sh.tmem_base;
-  const uint32_t col_o = tmem + 2u * N;
+  const uint32_t col_o = tmem + 2u * N;  // 2 N columns: the P_hi part, then the P_lo part
 
   auto next_unit = [&](int& a, int& u, int seg_hi, int ue) {
     a = seg_hi;
@@ -456,7 +471,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
     // =============================== MMA issue warp (one thread) =================================
     if (lane == 0) {
       const uint32_t idesc = tc_idesc(128, N, 0, 0);      // S^T = K Q^T: both operands K-major
-      const uint32_t idesc_pv = tc_idesc(128, N, 1, 1);   // O^T += V^T P^T: both MN-major
+      const uint32_t idesc_pv = tc_idesc(128, 2 * N, 1, 1);  // [O_hi^T | O_lo^T] += V^T [P_hi^T | P_lo^T]
       const uint32_t q_base = smem_u32(sh.q);
       bool ok = true;
       int it = 0, seg = 0;
@@ -489,14 +504,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
             tc_fence_after();
             const int ntok = min(kTcTile, tok_hi - (tok_lo + (n - 1) * kTcTile));
             const int ksteps = (ntok + 15) >> 4;
-            const uint32_t p_base = smem_u32(sh.kv[s]);          // P^T hi, then lo, in the K tile's bytes
+            const uint32_t p_base = smem_u32(sh.kv[s]);          // [P_hi^T | P_lo^T] in the K tile's bytes
             const uint32_t v_base = p_base + kTcTileBytes;
             for (int kk = 0; kk < ksteps; ++kk)
-              tc_mma_ss(col_o, tc_desc(v_base + kk * 2048, kTcTile * 128, 1024), tc_desc(p_base + kk * 2048, 0, 1024),
-                        idesc_pv, (n == 1 && kk == 0) ? 0u : 1u);
-            for (int kk = 0; kk < ksteps; ++kk)
               tc_mma_ss(col_o, tc_desc(v_base + kk * 2048, kTcTile * 128, 1024),
-                        tc_desc(p_base + 16384 + kk * 2048, 0, 1024), idesc_pv, 1u);
+                        tc_desc(p_base + kk * 2048, 16384, 1024), idesc_pv, (n == 1 && kk == 0) ? 0u : 1u);
             tc_commit(&sh.empty[s]);
             tc_commit(&sh.pv_done);
           }
@@ -547,6 +559,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         const int jt = P.tail ? (key_lane - (c_list - t0)) : -1;
         if (!fail && !mbar_wait(&sh.s_full[sb], (i >> 1) & 1u, &sh.abort_flag)) fail = true;
         tc_fence_after();
+        // a tile that holds in-flight tokens masks per (key, query); all others per key only
+        const bool tail_tile = P.tail && (t0 + kTcTile > c_list);
         // ---- pass 1: does any visible score exceed its row's reference maximum by 2^8? --------
         bool exceed = false;
         if (!__any_sync(0xffffffffu, fail)) {
@@ -554,15 +568,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           for (int c = 0; c < NT; ++c) {
             uint32_t sv[16];
             tc_ld16(sv, tmem + sb * N + lane_sel + c * 16);
+            float mr[16];
+            tc_lds16(mr, sh.m_ref + c * 16);
             tc_wait_ld();
+            if (!tail_tile) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int r = c * 16 + j;
-              const bool vis = kvalid && !(jt >= 0 && jt > sh.row_lim[r]);
-              const float x = fmaf(__uint_as_float(sv[j]), P.scale_log2, -sh.m_ref[r]);
-              exceed |= vis && !(x <= kTcRaise);
+              for (int j = 0; j < 16; ++j)
+                exceed |= !(fmaf(__uint_as_float(sv[j]), P.scale_log2, -mr[j]) <= kTcRaise);
+            } else {
+              int lim[16];
+              tc_lds16(lim, sh.row_lim + c * 16);
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                exceed |= ((jt < 0) | (jt <= lim[j])) & !(fmaf(__uint_as_float(sv[j]), P.scale_log2, -mr[j]) <= kTcRaise);
             }
           }
+          exceed &= kvalid;
         }
         if (__any_sync(0xffffffffu, exceed) && lane == 0) sh.raise_tile[sb] = i + 1;
         if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
@@ -576,11 +597,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
               if (blk * 2 + c < NT) {
                 uint32_t sv[16];
                 tc_ld16(sv, tmem + sb * N + lane_sel + (blk * 2 + c) * 16);
+                int lim[16];
+                tc_lds16(lim, sh.row_lim + (blk * 2 + c) * 16);
                 tc_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
-                  const int r = blk * 32 + c * 16 + j;
-                  const bool vis = kvalid && !(jt >= 0 && jt > sh.row_lim[r]);
+                  const bool vis = kvalid & (!tail_tile | (jt < 0) | (jt <= lim[j]));
                   v[c * 16 + j] = vis ? __uint_as_float(sv[j]) * P.scale_log2 : -INFINITY;
                 }
               } else {
@@ -605,19 +627,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
             tc_fence_after();
             if (!__any_sync(0xffffffffu, fail)) {
 #pragma unroll
-              for (int c = 0; c < NT; ++c) {
+              for (int c = 0; c < 2 * NT; ++c) {  // the P_hi and the P_lo half of O^T
                 uint32_t ov[16];
                 tc_ld16(ov, col_o + lane_sel + c * 16);
+                float al[16];
+                tc_lds16(al, sh.alpha + (c % NT) * 16);
                 tc_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 16; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * sh.alpha[c * 16 + j]);
+                for (int j = 0; j < 16; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * al[j]);
                 tc_st16(col_o + lane_sel + c * 16, ov);
               }
               tc_wait_st();
             }
           }
 #pragma unroll
-          for (int r = 0; r < N; ++r) l_part[r] *= sh.alpha[r];
+          for (int c = 0; c < NT; ++c) {
+            float al[16];
+            tc_lds16(al, sh.alpha + c * 16);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) l_part[c * 16 + j] *= al[j];
+          }
         }
         // ---- pass 2: P = exp2(S - m) as two bf16 terms, into the dead K tile ------------------
         if (!__any_sync(0xffffffffu, fail)) {
@@ -626,6 +655,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           for (int c = 0; c < NT; ++c) {
             uint32_t sv[16];
             tc_ld16(sv, tmem + sb * N + lane_sel + c * 16);
+            float mr[16];
+            tc_lds16(mr, sh.m_ref + c * 16);
             tc_wait_ld();
             if (c == NT - 1) {  // S^T buffer read for the last time
               tc_fence_before();
@@ -634,12 +665,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
             }
             float p[16];
 #pragma unroll
+            for (int j = 0; j < 16; ++j) p[j] = ex2(fmaf(__uint_as_float(sv[j]), P.scale_log2, -mr[j]));
+            if (tail_tile) {
+              int lim[16];
+              tc_lds16(lim, sh.row_lim + c * 16);
+#pragma unroll
+              for (int j = 0; j < 16; ++j) p[j] = ((jt < 0) | (jt <= lim[j])) ? p[j] : 0.f;
+            }
+#pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const int r = c * 16 + j;
-              const bool vis = kvalid && !(jt >= 0 && jt > sh.row_lim[r]);
-              const float x = fmaf(__uint_as_float(sv[j]), P.scale_log2, -sh.m_ref[r]);
-              p[j] = vis ? ex2(x) : 0.f;
-              l_part[r] += p[j];
+              p[j] = kvalid ? p[j] : 0.f;
+              l_part[c * 16 + j] += p[j];
             }
 #pragma unroll
             for (int g8 = 0; g8 < 2; ++g8) {
@@ -650,9 +686,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
                 hi[e] = pack_bf16(x0, x1);
                 lo[e] = pack_bf16(x0 - __uint_as_float(hi[e] << 16), x1 - __uint_as_float(hi[e] & 0xffff0000u));
               }
-              const uint32_t dst = pb + ((((c * 2 + g8) ^ (key_lane & 7))) << 4);
-              st_shared_v4(dst, hi[0], hi[1], hi[2], hi[3]);
-              st_shared_v4(dst + 16384, lo[0], lo[1], lo[2], lo[3]);
+              // B operand [P_hi^T | P_lo^T]: 2N columns, 16-byte chunk ch of a key's row at
+              // (ch / 8) * 16 KB + ((ch % 8) ^ (key % 8)) * 16
+              const int ch_hi = c * 2 + g8, ch_lo = ch_hi + N / 8;
+              st_shared_v4(pb + (ch_hi >> 3) * 16384 + (((ch_hi & 7) ^ (key_lane & 7)) << 4), hi[0], hi[1], hi[2], hi[3]);
+              st_shared_v4(pb + (ch_lo >> 3) * 16384 + (((ch_lo & 7) ^ (key_lane & 7)) << 4), lo[0], lo[1], lo[2], lo[3]);
             }
           }
           fence_proxy_async();  // P^T is read by the tensor core through the async proxy
@@ -684,15 +722,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
       if (whole) {
 #pragma unroll
         for (int c = 0; c < NT; ++c) {
-          uint32_t ov[16];
+          uint32_t ov[16], ow[16];
           tc_ld16(ov, col_o + lane_sel + c * 16);
+          tc_ld16(ow, col_o + lane_sel + N + c * 16);
           tc_wait_ld();
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int r = c * 16 + j;
             if (r < P.M) {
               const float l = sh.lsum[r];
-              P.out[(obase + sh.row_off[r]) * kD + d] = __uint_as_float(ov[j]) * ((l > 0.f) ? 1.f / l : 0.f);
+              P.out[(obase + sh.row_off[r]) * kD + d] =
+                  (__uint_as_float(ov[j]) + __uint_as_float(ow[j])) * ((l > 0.f) ? 1.f / l : 0.f);
             }
           }
         }
@@ -705,11 +745,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         float* rec = P.partials + static_cast<size_t>(2 * blockIdx.x + (a == a0 ? 0 : 1)) * NBLK * kTcRec;
 #pragma unroll
         for (int c = 0; c < NT; ++c) {
-          uint32_t ov[16];
+          uint32_t ov[16], ow[16];
           tc_ld16(ov, col_o + lane_sel + c * 16);
+          tc_ld16(ow, col_o + lane_sel + N + c * 16);
           tc_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 16; ++j) __stcg(rec + (c * 16 + j) * kD + d, __uint_as_float(ov[j]));
+          for (int j = 0; j < 16; ++j)
+            __stcg(rec + (c * 16 + j) * kD + d, __uint_as_float(ov[j]) + __uint_as_float(ow[j]));
         }
         if (tid < N) {
           __stcg(rec + N * kD + tid, sh.m_ref[tid]);
