@@ -168,6 +168,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   constexpr int NS = kTcStages;
   constexpr int NTH = kTcThreads;
   constexpr int NBLK = (N + 31) / 32;
+  constexpr bool kKeepS = true;  // scores stay in registers between the two passes
   extern __shared__ __align__(1024) unsigned char smem_raw_tc[];
   TcShared& sh =
       *reinterpret_cast<TcShared*>((reinterpret_cast<uintptr_t>(smem_raw_tc) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -483,36 +484,55 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         const int tok_hi = min(unit_count(P, u), (seg_hi - us) * kAtom);
         const int ntiles = (tok_hi - tok_lo + kTcTile - 1) / kTcTile;
         if (!mbar_wait(&sh.q_full, seg & 1u, &sh.abort_flag)) { ok = false; break; }
-        for (int n = 0; n <= ntiles && ok; ++n) {
-          if (n < ntiles) {  // S^T of tile it + n
-            const int i = it + n, s = i % NS, sb = i & 1;
-            if (!mbar_wait(&sh.full[s], (i / NS) & 1u, &sh.abort_flag)) { ok = false; break; }
-            if (!mbar_wait(&sh.s_free[sb], ((i >> 1) & 1u) ^ 1u, &sh.abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t k_base = smem_u32(sh.kv[s]);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)
-              tc_mma_ss(tmem + sb * N, tc_desc(k_base + (kk >> 2) * (kTcTile * 128) + (kk & 3) * 32, 16, 1024),
-                        tc_desc(q_base + (kk >> 2) * (64 * 128) + (kk & 3) * 32, 16, 1024), idesc, kk > 0);
-            tc_commit(&sh.s_full[sb]);
-            if (n == ntiles - 1) tc_commit(&sh.q_empty);  // the query tile may be replaced
+        // Issue whichever product is ready: the P V product of the oldest tile that has its P^T
+        // (it releases a stage), else S^T of the next tile whose K/V has landed.  Both kinds run
+        // in tile order; S^T may lead by the two S buffers.
+        int nq = 0, np = 0;  // tiles of this segment whose S^T / P V product has been issued
+        bool o_ready = false;
+        uint32_t polls = 0;
+        while (np < ntiles) {
+          bool did = false;
+          if (np < nq) {
+            const int j = it + np, s = j % NS;
+            if (!o_ready) o_ready = (np > 0) || mbar_test(&sh.o_free, (seg & 1u) ^ 1u);
+            if (o_ready && mbar_test(&sh.p_full, j & 1u)) {
+              tc_fence_after();
+              const int ntok = min(kTcTile, tok_hi - (tok_lo + np * kTcTile));
+              const int ksteps = (ntok + 15) >> 4;
+              const uint32_t p_base = smem_u32(sh.kv[s]);  // [P_hi^T | P_lo^T] in the K tile's bytes
+              const uint32_t v_base = p_base + kTcTileBytes;
+              for (int kk = 0; kk < ksteps; ++kk)
+                tc_mma_ss(col_o, tc_desc(v_base + kk * 2048, kTcTile * 128, 1024),
+                          tc_desc(p_base + kk * 2048, 16384, 1024), idesc_pv, (np == 0 && kk == 0) ? 0u : 1u);
+              tc_commit(&sh.empty[s]);
+              tc_commit(&sh.pv_done);
+              ++np;
+              did = true;
+            }
           }
-          if (n > 0) {  // O^T += V^T P^T of tile it + n - 1
-            const int j = it + n - 1, s = j % NS;
-            if (n == 1 && !mbar_wait(&sh.o_free, (seg & 1u) ^ 1u, &sh.abort_flag)) { ok = false; break; }
-            if (!mbar_wait(&sh.p_full, j & 1u, &sh.abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const int ntok = min(kTcTile, tok_hi - (tok_lo + (n - 1) * kTcTile));
-            const int ksteps = (ntok + 15) >> 4;
-            const uint32_t p_base = smem_u32(sh.kv[s]);          // [P_hi^T | P_lo^T] in the K tile's bytes
-            const uint32_t v_base = p_base + kTcTileBytes;
-            for (int kk = 0; kk < ksteps; ++kk)
-              tc_mma_ss(col_o, tc_desc(v_base + kk * 2048, kTcTile * 128, 1024),
-                        tc_desc(p_base + kk * 2048, 16384, 1024), idesc_pv, (n == 1 && kk == 0) ? 0u : 1u);
-            tc_commit(&sh.empty[s]);
-            tc_commit(&sh.pv_done);
+          if (!did && nq < ntiles) {
+            const int i = it + nq, s = i % NS, sb = i & 1;
+            if (mbar_test(&sh.full[s], (i / NS) & 1u) && mbar_test(&sh.s_free[sb], ((i >> 1) & 1u) ^ 1u)) {
+              tc_fence_after();
+              const uint32_t k_base = smem_u32(sh.kv[s]);
+#pragma unroll
+              for (int kk = 0; kk < 8; ++kk)
+                tc_mma_ss(tmem + sb * N, tc_desc(k_base + (kk >> 2) * (kTcTile * 128) + (kk & 3) * 32, 16, 1024),
+                          tc_desc(q_base + (kk >> 2) * (64 * 128) + (kk & 3) * 32, 16, 1024), idesc, kk > 0);
+              tc_commit(&sh.s_full[sb]);
+              if (nq == ntiles - 1) tc_commit(&sh.q_empty);  // the query tile may be replaced
+              ++nq;
+              did = true;
+            }
+          }
+          if (did) {
+            polls = 0;
+          } else {
+            if (++polls > (1u << 22) || (polls > 64 && sh.abort_flag)) { ok = false; break; }
+            if (polls > 256) __nanosleep(32);
           }
         }
+        if (!ok) break;
         it += ntiles;
         ++seg;
         next_unit(a, u, seg_hi, ue);
@@ -563,24 +583,29 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         const bool tail_tile = P.tail && (t0 + kTcTile > c_list);
         // ---- pass 1: does any visible score exceed its row's reference maximum by 2^8? --------
         bool exceed = false;
+        uint32_t sv[NT][16];  // this key's scores against every query row
         if (!__any_sync(0xffffffffu, fail)) {
 #pragma unroll
+          for (int c = 0; c < NT; ++c) tc_ld16(sv[c], tmem + sb * N + lane_sel + c * 16);
+          tc_wait_ld();
+          if (!kKeepS) {  // the scores are read again in pass 2; until then the registers are free
+            tc_fence_before();
+          }
+#pragma unroll
           for (int c = 0; c < NT; ++c) {
-            uint32_t sv[16];
-            tc_ld16(sv, tmem + sb * N + lane_sel + c * 16);
             float mr[16];
             tc_lds16(mr, sh.m_ref + c * 16);
-            tc_wait_ld();
             if (!tail_tile) {
 #pragma unroll
               for (int j = 0; j < 16; ++j)
-                exceed |= !(fmaf(__uint_as_float(sv[j]), P.scale_log2, -mr[j]) <= kTcRaise);
+                exceed |= !(fmaf(__uint_as_float(sv[c][j]), P.scale_log2, -mr[j]) <= kTcRaise);
             } else {
               int lim[16];
               tc_lds16(lim, sh.row_lim + c * 16);
 #pragma unroll
               for (int j = 0; j < 16; ++j)
-                exceed |= ((jt < 0) | (jt <= lim[j])) & !(fmaf(__uint_as_float(sv[j]), P.scale_log2, -mr[j]) <= kTcRaise);
+                exceed |= ((jt < 0) | (jt <= lim[j])) &
+                          !(fmaf(__uint_as_float(sv[c][j]), P.scale_log2, -mr[j]) <= kTcRaise);
             }
           }
           exceed &= kvalid;
@@ -595,15 +620,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
               if (blk * 2 + c < NT) {
-                uint32_t sv[16];
-                tc_ld16(sv, tmem + sb * N + lane_sel + (blk * 2 + c) * 16);
                 int lim[16];
                 tc_lds16(lim, sh.row_lim + (blk * 2 + c) * 16);
-                tc_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                   const bool vis = kvalid & (!tail_tile | (jt < 0) | (jt <= lim[j]));
-                  v[c * 16 + j] = vis ? __uint_as_float(sv[j]) * P.scale_log2 : -INFINITY;
+                  v[c * 16 + j] = vis ? __uint_as_float(sv[blk * 2 + c][j]) * P.scale_log2 : -INFINITY;
                 }
               } else {
 #pragma unroll
@@ -651,21 +673,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         // ---- pass 2: P = exp2(S - m) as two bf16 terms, into the dead K tile ------------------
         if (!__any_sync(0xffffffffu, fail)) {
           const uint32_t pb = smem_u32(sh.kv[s]) + (key_lane >> 3) * 1024 + (key_lane & 7) * 128;
+          // every score of this tile is in registers: the S^T buffer may be overwritten
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.s_free[sb]);
 #pragma unroll
           for (int c = 0; c < NT; ++c) {
-            uint32_t sv[16];
-            tc_ld16(sv, tmem + sb * N + lane_sel + c * 16);
             float mr[16];
             tc_lds16(mr, sh.m_ref + c * 16);
-            tc_wait_ld();
-            if (c == NT - 1) {  // S^T buffer read for the last time
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(&sh.s_free[sb]);
-            }
             float p[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) p[j] = ex2(fmaf(__uint_as_float(sv[j]), P.scale_log2, -mr[j]));
+            for (int j = 0; j < 16; ++j) p[j] = ex2(fmaf(__uint_as_float(sv[c][j]), P.scale_log2, -mr[j]));
             if (tail_tile) {
               int lim[16];
               tc_lds16(lim, sh.row_lim + c * 16);
@@ -679,12 +697,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
             }
 #pragma unroll
             for (int g8 = 0; g8 < 2; ++g8) {
+              // P = P_hi + P_lo in bf16 on the integer / FMA pipes: P_hi keeps the upper 16 bits
+              // (truncation), P_lo is the exact remainder rounded to nearest (P >= 0, so adding
+              // half an ulp to the bit pattern rounds): |P - P_hi - P_lo| <= 2^-16 P, unbiased
               uint32_t hi[4], lo[4];
 #pragma unroll
               for (int e = 0; e < 4; ++e) {
-                const float x0 = p[g8 * 8 + 2 * e], x1 = p[g8 * 8 + 2 * e + 1];
-                hi[e] = pack_bf16(x0, x1);
-                lo[e] = pack_bf16(x0 - __uint_as_float(hi[e] << 16), x1 - __uint_as_float(hi[e] & 0xffff0000u));
+                const uint32_t b0 = __float_as_uint(p[g8 * 8 + 2 * e]), b1 = __float_as_uint(p[g8 * 8 + 2 * e + 1]);
+                hi[e] = __byte_perm(b0, b1, 0x7632);
+                const uint32_t d0 = __float_as_uint(__uint_as_float(b0) - __uint_as_float(b0 & 0xffff0000u)) + 0x8000u;
+                const uint32_t d1 = __float_as_uint(__uint_as_float(b1) - __uint_as_float(b1 & 0xffff0000u)) + 0x8000u;
+                lo[e] = __byte_perm(d0, d1, 0x7632);
               }
               // B operand [P_hi^T | P_lo^T]: 2N columns, 16-byte chunk ch of a key's row at
               // (ch / 8) * 16 KB + ((ch % 8) ^ (key % 8)) * 16
