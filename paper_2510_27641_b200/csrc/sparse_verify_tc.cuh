@@ -529,7 +529,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
             polls = 0;
           } else {
             if (++polls > (1u << 22) || (polls > 64 && sh.abort_flag)) { ok = false; break; }
-            if (polls > 256) __nanosleep(32);
+            __nanosleep(polls > 4096 ? 100 : 20);  // the issue slots belong to the softmax warp of this sub-partition
           }
         }
         if (!ok) break;
@@ -798,22 +798,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           };
 #pragma unroll 1
           for (int c = 0; c < NT; ++c) {
+            // one pass with a running maximum: the 48 loads of a contributor are independent,
+            // and two contributors are in flight at a time
             float mx[16], acc[16], ls[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) { mx[j] = -INFINITY; acc[j] = 0.f; ls[j] = 0.f; }
-            for (int i = i_lo; i <= i_hi; ++i) {
-              const float* r2 = rec_of(i) + N * kD + c * 16;
-#pragma unroll
-              for (int j = 0; j < 16; ++j) mx[j] = fmaxf(mx[j], __ldcg(r2 + j));
-            }
+#pragma unroll 2
             for (int i = i_lo; i <= i_hi; ++i) {
               const float* r2 = rec_of(i);
+              float mi[16], li[16], oi[16];
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
-                const float base = (mx[j] == -INFINITY) ? 0.f : mx[j];
-                const float w = ex2(__ldcg(r2 + N * kD + c * 16 + j) - base);
-                ls[j] += __ldcg(r2 + N * kD + N + c * 16 + j) * w;
-                acc[j] += __ldcg(r2 + (c * 16 + j) * kD + d) * w;
+                mi[j] = __ldcg(r2 + N * kD + c * 16 + j);
+                li[j] = __ldcg(r2 + N * kD + N + c * 16 + j);
+                oi[j] = __ldcg(r2 + (c * 16 + j) * kD + d);
+              }
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                float mn, ao, ai;
+                merge_scales(mx[j], mi[j], mn, ao, ai);
+                mx[j] = mn;
+                ls[j] = ls[j] * ao + li[j] * ai;
+                acc[j] = acc[j] * ao + oi[j] * ai;
               }
             }
 #pragma unroll
