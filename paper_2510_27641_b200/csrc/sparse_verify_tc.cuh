@@ -150,7 +150,7 @@ struct TcShared {
   alignas(8) unsigned long long full[kTcStages];
   unsigned long long empty[kTcStages];
   unsigned long long q_full, q_empty;
-  unsigned long long s_full[2], s_free[2], p_full, pv_done, o_free;
+  unsigned long long s_full[2], s_free[2], p_full[2], pv_done[2], o_free;
   uint32_t tmem_base;
   int raise_tile[2];   // tile index + 1 of the last tile (per S buffer) that must raise m_ref
   int last_arriver;
@@ -195,9 +195,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sh.s_full[i], 1);
       mbar_init(&sh.s_free[i], 4);
+      mbar_init(&sh.p_full[i], 4);
+      mbar_init(&sh.pv_done[i], 1);
     }
-    mbar_init(&sh.p_full, 4);
-    mbar_init(&sh.pv_done, 1);
     mbar_init(&sh.o_free, 4);
     mbar_fence_init();
     sh.abort_flag = 0;
@@ -495,7 +495,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           if (np < nq) {
             const int j = it + np, s = j % NS;
             if (!o_ready) o_ready = (np > 0) || mbar_test(&sh.o_free, (seg & 1u) ^ 1u);
-            if (o_ready && mbar_test(&sh.p_full, j & 1u)) {
+            // per tile parity, like the S buffers: the softmax warps can finish tile j + 1 before
+            // this thread looks, and one barrier would then be two phases ahead of the test
+            if (o_ready && mbar_test(&sh.p_full[j & 1], (j >> 1) & 1u)) {
               tc_fence_after();
               const int ntok = min(kTcTile, tok_hi - (tok_lo + np * kTcTile));
               const int ksteps = (ntok + 15) >> 4;
@@ -505,7 +507,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
                 tc_mma_ss(col_o, tc_desc(v_base + kk * 2048, kTcTile * 128, 1024),
                           tc_desc(p_base + kk * 2048, 16384, 1024), idesc_pv, (np == 0 && kk == 0) ? 0u : 1u);
               tc_commit(&sh.empty[s]);
-              tc_commit(&sh.pv_done);
+              tc_commit(&sh.pv_done[j & 1]);
               ++np;
               did = true;
             }
@@ -547,10 +549,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
     constexpr int kBar = 1;
     bool fail = false;
     int it = 0, seg = 0;
-    int pv_next = 0;  // next phase of pv_done not yet waited for (every phase is waited, in order)
+    // P V products whose completion this thread has seen: every tile is waited for, in order, on
+    // the barrier of its parity.  (One barrier for all tiles could complete two phases between
+    // two polls -- the product of a short last tile takes a few dozen nanoseconds -- and a
+    // parity wait cannot tell that from none.)
+    int pv_next = 0;
     auto pv_catch_up = [&](int upto) {
       while (pv_next <= upto) {
-        if (!mbar_wait(&sh.pv_done, pv_next & 1u, &sh.abort_flag)) { fail = true; return; }
+        if (!mbar_wait(&sh.pv_done[pv_next & 1], (pv_next >> 1) & 1u, &sh.abort_flag)) { fail = true; return; }
         ++pv_next;
       }
     };
@@ -718,7 +724,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           }
           fence_proxy_async();  // P^T is read by the tensor core through the async proxy
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sh.p_full);
+          if (lane == 0) mbar_arrive(&sh.p_full[sb]);
         }
         if (n > 0 && !fail) pv_catch_up(i - 1);
       }

@@ -202,3 +202,26 @@ def test_argument_errors():
         kv_off = kv_d.view(-1)[4:4 + 3 * 32768].view(3, 2, 16, 8, 128)
         sa.sparse_verify(q_d, kv_off, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d)
     assert e.value.code == -4
+
+
+def test_back_to_back_launches_with_many_segments_per_cta():
+    # 256 units of ~125 atoms: every CTA walks several units, launches overlap through programmatic
+    # stream serialization, and short last tiles make consecutive completion signals arrive within
+    # nanoseconds of each other -- the case in which a completion barrier must not be missed
+    import paper_2510_27641_b200 as sa
+    case = _make_case(60, 32, 8, 64, 8, 16, [2100] * 32, counts=[[2000]] * 32)
+    kv_d = case["kv"].to(dev())
+    q_d, len_d, bt_d = bf16_to_dev(case["q"]), to_dev(case["lens"]), to_dev(case["bt"])
+    idx_d, cnt_d = to_dev(case["idx"]), to_dev(case["cnt"])
+    out, lse, status = _run(case)
+    assert int(status.abs().sum()) == 0
+    o, l = torch.empty_like(out), torch.empty_like(lse)
+    st = torch.zeros_like(status)
+    args = sa.make_verify_args(q_d, kv_d, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d, out=o, lse=l)
+    ws = sa.verify_workspace(args)
+    for _ in range(100):
+        sa.sparse_verify(q_d, kv_d, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d, out=o, lse=l, status=st,
+                         workspace=ws, flags=_ENGINE["flags"])
+    torch.cuda.synchronize()
+    assert int(st.abs().sum()) == 0
+    assert torch.equal(o, out) and torch.equal(l, lse)
