@@ -4,6 +4,7 @@ a serving engine's pool may own the whole GPU).  Its scratch is a fixed array in
 library, so the test checks that two calls in a row -- the second one meeting whatever the
 first left in that array -- both reproduce the regular entry point's results."""
 import ctypes as C
+import gc
 
 import numpy as np
 import pytest
@@ -41,10 +42,16 @@ def test_static_scratch_entry_point_matches_the_regular_one_twice_in_a_row():
             status = torch.zeros_like(ref_status)
             args = sa.make_verify_args(q, kv, kv_len, block_table=bt, idx=idx, counts=cnt, out=out, lse=lse,
                                        status=status)          # no workspace: none is needed
-            before = torch.cuda.memory_allocated()
+            # nothing is allocated: neither through torch's caching allocator (its allocation
+            # counter stands still) nor from the driver (the device's free memory stands still)
+            gc.collect()
+            torch.cuda.synchronize()
+            n_alloc = torch.cuda.memory_stats()["allocation.all.allocated"]
+            free_before = torch.cuda.mem_get_info()[0]
             sa.sparse_verify_static(args)
             torch.cuda.synchronize()
-            assert torch.cuda.memory_allocated() == before
+            assert torch.cuda.memory_stats()["allocation.all.allocated"] == n_alloc
+            assert torch.cuda.mem_get_info()[0] == free_before
             assert float((out - ref_out).abs().max()) <= OUT_TOL, f"call {call}"
             assert lse_err(lse.cpu().numpy().astype(np.float64), ref_lse.cpu().numpy().astype(np.float64)) <= LSE_TOL
             assert torch.equal(status, ref_status)
