@@ -43,6 +43,8 @@ def lib() -> C.CDLL:
         _lib.specattn_oracle_aggregate.restype = C.c_int
         _lib.specattn_oracle_num_threads.restype = C.c_int
         _lib.specattn_oracle_select_topp.restype = None
+        _lib.specattn_oracle_bisect.restype = C.c_int64
+        _lib.specattn_oracle_select_variant.restype = None
         _lib.specattn_oracle_attend_rows.restype = None
         _lib.specattn_oracle_sparse_verify.restype = None
     return _lib
@@ -111,6 +113,45 @@ def select_topp(draft_probs, layer_map, kv_len, p, n_groups=1, head_group=None, 
     lib().specattn_oracle_select_topp(ptrs, n_d, _p(layer_map), len(layer_map), B, H, gamma, G,
                                       C.c_int64(Ls), _p(kv_len), _p(hg), C.c_float(p), _p(idx),
                                       C.c_int64(stride), _p(counts), _p(status), _p(diag))
+    return idx, counts, status, diag
+
+
+def bisect(a: np.ndarray, p: float, n_iters: int = 10, idx_cap: int | None = None):
+    """O2b for one row: Alg. 2's bisection with a fixed number of iterations.
+    Returns (idx[int32, ascending], count, diag dict)."""
+    a = _chk(a, np.float32)
+    L = a.shape[0]
+    cap = L if idx_cap is None else idx_cap
+    idx = np.full(max(cap, 1), -1, dtype=np.int32)
+    diag = np.zeros(6, dtype=np.float64)
+    n = int(lib().specattn_oracle_bisect(_p(a), L, C.c_float(p), int(n_iters), _p(idx), C.c_int64(cap), _p(diag)))
+    d = dict(total=diag[0], target=diag[1], kept_mass=diag[2], theta_mid=diag[3], margin=diag[4], max=diag[5])
+    return idx[:min(n, cap)].copy(), n, d
+
+
+def select_variant(draft_probs, layer_map, kv_len, p, *, per_step=False, n_iters=0, n_groups=1,
+                   head_group=None, idx_stride=None):
+    """O1+O2 over a step with Alg. 2's variants: per_step = one nucleus per speculated query,
+    unioned; n_iters >= 1 = literal bisection.  Same outputs as select_topp; diag[..., 4] is the
+    smallest margin over the rows of a list."""
+    n_d = len(draft_probs)
+    ref = next(x for x in draft_probs if x is not None)
+    B, H, gamma, Ls = ref.shape
+    arrs = [None if x is None else _chk(x, np.float32) for x in draft_probs]
+    ptrs = (C.c_void_p * n_d)(*[None if x is None else x.ctypes.data for x in arrs])
+    layer_map = _chk(layer_map, np.int32)
+    kv_len = _chk(kv_len, np.int32)
+    hg = None if head_group is None else _chk(head_group, np.int32)
+    G = n_groups
+    stride = int(Ls if idx_stride is None else idx_stride)
+    idx = np.full((n_d, B, G, max(stride, 1)), -1, dtype=np.int32)
+    counts = np.full((n_d, B, G), -1, dtype=np.int32)
+    status = np.full((n_d, B, G), -1, dtype=np.int32)
+    diag = np.zeros((n_d, B, G, 6), dtype=np.float64)
+    lib().specattn_oracle_select_variant(ptrs, n_d, _p(layer_map), len(layer_map), B, H, gamma, G,
+                                         C.c_int64(Ls), _p(kv_len), _p(hg), C.c_float(p),
+                                         int(bool(per_step)), int(n_iters), _p(idx), C.c_int64(stride),
+                                         _p(counts), _p(status), _p(diag))
     return idx, counts, status, diag
 
 

@@ -231,6 +231,156 @@ void specattn_oracle_select_topp(const float* const* draft_probs, int n_draft_la
 }
 
 // ---------------------------------------------------------------------------
+// O2b.  The bisection of Alg. 2 for one row, taken literally, with a fixed number of
+// iterations (the paper's implementation note: 10).
+//   total  = sum_i (double) a[i], index order; target = (double) p * total
+//   theta_high = max_i a[i], theta_low = 0          (binary32)
+//   repeat n_iters times:
+//     theta_mid = (theta_high + theta_low) / 2      (binary32)
+//     M_current = sum_{i : a[i] >= theta_mid} (double) a[i], index order
+//     M_current < target ? theta_high = theta_mid : theta_low = theta_mid
+//   kept = {i : a[i] >= theta_mid of the last iteration}, ascending.
+// Unlike O2 the result may fall short of the target mass (when the last midpoint lies above the
+// exact threshold) or keep more than the smallest set (when it lies below).
+//   p >= 1: every position is kept (the same rule as O2).  n_iters >= 1.
+//   diag[0..5] = total, target, mass of the kept set, theta_mid (last), margin, max
+//   margin = min over the iterations of |M_current - target| / total (1 when total == 0 or
+//            p >= 1): how far the nearest comparison was from flipping.
+// [Alg. 2, the loop over theta and "T_s <- {i : a_{s,i} >= theta_mid}"; footnote to Sec. 3.4]
+// ---------------------------------------------------------------------------
+int64_t specattn_oracle_bisect(const float* a, int L, float p, int n_iters, int32_t* idx,
+                               int64_t idx_cap, double* diag) {
+  double total = 0.0;
+  float vmax = 0.0f;
+  for (int i = 0; i < L; ++i) {
+    total += static_cast<double>(a[i]);
+    if (a[i] > vmax) vmax = a[i];
+  }
+  const double target = static_cast<double>(p) * total;
+  double margin = 1.0, kept_mass = total;
+  float theta_mid = 0.0f;
+  int64_t count = 0;
+  if (L > 0 && !(p >= 1.0f)) {
+    float theta_high = vmax, theta_low = 0.0f;
+    for (int it = 0; it < n_iters; ++it) {
+      theta_mid = (theta_high + theta_low) / 2.0f;
+      double m_current = 0.0;
+      for (int i = 0; i < L; ++i)
+        if (a[i] >= theta_mid) m_current += static_cast<double>(a[i]);
+      if (total > 0.0) margin = std::min(margin, std::fabs(m_current - target) / total);
+      if (m_current < target) theta_high = theta_mid; else theta_low = theta_mid;
+      kept_mass = m_current;
+    }
+  }
+  for (int i = 0; i < L; ++i) {
+    if (a[i] >= theta_mid) {
+      if (count < idx_cap) idx[count] = i;
+      ++count;
+    }
+  }
+  if (diag != nullptr) {
+    diag[0] = total;
+    diag[1] = target;
+    diag[2] = kept_mass;
+    diag[3] = static_cast<double>(theta_mid);
+    diag[4] = margin;
+    diag[5] = static_cast<double>(vmax);
+  }
+  return count;
+}
+
+// ---------------------------------------------------------------------------
+// O1 + O2 over a whole step with the selection variants of Alg. 2.
+//   per_step == 0: one row per list, aggregated over heads AND speculated queries (O1), one
+//                  nucleus -- specattn_oracle_select_topp when n_iters == 0.
+//   per_step == 1: Alg. 2 as printed: for every speculated query s the row
+//                  a_s[i] = sum over the group's heads h (ascending, binary32, from +0) of
+//                  A[h, s, i] gets its own nucleus T_s, and the list is the union of the T_s.
+//   n_iters == 0: exact nucleus (O2); n_iters >= 1: literal bisection (O2b).
+// Other arguments, truncation and status as in specattn_oracle_select_topp.
+//   diag [n_draft_layers, B, G, 6]: [4] = smallest margin over the rows of the list, the other
+//   entries are those of the last row processed.
+// [Alg. 2 "for s = 1 to gamma ... T <- T u T_s"]
+// ---------------------------------------------------------------------------
+void specattn_oracle_select_variant(const float* const* draft_probs, int n_draft_layers,
+                                    const int32_t* layer_map, int n_target_layers, int B,
+                                    int n_heads, int gamma, int G, int64_t L_stride,
+                                    const int32_t* kv_len, const int32_t* head_group, float p,
+                                    int per_step, int n_iters, int32_t* idx, int64_t idx_stride,
+                                    int32_t* counts, int32_t* status, double* diag) {
+  std::vector<char> used(n_draft_layers, 0);
+  for (int j = 0; j < n_target_layers; ++j)
+    if (layer_map[j] >= 0 && layer_map[j] < n_draft_layers) used[layer_map[j]] = 1;
+  const int64_t n_lists = static_cast<int64_t>(n_draft_layers) * B * G;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t li = 0; li < n_lists; ++li) {
+    const int u = static_cast<int>(li / (static_cast<int64_t>(B) * G));
+    const int b = static_cast<int>((li / G) % B);
+    const int g = static_cast<int>(li % G);
+    if (!used[u]) continue;
+    const int L = kv_len[b];
+    const float* A = draft_probs[u] + static_cast<int64_t>(b) * n_heads * gamma * L_stride;
+    std::vector<float> row(std::max(L, 1));
+    std::vector<int32_t> tmp(std::max(L, 1));
+    std::vector<char> in_set(std::max(L, 1), 0);
+    double dg[6] = {0, 0, 0, 0, 1.0, 0};
+    double min_margin = 1.0;
+    bool invalid = false;
+    const int n_rows = per_step ? gamma : 1;
+    for (int s = 0; s < n_rows && !invalid; ++s) {
+      int st;
+      if (per_step) {
+        // heads only: the row of speculated query s
+        st = ORACLE_OK;
+        for (int i = 0; i < L; ++i) {
+          float acc = 0.0f;
+          for (int h = 0; h < n_heads; ++h) {
+            if (head_group != nullptr && head_group[h] != g) continue;
+            const float x = A[(static_cast<int64_t>(h) * gamma + s) * L_stride + i];
+            if (!valid_prob(x)) st = ORACLE_INVALID_PROB;
+            acc = acc + x;
+          }
+          if (!(acc <= FLT_MAX)) st = ORACLE_INVALID_PROB;
+          row[i] = acc;
+        }
+      } else {
+        st = specattn_oracle_aggregate(A, n_heads, gamma, L_stride, L, head_group, g, row.data());
+      }
+      if (st == ORACLE_INVALID_PROB) {
+        invalid = true;
+        break;
+      }
+      const int64_t c = (n_iters > 0)
+                            ? specattn_oracle_bisect(row.data(), L, p, n_iters, tmp.data(), L, dg)
+                            : specattn_oracle_nucleus(row.data(), L, p, tmp.data(), L, dg);
+      min_margin = std::min(min_margin, dg[4]);
+      for (int64_t k = 0; k < c; ++k) in_set[tmp[k]] = 1;
+    }
+    // (an invalid probability in any contributing row voids the list: the loop stopped there)
+    double* out_dg = diag ? diag + li * 6 : nullptr;
+    if (invalid) {
+      counts[li] = 0;
+      status[li] = ORACLE_INVALID_PROB;
+      if (out_dg) for (int k = 0; k < 6; ++k) out_dg[k] = std::numeric_limits<double>::quiet_NaN();
+      continue;
+    }
+    int64_t c = 0;
+    int32_t* out = idx + li * idx_stride;
+    for (int i = 0; i < L; ++i)
+      if (in_set[i]) {
+        if (c < idx_stride) out[c] = i;
+        ++c;
+      }
+    counts[li] = static_cast<int32_t>(c);
+    status[li] = (c > idx_stride) ? ORACLE_OVERFLOW : ORACLE_OK;
+    if (out_dg) {
+      for (int k = 0; k < 6; ++k) out_dg[k] = dg[k];
+      out_dg[4] = min_margin;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // O3 core.  Softmax attention of M query rows over c gathered key/value rows.
 //   q  [M, d] bf16 bits, K and V [c, d] bf16 bits (row stride given in elements)
 //   s_i = (q . k_i) * scale ; m = max_i s_i ; l = sum_i exp(s_i - m)

@@ -441,3 +441,145 @@ def test_sparse_verify_causal_tail_matches_library_attention_per_query():
     o0, l0 = oracle.sparse_verify(q, kv, strides, bt, kv_len, idx, counts, n_kv_heads=Hkv, page_size=page)
     o1, l1 = oracle.sparse_verify(q, kv, strides, bt, kv_len, idx, counts, n_kv_heads=Hkv, page_size=page, tail_len=0)
     assert np.array_equal(o0, o1) and np.array_equal(l0, l1)
+
+
+# ---------------------------------------------------------------------------------------------
+# O2b: Alg. 2's bisection taken literally (fixed iterations), and the per-step union
+# ---------------------------------------------------------------------------------------------
+def _bisection_rows():
+    rows = []
+    for line in (Path(__file__).parent / "golden" / "bisection_worked_rows.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        p, k, vals, kept, theta = [x.strip() for x in line.split("|")]
+        rows.append((float(p), int(k), [float(v) for v in vals.split()], [int(v) for v in kept.split()], float(theta)))
+    return rows
+
+
+@pytest.mark.parametrize("p,k,vals,kept,theta", _bisection_rows())
+def test_bisection_worked_rows(p, k, vals, kept, theta):
+    idx, cnt, d = oracle.bisect(np.asarray(vals, np.float32), p, k)
+    assert idx.tolist() == kept and cnt == len(kept)
+    if p < 1.0:
+        assert d["theta_mid"] == theta
+
+
+def _rows_for_bisection(seed):
+    rng = np.random.default_rng(seed)
+    n = int(rng.integers(20, 4000))
+    kind = seed % 3
+    if kind == 0:
+        a = rng.random(n, dtype=np.float32) ** 3
+    elif kind == 1:
+        a = (1.0 / np.arange(1, n + 1) ** 1.1).astype(np.float32)[rng.permutation(n)]
+    else:
+        z = rng.standard_normal(n).astype(np.float32) * 4
+        a = np.exp(z - z.max()).astype(np.float32)
+    return (a / a.sum(dtype=np.float32)).astype(np.float32)
+
+
+@pytest.mark.parametrize("seed", range(9))
+def test_bisection_is_a_scalar_bisection_against_the_exact_threshold(seed):
+    # M(theta) = mass of {a >= theta} is non-increasing in theta, so "M(theta_mid) < target" holds
+    # exactly when theta_mid lies above the exact threshold theta* of the sorted-prefix definition:
+    # the literal loop must walk the same midpoints as a bisection that only knows theta* --
+    # derived here from numpy's sort, not from the oracle's loop.
+    a = _rows_for_bisection(400 + seed)
+    for p in (0.5, 0.9, 0.97):
+        order = np.argsort(-a, kind="stable")
+        csum = np.cumsum(a[order].astype(np.float64))
+        target = np.float64(np.float32(p)) * a.astype(np.float64).sum()
+        theta_star = a[order[int(np.searchsorted(csum, target, side="left"))]]
+        for k in (1, 3, 10, 30):
+            idx, cnt, d = oracle.bisect(a, p, k)
+            if d["margin"] < 1e-12:
+                continue
+            lo, hi, mid = np.float32(0), a.max(), np.float32(0)
+            for _ in range(k):
+                mid = np.float32((hi + lo) / np.float32(2))
+                if mid > theta_star:
+                    hi = mid
+                else:
+                    lo = mid
+            assert d["theta_mid"] == float(mid)
+            assert np.array_equal(idx, np.nonzero(a >= mid)[0])
+            # the bracket halves every iteration and always holds theta*
+            # (down to one binary32 spacing, where the midpoint stops moving)
+            assert abs(float(mid) - float(theta_star)) <= max(float(a.max()) * 2.0 ** (-k), float(np.spacing(mid))) * (1 + 1e-6)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_bisection_at_convergence_is_the_nucleus_with_or_without_its_threshold_ties(seed):
+    a = _rows_for_bisection(500 + seed)
+    for p in (0.6, 0.95):
+        nuc, _, dn = oracle.nucleus(a, p)
+        idx, _, d = oracle.bisect(a, p, 60)
+        if min(d["margin"], dn["margin"]) < 1e-12:
+            continue
+        theta = np.float32(dn["theta"])
+        assert np.array_equal(idx, nuc) or np.array_equal(idx, np.nonzero(a > theta)[0])
+        # short of the target by at most the mass tied at the threshold
+        assert d["kept_mass"] >= dn["m_gt"] - 1e-12
+
+
+def _numpy_nucleus(a, p):
+    order = np.argsort(-a, kind="stable")
+    csum = np.cumsum(a[order].astype(np.float64))
+    target = np.float64(np.float32(p)) * a.astype(np.float64).sum()
+    theta = a[order[int(np.searchsorted(csum, target, side="left"))]]
+    return np.nonzero(a >= theta)[0]
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_per_step_union_equals_the_union_of_per_row_nuclei(seed):
+    rng = np.random.default_rng(600 + seed)
+    B, H, gamma, L = 2, 3, 4, int(rng.integers(40, 900))
+    x = rng.random((B, H, gamma, L), dtype=np.float32) ** 4
+    x /= x.sum(axis=-1, keepdims=True)
+    x = x.astype(np.float32)
+    kv_len = np.array([L, max(1, L // 3)], np.int32)
+    p = 0.85
+    idx, cnt, st, dg = oracle.select_variant([x], [0], kv_len, p, per_step=True)
+    for b in range(B):
+        Lb = int(kv_len[b])
+        union = set()
+        sizes = []
+        for s in range(gamma):
+            row = np.zeros(Lb, np.float32)
+            for h in range(H):                      # heads ascending, binary32
+                row = (row + x[b, h, s, :Lb]).astype(np.float32)
+            kept = _numpy_nucleus(row, p)
+            sizes.append(len(kept))
+            union |= set(kept.tolist())
+        if dg[0, b, 0, 4] < 1e-12:
+            continue
+        assert st[0, b, 0] == 0
+        assert idx[0, b, 0, :cnt[0, b, 0]].tolist() == sorted(union)
+        assert max(sizes) <= cnt[0, b, 0] <= sum(sizes)
+
+
+def test_variant_special_cases():
+    rng = np.random.default_rng(7)
+    x = rng.random((1, 2, 1, 64), dtype=np.float32)
+    kv = np.array([64], np.int32)
+    # one speculated query: per-step selection is the aggregated selection
+    a = oracle.select_topp([x], [0], kv, 0.9)
+    b = oracle.select_variant([x], [0], kv, 0.9, per_step=True)
+    c = oracle.select_variant([x], [0], kv, 0.9, per_step=False)
+    for u, v in zip(a[:3], b[:3]):
+        assert np.array_equal(u, v)
+    for u, v in zip(a[:3], c[:3]):
+        assert np.array_equal(u, v)
+    # p >= 1 keeps everything in every variant; an invalid probability voids the list
+    for per_step in (False, True):
+        for it in (0, 10):
+            i, n, s, _ = oracle.select_variant([x], [0], kv, 1.0, per_step=per_step, n_iters=it)
+            assert n[0, 0, 0] == 64 and s[0, 0, 0] == 0
+    y = np.tile(x, (1, 1, 3, 1)).copy()
+    y[0, 1, 2, 5] = -0.25
+    for per_step in (False, True):
+        i, n, s, _ = oracle.select_variant([y], [0], kv, 0.9, per_step=per_step, n_iters=10)
+        assert n[0, 0, 0] == 0 and s[0, 0, 0] == 1
+    # truncation keeps the true count
+    i, n, s, _ = oracle.select_variant([x], [0], kv, 0.99, per_step=True, idx_stride=4)
+    assert n[0, 0, 0] > 4 and s[0, 0, 0] == 2 and np.all(np.diff(i[0, 0, 0]) > 0)
