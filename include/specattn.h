@@ -83,6 +83,17 @@ extern "C" {
  *   diag    optional double [.., 4] = {total, target, mass strictly above theta,
  *           mass of the kept set}; NULL to skip.
  *
+ * Variants of Alg. 2 (both off by default; results differ from the exact nucleus by design):
+ *   per_step = 1: Alg. 2 as printed -- every speculated query s gets its own row
+ *       a_s[i] = +0 + sum over heads h feeding g (ascending) of draft_probs[u][b, h, s, i], its
+ *       own threshold, and the list is the ascending union of the gamma sets.
+ *   bisect_iters = n in [1, 64]: the threshold of a row is the LAST midpoint of n bisection
+ *       steps (theta_high = max of the row, theta_low = 0, theta_mid = (high + low) / 2 in
+ *       binary32; mass of {a >= theta_mid} < target lowers theta_high, otherwise raises
+ *       theta_low) -- the paper's implementation uses n = 10.  The set {a >= theta_mid} may fall
+ *       short of the target mass or exceed the smallest set.  p >= 1 and all-zero rows still
+ *       keep every position.  diag then describes the exact threshold of the last row searched.
+ *
  * Requirements: 1 <= n_draft_layers <= 64; n_draft_heads <= 256; gamma >= 1; L_stride a
  * multiple of 4 and <= SPECATTN_MAX_KV_LEN; every draft_probs[u] 16-byte aligned;
  * 0 <= kv_len[b] <= L_stride (larger values are clamped); 0 < p (NaN rejected);
@@ -112,6 +123,8 @@ typedef struct specattn_select_args {
   int32_t* counts;
   int32_t* row_status;
   double* diag;
+  int32_t per_step;     /* 0 | 1 */
+  int32_t bisect_iters; /* 0 = exact threshold, else 1..64 */
 } specattn_select_args;
 
 int specattn_select_topp(const specattn_select_args* args, void* cuda_stream);

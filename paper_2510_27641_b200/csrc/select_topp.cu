@@ -78,6 +78,8 @@ struct SelectParams {
   int* status;
   double* diag;
   int single_row;  // every list has exactly one contributing row: read it in place
+  int per_step;    // Alg. 2 as printed: one nucleus per speculated query, unioned
+  int bisect_iters;  // > 0: the threshold is the last midpoint of that many bisection steps
 };
 
 // A histogram of exact mantissa sums, kept as two 32-bit words: `lo` sums the low 16 mantissa
@@ -97,6 +99,8 @@ struct Shared {
   int warp_cnt[kWarps];
   int n_rows;
   int n_invalid;            // threads of this CTA that met an invalid input
+  float warp_max[kWarps];   // largest aggregated value seen by each warp (literal bisection only)
+  float cta_max;            // read by the other CTAs of the cluster
   int local_kept;           // read by the other CTAs of the cluster
   // result of a scan (written by warp 0)
   int found_bin;
@@ -245,7 +249,9 @@ __device__ void scan_bins(Shared& sh, const double* mass, int nbins, double carr
   __syncthreads();
 }
 
-template <bool kInPlace>
+// kVariant: the selection variants of Alg. 2 (per-step union, fixed-iteration bisection); the
+// default instantiation contains none of their code.
+template <bool kInPlace, bool kVariant>
 __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel(const __grid_constant__ SelectParams P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
@@ -274,20 +280,6 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   const int hi = min(L, lo + per);
   const int n_loc = hi - lo;
 
-  // contributing rows in the order that defines the aggregated value
-  if (tid == 0) {
-    int n = 0;
-    for (int h = 0; h < P.H; ++h) {
-      if (P.has_groups && P.head_group[h] != g) continue;
-      for (int s = 0; s < P.gamma; ++s) sh.row_off[n++] = static_cast<long long>(h * P.gamma + s) * P.L_stride;
-    }
-    sh.n_rows = n;
-    sh.n_invalid = 0;
-  }
-  for (int i = tid; i < kL1Bins; i += kThreads) sh.h_hi[i] = sh.h_lo[i] = 0u;
-  __syncthreads();
-  const int R = sh.n_rows;
-
   // dynamic shared memory behind the fixed part
   const int slice_cap = kInPlace ? 0 : static_cast<int>(((((P.L_stride + cs - 1) / cs + 3) & ~3ll) + 31) & ~31ll);
   float* ring = a + slice_cap;
@@ -295,7 +287,6 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   unsigned int* const lvl_base = reinterpret_cast<unsigned int*>(ring + 4096);  // 2 levels x (lo, hi) x 1024
   const Hist h1 = {sh.h_lo, sh.h_hi};
 
-  // ---- 1+2: aggregate the slice and build the level-1 histogram ------------------------------
   const float* A = P.probs[slot] + static_cast<long long>(b) * P.H * P.gamma * P.L_stride + lo;
   constexpr bool in_place = kInPlace;
   // bit pattern of aggregated position i of the slice (-0.0 reads as +0.0)
@@ -305,6 +296,34 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   const int n4 = (n_loc + 3) >> 2;
   const int n_pos4 = n4 * 4;                       // slice length rounded up to whole float4s
   const int n_chunks = (n_pos4 + kChunk - 1) / kChunk;
+  // Alg. 2 as printed selects per speculated query and unions the sets: then everything up to
+  // the threshold runs once per query over the row summed over heads only, and the kept
+  // positions are collected in a bit mask of the slice.
+  const int n_steps = (kVariant && P.per_step) ? P.gamma : 1;
+  unsigned int theta_key = 0u;  // keep everything with key >= theta_key
+  double total = 0.0, target = 0.0, m_gt = 0.0, m_ge = 0.0;
+  bool invalid = false;
+  if (tid == 0) sh.n_invalid = 0;
+  for (int step = 0; step < n_steps; ++step) {
+  // contributing rows in the order that defines the aggregated value
+  if (tid == 0) {
+    int n = 0;
+    for (int h = 0; h < P.H; ++h) {
+      if (P.has_groups && P.head_group[h] != g) continue;
+      if (kVariant && P.per_step) {
+        sh.row_off[n++] = static_cast<long long>(h * P.gamma + step) * P.L_stride;
+      } else {
+        for (int s = 0; s < P.gamma; ++s) sh.row_off[n++] = static_cast<long long>(h * P.gamma + s) * P.L_stride;
+      }
+    }
+    sh.n_rows = n;
+  }
+  for (int i = tid; i < kL1Bins; i += kThreads) sh.h_hi[i] = sh.h_lo[i] = 0u;
+  __syncthreads();
+  const int R = sh.n_rows;
+  float vmax = 0.f;  // largest aggregated value of this thread's positions (literal bisection)
+
+  // ---- 1+2: aggregate the slice and build the level-1 histogram ------------------------------
   bool bad = false;
   if (in_place) {
     // single contributing row: one pass over the slice for validity and the level-1 histogram
@@ -322,6 +341,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
                !(v.z >= 0.f && v.z <= FLT_MAX) | !(v.w >= 0.f && v.w <= FLT_MAX);
       }
       const float vals[4] = {v.x + 0.f, v.y + 0.f, v.z + 0.f, v.w + 0.f};
+      if (kVariant) vmax = fmaxf(vmax, fmaxf(fmaxf(vals[0], vals[1]), fmaxf(vals[2], vals[3])));
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const unsigned int key = __float_as_uint(vals[e]);
@@ -403,6 +423,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
           bad |= !(v.x <= FLT_MAX) | !(v.y <= FLT_MAX) | !(v.z <= FLT_MAX) | !(v.w <= FLT_MAX);
         }
         const float vals[4] = {v.x, v.y, v.z, v.w};
+        if (kVariant && act) vmax = fmaxf(vmax, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const unsigned int key = __float_as_uint(vals[e]);
@@ -416,7 +437,17 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     asm volatile("cp.async.wait_group 0;" ::: "memory");
   }
   if (bad) atomicAdd(&sh.n_invalid, 1);
+  if (kVariant) {
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) vmax = fmaxf(vmax, __shfl_xor_sync(kFull, vmax, o));
+    if (lane == 0) sh.warp_max[warp] = vmax;
+  }
   __syncthreads();
+  if (kVariant && tid == 0) {
+    float m = 0.f;
+    for (int w = 0; w < kWarps; ++w) m = fmaxf(m, sh.warp_max[w]);
+    sh.cta_max = m;
+  }
   // the ring is idle from here on: zero this CTA's level-2 and level-3 histograms
   for (int i = tid; i < 2 * 2 * kL23Bins; i += kThreads) lvl_base[i] = 0u;
   __syncthreads();
@@ -426,9 +457,8 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   int n_bad = 0;
   for (int r = 0; r < cs; ++r) n_bad += *cluster.map_shared_rank(&sh.n_invalid, r);
 
-  unsigned int theta_key = 0u;  // keep everything with key >= theta_key
-  double total = 0.0, target = 0.0, m_gt = 0.0, m_ge = 0.0;
-  const bool invalid = n_bad != 0;
+  theta_key = 0u;
+  invalid = n_bad != 0;  // the count only grows from step to step: the last one decides
   bool searching = !invalid;
   if (searching) {
     // level 1: every CTA reduces its own range of bins over the cluster, then all gather
@@ -502,17 +532,53 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     m_gt = sh.mass_above;
     m_ge = sh.mass_ge;
   }
+  if (kVariant) {
+    if (searching && P.bisect_iters > 0) {
+      // Alg. 2's loop, literally: theta_high = max, theta_low = 0, n midpoints in binary32.  The
+      // mass of {a >= theta} does not grow with theta, so "mass(theta_mid) < target" holds
+      // exactly when theta_mid lies above the exact threshold found above: the midpoints are
+      // those of the printed loop without another pass over the row.
+      float th_hi = 0.f, th_lo = 0.f, th_mid = 0.f;
+      for (int r = 0; r < cs; ++r) th_hi = fmaxf(th_hi, *cluster.map_shared_rank(&sh.cta_max, r));
+      for (int it = 0; it < P.bisect_iters; ++it) {
+        th_mid = __fmul_rn(__fadd_rn(th_hi, th_lo), 0.5f);
+        if (__float_as_uint(th_mid) > theta_key) th_hi = th_mid; else th_lo = th_mid;
+      }
+      theta_key = __float_as_uint(th_mid);
+    }
+    if (P.per_step) {
+      // collect this query's set in the mask: a warp owns whole 32-position words
+      unsigned int* mask = reinterpret_cast<unsigned int*>(ring + kRingFloats);
+      const int chunk_m = (((n_loc + kWarps - 1) / kWarps) + 31) & ~31;
+      const int m_lo = min(n_loc, warp * chunk_m), m_hi = min(n_loc, m_lo + chunk_m);
+      for (int i0 = m_lo; i0 < m_hi; i0 += 32) {
+        const int i = i0 + lane;
+        const bool keep = !invalid && i < m_hi && key_at(i) >= theta_key;
+        const unsigned int m = __ballot_sync(kFull, keep);
+        if (lane == 0) mask[i0 >> 5] = (step == 0) ? m : (mask[i0 >> 5] | m);
+      }
+      // the next query's row overwrites the slice and the staging ring, which peers may still
+      // be reading (their scans of this CTA's last histogram)
+      cluster.sync();
+    }
+  }
+  }  // for step
 
   // ---- 4: ordered compaction --------------------------------------------------------------------
   // per-warp contiguous chunks of the slice, 32 positions per step
   const int chunk = (((n_loc + kWarps - 1) / kWarps) + 31) & ~31;
   const int w_lo = min(n_loc, warp * chunk);
   const int w_hi = min(n_loc, w_lo + chunk);
+  const unsigned int* const kept_mask = reinterpret_cast<const unsigned int*>(ring + kRingFloats);
+  auto kept = [&](int i) -> bool {
+    if (kVariant && P.per_step) return (kept_mask[i >> 5] >> (i & 31)) & 1u;
+    return key_at(i) >= theta_key;
+  };
   int wc = 0;
   if (!invalid) {
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
       const int i = i0 + lane;
-      const bool keep = i < w_hi && key_at(i) >= theta_key;
+      const bool keep = i < w_hi && kept(i);
       wc += __popc(__ballot_sync(kFull, keep));
     }
   }
@@ -539,7 +605,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     long long pos = offset + sh.warp_cnt[warp];
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
       const int i = i0 + lane;
-      const bool keep = i < w_hi && key_at(i) >= theta_key;
+      const bool keep = i < w_hi && kept(i);
       const unsigned m = __ballot_sync(kFull, keep);
       const long long my = pos + __popc(m & ((1u << lane) - 1u));
       if (keep && my < P.idx_stride) out[my] = lo + i;
@@ -590,6 +656,7 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   if (A.n_draft_heads < 1 || A.n_draft_heads > SPECATTN_MAX_DRAFT_HEADS) return SPECATTN_ERR_RANGE;
   if (A.L_stride < 0 || A.idx_stride < 0) return SPECATTN_ERR_RANGE;
   if (!(A.p > 0.0f)) return SPECATTN_ERR_RANGE;  // also rejects NaN
+  if (A.bisect_iters < 0 || A.bisect_iters > 64 || (A.per_step != 0 && A.per_step != 1)) return SPECATTN_ERR_RANGE;
   if (A.L_stride % 4 != 0) return SPECATTN_ERR_ALIGN;
   if (A.L_stride > SPECATTN_MAX_KV_LEN) return SPECATTN_ERR_UNSUPPORTED;
   if (static_cast<long long>(A.n_draft_heads) * A.gamma > SPECATTN_MAX_ROWS_PER_LIST)
@@ -642,6 +709,9 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   // single-row lists are read in place once the rows are long enough for the extra CTAs per
   // SM to pay for re-reading them from L2 (measured cross-over between 8k and 64k positions)
   P.single_row = (static_cast<long long>(A.n_draft_heads) * A.gamma == 1 && A.L_stride >= 32768) ? 1 : 0;
+  P.per_step = (A.per_step && A.gamma > 1) ? 1 : 0;  // with one query the union is the single nucleus
+  P.bisect_iters = A.bisect_iters;
+  const bool variant = P.per_step || P.bisect_iters > 0;
   const int cs = specattn::pick_cluster(A.L_stride, n_lists);
   const long long slice = P.single_row ? 0 : (((A.L_stride + cs - 1) / cs) + 3) / 4 * 4;
   if (slice > specattn::kSliceCap) return SPECATTN_ERR_UNSUPPORTED;
@@ -652,7 +722,8 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   const size_t slice_bytes = static_cast<size_t>((slice + 31) / 32 * 32) * sizeof(float);
   // (a single-row list keeps nothing but the 32 KB of scan arrays behind the fixed part)
   const size_t smem = fixed + slice_bytes +
-                      (P.single_row ? static_cast<size_t>(32 * 1024) : static_cast<size_t>(specattn::kRingFloats) * sizeof(float));
+                      (P.single_row ? static_cast<size_t>(32 * 1024) : static_cast<size_t>(specattn::kRingFloats) * sizeof(float)) +
+                      (P.per_step ? static_cast<size_t>(specattn::kSliceCap / 8) : 0);  // the union's bit mask
   if (smem > 224 * 1024) return SPECATTN_ERR_UNSUPPORTED;
 
   // Opt in to large dynamic shared memory once per device, so that later calls issue nothing
@@ -663,11 +734,17 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPECATTN_ERR_CUDA;
     if (!((done_mask.load(std::memory_order_acquire) >> dev) & 1ull)) {
-      err = cudaFuncSetAttribute(specattn::select_topp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 224 * 1024);
+      err = cudaFuncSetAttribute(specattn::select_topp_kernel<false, false>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
       if (err == cudaSuccess)
-        err = cudaFuncSetAttribute(specattn::select_topp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   224 * 1024);
+        err = cudaFuncSetAttribute(specattn::select_topp_kernel<true, false>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+      if (err == cudaSuccess)
+        err = cudaFuncSetAttribute(specattn::select_topp_kernel<false, true>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
+      if (err == cudaSuccess)
+        err = cudaFuncSetAttribute(specattn::select_topp_kernel<true, true>,
+                                   cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024);
       if (err != cudaSuccess) {
         cudaGetLastError();
         return SPECATTN_ERR_CUDA;
@@ -689,8 +766,12 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  err = P.single_row ? cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<true>, P)
-                     : cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<false>, P);
+  if (variant)
+    err = P.single_row ? cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<true, true>, P)
+                       : cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<false, true>, P);
+  else
+    err = P.single_row ? cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<true, false>, P)
+                       : cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<false, false>, P);
   if (err != cudaSuccess) {
     cudaGetLastError();
     return SPECATTN_ERR_CUDA;

@@ -179,3 +179,74 @@ def test_argument_errors_are_synchronous_and_launch_nothing():
     n = int(a[1][0, 0, 0])
     assert torch.equal(a[0][0, 0, 0, :n], b[0][0, 0, 0, :n])
     assert sa.kernel_launch_count() == before + 2
+
+
+# ---------------------------------------------------------------------------------------------
+# Alg. 2's variants: one nucleus per speculated query, unioned; fixed-iteration bisection
+# ---------------------------------------------------------------------------------------------
+def _compare_variant(gi, gc, gs, oi, oc, os_, od):
+    """Lists must equal the oracle's bit for bit unless one of the oracle's comparisons was
+    within NEAR of flipping (a binary64 sum in another order may then decide otherwise)."""
+    from gpu_util import NEAR
+    gi, gc, gs = gi.cpu().numpy(), gc.cpu().numpy(), gs.cpu().numpy()
+    n = near = 0
+    for i in np.ndindex(oc.shape):
+        if oc[i] < 0:
+            assert gc[i] == -1
+            continue
+        n += 1
+        assert gs[i] == os_[i]
+        k = min(int(oc[i]), oi.shape[-1])
+        if gc[i] == oc[i] and np.array_equal(gi[i][:k], oi[i][:k]):
+            continue
+        assert od[i][4] <= NEAR, f"list {i}: count {gc[i]} vs oracle {oc[i]}, margin {od[i][4]:.3e}"
+        near += 1
+    assert near <= max(1, n // 20)
+    return n
+
+
+@pytest.mark.parametrize("per_step,iters", [(True, 0), (False, 10), (True, 10), (False, 3), (True, 1), (False, 40)])
+def test_selection_variants_match_oracle(per_step, iters):
+    import paper_2510_27641_b200 as sa
+    # (a) ragged lengths, two draft layers, per-group head sets; (b) rows that span a cluster
+    cases = [(3, 8, 5, 4096, np.array([4096, 1000, 2731], np.int32), 2),
+             (2, 3, 4, 40000, np.array([40000, 33333], np.int32), 1)]
+    for B, H, gamma, Ls, kv_len, G in cases:
+        probs = [wl.draft_probs(11, u, kv_len, H, gamma, Ls, sink=6.0, slope=0.004) for u in range(2)]
+        hg = None if G == 1 else (np.arange(H) * G // H).astype(np.int32)
+        for p in (0.8, 0.95):
+            gi, gc, gs, _ = sa.select_topp([to_dev(x) for x in probs], to_dev(kv_len), [0, 1, 1], p, n_groups=G,
+                                           head_group=None if hg is None else hg.tolist(),
+                                           per_step=per_step, bisect_iters=iters)
+            torch.cuda.synchronize()
+            oi, oc, os_, od = oracle.select_variant(probs, [0, 1, 1], kv_len, p, per_step=per_step, n_iters=iters,
+                                                    n_groups=G, head_group=hg)
+            assert _compare_variant(gi, gc, gs, oi, oc, os_, od) == 2 * B * G
+
+
+def test_selection_variants_special_cases():
+    import paper_2510_27641_b200 as sa
+    kv = np.array([3000, 17], np.int32)
+    probs = wl.draft_probs(12, 0, kv, 4, 3, 3008, sink=6.0, slope=0.004)
+    d = to_dev(probs)
+    # p >= 1 keeps everything whatever the variant
+    for per_step, iters in ((True, 0), (False, 10), (True, 10)):
+        gi, gc, gs, _ = sa.select_topp([d], to_dev(kv), [0], 1.0, per_step=per_step, bisect_iters=iters)
+        assert gc.cpu().numpy().reshape(-1).tolist() == [3000, 17] and int(gs.abs().sum()) == 0
+    # a negative probability in any query's row voids the list in the per-step variant too
+    bad = probs.copy()
+    bad[0, 2, 1, 77] = -1e-3
+    gi, gc, gs, _ = sa.select_topp([to_dev(bad)], to_dev(kv), [0], 0.9, per_step=True, bisect_iters=10)
+    oi, oc, os_, od = oracle.select_variant([bad], [0], kv, 0.9, per_step=True, n_iters=10)
+    assert gs.cpu().numpy().reshape(-1).tolist() == os_.reshape(-1).tolist() == [sa.ROW_INVALID_PROB, 0]
+    assert gc.cpu().numpy().reshape(-1).tolist() == oc.reshape(-1).tolist()
+    # a single long row (read in place) with the literal bisection
+    row = wl.topp_rows("zipf", 2, 65536, 3).reshape(2, 1, 1, 65536)
+    kv1 = np.array([65536, 50001], np.int32)
+    gi, gc, gs, _ = sa.select_topp([to_dev(row)], to_dev(kv1), [0], 0.9, bisect_iters=10)
+    oi, oc, os_, od = oracle.select_variant([row], [0], kv1, 0.9, n_iters=10)
+    _compare_variant(gi, gc, gs, oi, oc, os_, od)
+    # out-of-range variant arguments are refused synchronously
+    a, keep = sa.make_select_args([d], to_dev(kv), [0], 0.9, idx=gi.new_zeros((1, 2, 1, 8)), counts=gc.new_zeros((1, 2, 1)),
+                                  row_status=gs.new_zeros((1, 2, 1)), bisect_iters=65)
+    assert sa.lib().specattn_select_topp(C.byref(a), None) == -3
