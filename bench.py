@@ -335,6 +335,34 @@ def topp_sweep(dev, reps=5):
     return out
 
 
+def select_variants(step, cfg, reps=5):
+    """The selection variants of Alg. 2 on the step's own draft rows (separate output buffers):
+    device time per launch and mean kept count, beside the default (aggregate, exact)."""
+    import torch
+    import paper_2510_27641_b200 as sa
+    out = {}
+    idx = torch.empty_like(step.idx)
+    for name, kw in (("aggregate_exact", {}), ("per_step_union_exact", dict(per_step=True)),
+                     ("aggregate_bisect10", dict(bisect_iters=10)),
+                     ("per_step_union_bisect10", dict(per_step=True, bisect_iters=10))):
+        counts = torch.full_like(step.counts, -1)
+        status = torch.full_like(step.row_status, -1)
+        f = lambda: sa.select_topp(step.draft_probs, step.kv_len, step.layer_map, cfg.p, idx=idx, counts=counts,
+                                   row_status=status, **kw)
+        for _ in range(2):
+            f()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            f()
+        e1.record()
+        torch.cuda.synchronize()
+        c = counts.cpu().numpy()
+        out[name] = {"us": round(e0.elapsed_time(e1) * 1e3 / reps, 1), "kept_mean": round(float(c[c >= 0].mean()), 1)}
+    return out
+
+
 def verify_micro(dev, reps=10, flags=0):
     """sparse_verify alone on synthetic shapes: dense long context and sparse lists of several
     lengths (shuffled block table, page 16).  Returns {case: {us, gbs}}; bytes = K/V rows read."""
@@ -523,6 +551,8 @@ def main():
                       "kv_touched_fraction": round(kv_bytes_step / dense_kv_step, 5),
                       "sequences_per_s": round(cfg.batch * world / us_step * 1e6, 1)}}
 
+    if rank == 0:
+        line["extra"]["select_variants"] = select_variants(step, cfg_r)
     if rank == 0 and not args.no_cpu_baseline:
         smp = OracleSample(cfg_r, si, n_attn_layers=8, pools=pools)
         us_cpu, sample = smp.step_us()
