@@ -129,10 +129,11 @@ def bisect(a: np.ndarray, p: float, n_iters: int = 10, idx_cap: int | None = Non
     return idx[:min(n, cap)].copy(), n, d
 
 
-def select_variant(draft_probs, layer_map, kv_len, p, *, per_step=False, n_iters=0, n_groups=1,
+def select_variant(draft_probs, layer_map, kv_len, p, *, per_step=False, n_iters=0, chunk=1, n_groups=1,
                    head_group=None, idx_stride=None):
     """O1+O2 over a step with Alg. 2's variants: per_step = one nucleus per speculated query,
-    unioned; n_iters >= 1 = literal bisection.  Same outputs as select_topp; diag[..., 4] is the
+    unioned; n_iters >= 1 = literal bisection; chunk > 1 = selection over per-chunk sums, kept
+    chunks keep all their positions.  Same outputs as select_topp; diag[..., 4] is the
     smallest margin over the rows of a list."""
     n_d = len(draft_probs)
     ref = next(x for x in draft_probs if x is not None)
@@ -150,7 +151,7 @@ def select_variant(draft_probs, layer_map, kv_len, p, *, per_step=False, n_iters
     diag = np.zeros((n_d, B, G, 6), dtype=np.float64)
     lib().specattn_oracle_select_variant(ptrs, n_d, _p(layer_map), len(layer_map), B, H, gamma, G,
                                          C.c_int64(Ls), _p(kv_len), _p(hg), C.c_float(p),
-                                         int(bool(per_step)), int(n_iters), _p(idx), C.c_int64(stride),
+                                         int(bool(per_step)), int(n_iters), int(chunk), _p(idx), C.c_int64(stride),
                                          _p(counts), _p(status), _p(diag))
     return idx, counts, status, diag
 

@@ -297,6 +297,10 @@ int64_t specattn_oracle_bisect(const float* a, int L, float p, int n_iters, int3
 //                  a_s[i] = sum over the group's heads h (ascending, binary32, from +0) of
 //                  A[h, s, i] gets its own nucleus T_s, and the list is the union of the T_s.
 //   n_iters == 0: exact nucleus (O2); n_iters >= 1: literal bisection (O2b).
+//   chunk > 1:    selection at chunk granularity (Sec. 4: "chunk size ... 16"): the row that
+//                 is searched holds one score per chunk of `chunk` consecutive positions, the
+//                 binary32 sum of the chunk's values in ascending order; kept chunks keep all
+//                 their positions.  chunk == 1 is per-position selection.
 // Other arguments, truncation and status as in specattn_oracle_select_topp.
 //   diag [n_draft_layers, B, G, 6]: [4] = smallest margin over the rows of the list, the other
 //   entries are those of the last row processed.
@@ -306,8 +310,9 @@ void specattn_oracle_select_variant(const float* const* draft_probs, int n_draft
                                     const int32_t* layer_map, int n_target_layers, int B,
                                     int n_heads, int gamma, int G, int64_t L_stride,
                                     const int32_t* kv_len, const int32_t* head_group, float p,
-                                    int per_step, int n_iters, int32_t* idx, int64_t idx_stride,
-                                    int32_t* counts, int32_t* status, double* diag) {
+                                    int per_step, int n_iters, int chunk, int32_t* idx,
+                                    int64_t idx_stride, int32_t* counts, int32_t* status,
+                                    double* diag) {
   std::vector<char> used(n_draft_layers, 0);
   for (int j = 0; j < n_target_layers; ++j)
     if (layer_map[j] >= 0 && layer_map[j] < n_draft_layers) used[layer_map[j]] = 1;
@@ -322,6 +327,7 @@ void specattn_oracle_select_variant(const float* const* draft_probs, int n_draft
     const float* A = draft_probs[u] + static_cast<int64_t>(b) * n_heads * gamma * L_stride;
     std::vector<float> row(std::max(L, 1));
     std::vector<int32_t> tmp(std::max(L, 1));
+    std::vector<float> score(std::max(L, 1));
     std::vector<char> in_set(std::max(L, 1), 0);
     double dg[6] = {0, 0, 0, 0, 1.0, 0};
     double min_margin = 1.0;
@@ -350,11 +356,31 @@ void specattn_oracle_select_variant(const float* const* draft_probs, int n_draft
         invalid = true;
         break;
       }
+      // chunk > 1: the selection runs over chunk scores, score_j = +0 + a[j*chunk] + a[j*chunk+1]
+      // + ... (binary32, ascending, the last chunk cut at L), and a kept chunk keeps all its
+      // positions
+      const int n_sel = (chunk > 1) ? (L + chunk - 1) / chunk : L;
+      if (chunk > 1) {
+        for (int j = 0; j < n_sel; ++j) {
+          float acc = 0.0f;
+          for (int i = j * chunk; i < std::min(L, (j + 1) * chunk); ++i) acc = acc + row[i];
+          if (!(acc <= FLT_MAX)) invalid = true;
+          score[j] = acc;
+        }
+        if (invalid) break;
+      }
+      const float* sel = (chunk > 1) ? score.data() : row.data();
       const int64_t c = (n_iters > 0)
-                            ? specattn_oracle_bisect(row.data(), L, p, n_iters, tmp.data(), L, dg)
-                            : specattn_oracle_nucleus(row.data(), L, p, tmp.data(), L, dg);
+                            ? specattn_oracle_bisect(sel, n_sel, p, n_iters, tmp.data(), n_sel, dg)
+                            : specattn_oracle_nucleus(sel, n_sel, p, tmp.data(), n_sel, dg);
       min_margin = std::min(min_margin, dg[4]);
-      for (int64_t k = 0; k < c; ++k) in_set[tmp[k]] = 1;
+      for (int64_t k = 0; k < c; ++k) {
+        if (chunk > 1) {
+          for (int i = tmp[k] * chunk; i < std::min(L, (tmp[k] + 1) * chunk); ++i) in_set[i] = 1;
+        } else {
+          in_set[tmp[k]] = 1;
+        }
+      }
     }
     // (an invalid probability in any contributing row voids the list: the loop stopped there)
     double* out_dg = diag ? diag + li * 6 : nullptr;

@@ -583,3 +583,73 @@ def test_variant_special_cases():
     # truncation keeps the true count
     i, n, s, _ = oracle.select_variant([x], [0], kv, 0.99, per_step=True, idx_stride=4)
     assert n[0, 0, 0] > 4 and s[0, 0, 0] == 2 and np.all(np.diff(i[0, 0, 0]) > 0)
+
+
+# ---------------------------------------------------------------------------------------------
+# selection at chunk granularity
+# ---------------------------------------------------------------------------------------------
+def _chunk_rows():
+    rows = []
+    for line in (Path(__file__).parent / "golden" / "chunk_worked_rows.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        p, c, vals, kept = [x.strip() for x in line.split("|")]
+        rows.append((float(p), int(c), [float(v) for v in vals.split()], [int(v) for v in kept.split()]))
+    return rows
+
+
+@pytest.mark.parametrize("p,chunk,vals,kept", _chunk_rows())
+def test_chunk_selection_worked_rows(p, chunk, vals, kept):
+    x = np.asarray(vals, np.float32).reshape(1, 1, 1, -1)
+    idx, cnt, st, _ = oracle.select_variant([x], [0], np.array([x.shape[-1]], np.int32), p, chunk=chunk)
+    assert st[0, 0, 0] == 0 and idx[0, 0, 0, :cnt[0, 0, 0]].tolist() == kept
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_chunk_selection_equals_numpy_nucleus_over_chunk_sums(seed):
+    rng = np.random.default_rng(700 + seed)
+    H, gamma, L = 2, 3, int(rng.integers(50, 2000))
+    chunk = int(rng.choice([4, 16, 64]))
+    x = (rng.random((1, H, gamma, L), dtype=np.float32) ** 5).astype(np.float32)
+    kv = np.array([L - int(rng.integers(0, chunk))], np.int32)       # usually a cut last chunk
+    Lb = int(kv[0])
+    for per_step in (False, True):
+        idx, cnt, st, dg = oracle.select_variant([x], [0], kv, 0.9, per_step=per_step, chunk=chunk)
+        if dg[0, 0, 0, 4] < 1e-12:
+            continue
+        rows = []
+        for s in (range(gamma) if per_step else [None]):
+            row = np.zeros(Lb, np.float32)
+            for h in range(H):                                  # heads ascending, queries inside
+                for ss in ([s] if per_step else range(gamma)):
+                    row = (row + x[0, h, ss, :Lb]).astype(np.float32)
+            rows.append(row)
+        want = set()
+        for row in rows:
+            nc = (Lb + chunk - 1) // chunk
+            score = np.zeros(nc, np.float32)
+            for j in range(nc):
+                acc = np.float32(0)
+                for v in row[j * chunk:(j + 1) * chunk]:
+                    acc = np.float32(acc + v)
+                score[j] = acc
+            for j in _numpy_nucleus(score, 0.9):
+                want |= set(range(j * chunk, min(Lb, (j + 1) * chunk)))
+        got = idx[0, 0, 0, :cnt[0, 0, 0]].tolist()
+        assert got == sorted(want)
+        # whole chunks only
+        kept = np.zeros(Lb, bool)
+        kept[got] = True
+        for j in range((Lb + chunk - 1) // chunk):
+            seg = kept[j * chunk:(j + 1) * chunk]
+            assert seg.all() or not seg.any()
+
+
+def test_chunk_one_is_per_position_selection():
+    rng = np.random.default_rng(9)
+    x = rng.random((2, 2, 2, 300), dtype=np.float32)
+    kv = np.array([300, 123], np.int32)
+    for per_step, it in ((False, 0), (True, 0), (False, 10)):
+        a = oracle.select_variant([x], [0], kv, 0.85, per_step=per_step, n_iters=it, chunk=1)
+        b = oracle.select_variant([x], [0], kv, 0.85, per_step=per_step, n_iters=it)
+        assert all(np.array_equal(u, v) for u, v in zip(a[:3], b[:3]))
