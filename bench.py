@@ -344,7 +344,9 @@ def select_variants(step, cfg, reps=5):
     idx = torch.empty_like(step.idx)
     for name, kw in (("aggregate_exact", {}), ("per_step_union_exact", dict(per_step=True)),
                      ("aggregate_bisect10", dict(bisect_iters=10)),
-                     ("per_step_union_bisect10", dict(per_step=True, bisect_iters=10))):
+                     ("per_step_union_bisect10", dict(per_step=True, bisect_iters=10)),
+                     ("chunk16_aggregate_exact", dict(chunk=16)),
+                     ("chunk16_per_step_union_bisect10", dict(chunk=16, per_step=True, bisect_iters=10))):
         counts = torch.full_like(step.counts, -1)
         status = torch.full_like(step.row_status, -1)
         f = lambda: sa.select_topp(step.draft_probs, step.kv_len, step.layer_map, cfg.p, idx=idx, counts=counts,

@@ -94,6 +94,12 @@ extern "C" {
  *       short of the target mass or exceed the smallest set.  p >= 1 and all-zero rows still
  *       keep every position.  diag then describes the exact threshold of the last row searched.
  *
+ *   chunk = c in {4, 8, 16, 32, 64} (0 or 1 = off): selection at chunk granularity (Sec. 4 sets
+ *       the chunk size to 16; how a chunk is scored is not stated -- here: its score is
+ *       +0 + a[c j] + a[c j + 1] + ... in binary32, ascending, the last chunk cut at kv_len).  The
+ *       nucleus (either variant above applies) is taken over the row of chunk scores and a kept
+ *       chunk keeps all its positions; counts / idx_stride stay in positions.
+ *
  * Requirements: 1 <= n_draft_layers <= 64; n_draft_heads <= 256; gamma >= 1; L_stride a
  * multiple of 4 and <= SPECATTN_MAX_KV_LEN; every draft_probs[u] 16-byte aligned;
  * 0 <= kv_len[b] <= L_stride (larger values are clamped); 0 < p (NaN rejected);
@@ -125,6 +131,8 @@ typedef struct specattn_select_args {
   double* diag;
   int32_t per_step;     /* 0 | 1 */
   int32_t bisect_iters; /* 0 = exact threshold, else 1..64 */
+  int32_t chunk;        /* 0 | 1 = per position, else 4, 8, 16, 32 or 64 */
+  int32_t reserved;     /* 0 */
 } specattn_select_args;
 
 int specattn_select_topp(const specattn_select_args* args, void* cuda_stream);

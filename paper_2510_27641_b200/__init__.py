@@ -41,7 +41,8 @@ class SelectArgs(C.Structure):
                 ("layer_map", C.POINTER(C.c_int32)), ("head_group", C.POINTER(C.c_int32)),
                 ("p", C.c_float), ("idx", C.c_void_p), ("idx_stride", C.c_int64),
                 ("counts", C.c_void_p), ("row_status", C.c_void_p), ("diag", C.c_void_p),
-                ("per_step", C.c_int32), ("bisect_iters", C.c_int32)]
+                ("per_step", C.c_int32), ("bisect_iters", C.c_int32), ("chunk", C.c_int32),
+                ("reserved", C.c_int32)]
 
 
 class VerifyArgs(C.Structure):
@@ -119,7 +120,8 @@ def make_select_args(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.T
                      layer_map: Sequence[int], p: float, *, n_groups: int = 1,
                      head_group: Sequence[int] | None = None, idx: torch.Tensor,
                      counts: torch.Tensor, row_status: torch.Tensor,
-                     diag: torch.Tensor | None = None, per_step: bool = False, bisect_iters: int = 0):
+                     diag: torch.Tensor | None = None, per_step: bool = False, bisect_iters: int = 0,
+                     chunk: int = 1):
     """Fills a SelectArgs.  Returns (args, keepalive) -- keepalive holds the host arrays the
     struct points at and must outlive the call."""
     n_d = len(draft_probs)
@@ -145,7 +147,7 @@ def make_select_args(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.T
     a.idx, a.idx_stride = idx.data_ptr(), idx.shape[3]
     a.counts, a.row_status = counts.data_ptr(), row_status.data_ptr()
     a.diag = None if diag is None else diag.data_ptr()
-    a.per_step, a.bisect_iters = int(bool(per_step)), int(bisect_iters)
+    a.per_step, a.bisect_iters, a.chunk = int(bool(per_step)), int(bisect_iters), int(chunk)
     return a, (ptrs, lm, hg, draft_probs, kv_len, idx, counts, row_status, diag)
 
 
@@ -154,7 +156,8 @@ def select_topp(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.Tensor
                 head_group: Sequence[int] | None = None, idx_stride: int | None = None,
                 idx: torch.Tensor | None = None, counts: torch.Tensor | None = None,
                 row_status: torch.Tensor | None = None, diag: torch.Tensor | None = None,
-                want_diag: bool = False, per_step: bool = False, bisect_iters: int = 0, stream=None):
+                want_diag: bool = False, per_step: bool = False, bisect_iters: int = 0, chunk: int = 1,
+                stream=None):
     """specattn_select_topp.  draft_probs: per draft layer a float32 CUDA tensor
     [B, H_d, gamma, L_stride] (None for layers no target layer maps to).  Returns
     (idx [n_d,B,G,idx_stride] int32, counts [n_d,B,G], row_status [n_d,B,G], diag or None)."""
@@ -174,7 +177,7 @@ def select_topp(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.Tensor
     args, keep = make_select_args(draft_probs, kv_len, layer_map, p, n_groups=n_groups,
                                   head_group=head_group, idx=idx, counts=counts,
                                   row_status=row_status, diag=diag, per_step=per_step,
-                                  bisect_iters=bisect_iters)
+                                  bisect_iters=bisect_iters, chunk=chunk)
     rc = lib().specattn_select_topp(C.byref(args), _stream_ptr(stream))
     if rc != 0:
         raise SpecAttnError(rc, "specattn_select_topp")

@@ -80,6 +80,7 @@ struct SelectParams {
   int single_row;  // every list has exactly one contributing row: read it in place
   int per_step;    // Alg. 2 as printed: one nucleus per speculated query, unioned
   int bisect_iters;  // > 0: the threshold is the last midpoint of that many bisection steps
+  int chunk;         // > 1: selection over per-chunk sums (power of two, 4..64); kept chunks keep all positions
 };
 
 // A histogram of exact mantissa sums, kept as two 32-bit words: `lo` sums the low 16 mantissa
@@ -275,13 +276,14 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   if (Lll < 0) Lll = 0;
   if (Lll > P.L_stride) Lll = P.L_stride;
   const int L = static_cast<int>(Lll);
-  const int per = ((L + cs - 1) / cs + 3) & ~3;  // slice length, 16-byte aligned start
+  const int align = (kVariant && P.chunk > 4) ? P.chunk : 4;  // slices start on 16 bytes and on a chunk
+  const int per = ((L + cs - 1) / cs + align - 1) & ~(align - 1);
   const int lo = min(L, rank * per);
   const int hi = min(L, lo + per);
   const int n_loc = hi - lo;
 
   // dynamic shared memory behind the fixed part
-  const int slice_cap = kInPlace ? 0 : static_cast<int>(((((P.L_stride + cs - 1) / cs + 3) & ~3ll) + 31) & ~31ll);
+  const int slice_cap = kInPlace ? 0 : static_cast<int>(((((P.L_stride + cs - 1) / cs + align - 1) & ~static_cast<long long>(align - 1)) + 31) & ~31ll);
   float* ring = a + slice_cap;
   double* const r_mass = reinterpret_cast<double*>(ring);
   unsigned int* const lvl_base = reinterpret_cast<unsigned int*>(ring + 4096);  // 2 levels x (lo, hi) x 1024
@@ -296,6 +298,10 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   const int n4 = (n_loc + 3) >> 2;
   const int n_pos4 = n4 * 4;                       // slice length rounded up to whole float4s
   const int n_chunks = (n_pos4 + kChunk - 1) / kChunk;
+  // selection at chunk granularity: the searched row (one score per chunk) is built after the
+  // aggregation, and the search and the compaction walk n_srch entries instead of n_loc
+  const bool chunked = kVariant && P.chunk > 1;
+  const int n_srch = chunked ? (n_loc + P.chunk - 1) / P.chunk : n_loc;
   // Alg. 2 as printed selects per speculated query and unions the sets: then everything up to
   // the threshold runs once per query over the row summed over heads only, and the kept
   // positions are collected in a bit mask of the slice.
@@ -341,11 +347,11 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
                !(v.z >= 0.f && v.z <= FLT_MAX) | !(v.w >= 0.f && v.w <= FLT_MAX);
       }
       const float vals[4] = {v.x + 0.f, v.y + 0.f, v.z + 0.f, v.w + 0.f};
-      if (kVariant) vmax = fmaxf(vmax, fmaxf(fmaxf(vals[0], vals[1]), fmaxf(vals[2], vals[3])));
+      if (kVariant && !chunked) vmax = fmaxf(vmax, fmaxf(fmaxf(vals[0], vals[1]), fmaxf(vals[2], vals[3])));
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const unsigned int key = __float_as_uint(vals[e]);
-        const bool take = act && (4 * i4 + e < n_loc) && key != 0u && !(key >> 31);
+        const bool take = act && (4 * i4 + e < n_loc) && key != 0u && !(key >> 31) && !chunked;
         hist_add(h1, take, static_cast<int>(key >> 20), mantissa_of(key));
       }
     }
@@ -423,18 +429,49 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
           bad |= !(v.x <= FLT_MAX) | !(v.y <= FLT_MAX) | !(v.z <= FLT_MAX) | !(v.w <= FLT_MAX);
         }
         const float vals[4] = {v.x, v.y, v.z, v.w};
-        if (kVariant && act) vmax = fmaxf(vmax, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
+        if (kVariant && act && !chunked) vmax = fmaxf(vmax, fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w)));
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const unsigned int key = __float_as_uint(vals[e]);
           // zeros carry no mass and can never be the threshold of a row with positive total
-          const bool take = act && (pos + e < n_loc) && key != 0u && !(key >> 31);
+          const bool take = act && (pos + e < n_loc) && key != 0u && !(key >> 31) && !chunked;
           hist_add(h1, take, static_cast<int>(key >> 20), mantissa_of(key));
         }
         acc[k] = mn[k] = make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
+  }
+  if (chunked) {
+    // Selection at chunk granularity: entry j of the searched row is the binary32 sum of the
+    // chunk's aggregated values in ascending order (the last chunk of the list is cut at L).
+    // The scores replace the head of the slice: a round reads 256 chunks, then writes 256
+    // entries that no later round reads.
+    __syncthreads();  // the aggregated slice is complete
+    for (int base = 0; base < n_srch; base += kThreads) {
+      const int j = base + tid;
+      const bool act = j < n_srch;
+      float acc = 0.f;
+      if (act) {
+        const int p0 = j * P.chunk;
+        for (int e = 0; e < P.chunk; e += 4) {
+          const float4 v = *reinterpret_cast<const float4*>(a + p0 + e);
+          const int left = n_loc - (p0 + e);
+          if (left > 0) acc = acc + v.x;
+          if (left > 1) acc = acc + v.y;
+          if (left > 2) acc = acc + v.z;
+          if (left > 3) acc = acc + v.w;
+        }
+      }
+      __syncthreads();
+      if (act) {
+        a[j] = acc;
+        bad |= !(acc <= FLT_MAX);
+        vmax = fmaxf(vmax, acc);
+      }
+      const unsigned int key = __float_as_uint(acc);
+      hist_add(h1, act && key != 0u && !(key >> 31), static_cast<int>(key >> 20), mantissa_of(key));
+    }
   }
   if (bad) atomicAdd(&sh.n_invalid, 1);
   if (kVariant) {
@@ -498,11 +535,11 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     if (searching) {
       // only the elements inside the threshold bin take part
       const Hist hr = {lb, lb + kL23Bins};
-      for (int base = 0; base < n_loc; base += kThreads) {
+      for (int base = 0; base < n_srch; base += kThreads) {
         const int i = base + tid;
         unsigned int key = 0u;
         bool take = false;
-        if (i < n_loc) {
+        if (i < n_srch) {
           key = key_at(i);
           take = (key >> (shift + 10)) == prefix;
         }
@@ -549,8 +586,8 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     if (P.per_step) {
       // collect this query's set in the mask: a warp owns whole 32-position words
       unsigned int* mask = reinterpret_cast<unsigned int*>(ring + kRingFloats);
-      const int chunk_m = (((n_loc + kWarps - 1) / kWarps) + 31) & ~31;
-      const int m_lo = min(n_loc, warp * chunk_m), m_hi = min(n_loc, m_lo + chunk_m);
+      const int chunk_m = (((n_srch + kWarps - 1) / kWarps) + 31) & ~31;
+      const int m_lo = min(n_srch, warp * chunk_m), m_hi = min(n_srch, m_lo + chunk_m);
       for (int i0 = m_lo; i0 < m_hi; i0 += 32) {
         const int i = i0 + lane;
         const bool keep = !invalid && i < m_hi && key_at(i) >= theta_key;
@@ -565,21 +602,25 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   }  // for step
 
   // ---- 4: ordered compaction --------------------------------------------------------------------
-  // per-warp contiguous chunks of the slice, 32 positions per step
-  const int chunk = (((n_loc + kWarps - 1) / kWarps) + 31) & ~31;
-  const int w_lo = min(n_loc, warp * chunk);
-  const int w_hi = min(n_loc, w_lo + chunk);
+  // per-warp contiguous ranges of the searched entries, 32 per step; an entry stands for one
+  // position, or for the positions of one chunk (all `chunk` of them, except the last chunk of
+  // the list, which nothing follows)
+  const int wchunk = (((n_srch + kWarps - 1) / kWarps) + 31) & ~31;
+  const int w_lo = min(n_srch, warp * wchunk);
+  const int w_hi = min(n_srch, w_lo + wchunk);
   const unsigned int* const kept_mask = reinterpret_cast<const unsigned int*>(ring + kRingFloats);
   auto kept = [&](int i) -> bool {
     if (kVariant && P.per_step) return (kept_mask[i >> 5] >> (i & 31)) & 1u;
     return key_at(i) >= theta_key;
   };
+  auto n_pos = [&](int i) -> int { return chunked ? min(P.chunk, n_loc - i * P.chunk) : 1; };
   int wc = 0;
   if (!invalid) {
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
       const int i = i0 + lane;
       const bool keep = i < w_hi && kept(i);
-      wc += __popc(__ballot_sync(kFull, keep));
+      if (chunked) wc += __reduce_add_sync(kFull, keep ? n_pos(i) : 0);
+      else wc += __popc(__ballot_sync(kFull, keep));
     }
   }
   if (lane == 0) sh.warp_cnt[warp] = wc;
@@ -607,9 +648,17 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       const int i = i0 + lane;
       const bool keep = i < w_hi && kept(i);
       const unsigned m = __ballot_sync(kFull, keep);
-      const long long my = pos + __popc(m & ((1u << lane) - 1u));
-      if (keep && my < P.idx_stride) out[my] = lo + i;
-      pos += __popc(m);
+      if (chunked) {
+        const int np = keep ? n_pos(i) : 0;
+        const long long my = pos + static_cast<long long>(__popc(m & ((1u << lane) - 1u))) * P.chunk;
+        for (int e = 0; e < np; ++e)
+          if (my + e < P.idx_stride) out[my + e] = lo + i * P.chunk + e;
+        pos += __reduce_add_sync(kFull, np);
+      } else {
+        const long long my = pos + __popc(m & ((1u << lane) - 1u));
+        if (keep && my < P.idx_stride) out[my] = lo + i;
+        pos += __popc(m);
+      }
     }
   }
   if (rank == 0 && tid == 0) {
@@ -657,6 +706,8 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   if (A.L_stride < 0 || A.idx_stride < 0) return SPECATTN_ERR_RANGE;
   if (!(A.p > 0.0f)) return SPECATTN_ERR_RANGE;  // also rejects NaN
   if (A.bisect_iters < 0 || A.bisect_iters > 64 || (A.per_step != 0 && A.per_step != 1)) return SPECATTN_ERR_RANGE;
+  if (A.chunk < 0 || A.chunk > 64 || (A.chunk > 1 && (A.chunk < 4 || (A.chunk & (A.chunk - 1)) != 0)))
+    return SPECATTN_ERR_RANGE;  // 0 / 1 = per position, else a power of two in [4, 64]
   if (A.L_stride % 4 != 0) return SPECATTN_ERR_ALIGN;
   if (A.L_stride > SPECATTN_MAX_KV_LEN) return SPECATTN_ERR_UNSUPPORTED;
   if (static_cast<long long>(A.n_draft_heads) * A.gamma > SPECATTN_MAX_ROWS_PER_LIST)
@@ -711,9 +762,12 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   P.single_row = (static_cast<long long>(A.n_draft_heads) * A.gamma == 1 && A.L_stride >= 32768) ? 1 : 0;
   P.per_step = (A.per_step && A.gamma > 1) ? 1 : 0;  // with one query the union is the single nucleus
   P.bisect_iters = A.bisect_iters;
-  const bool variant = P.per_step || P.bisect_iters > 0;
+  P.chunk = (A.chunk > 1) ? A.chunk : 1;
+  if (P.chunk > 1) P.single_row = 0;  // chunk scores live in the shared-memory slice
+  const bool variant = P.per_step || P.bisect_iters > 0 || P.chunk > 1;
   const int cs = specattn::pick_cluster(A.L_stride, n_lists);
-  const long long slice = P.single_row ? 0 : (((A.L_stride + cs - 1) / cs) + 3) / 4 * 4;
+  const long long s_align = (P.chunk > 4) ? P.chunk : 4;
+  const long long slice = P.single_row ? 0 : (((A.L_stride + cs - 1) / cs) + s_align - 1) / s_align * s_align;
   if (slice > specattn::kSliceCap) return SPECATTN_ERR_UNSUPPORTED;
   // shared memory: fixed part, the aggregated slice, then the per-thread staging ring
   // (kDepth pieces of 8 KB; it later hosts the scan arrays).  Small slices leave room for two

@@ -250,3 +250,52 @@ def test_selection_variants_special_cases():
     a, keep = sa.make_select_args([d], to_dev(kv), [0], 0.9, idx=gi.new_zeros((1, 2, 1, 8)), counts=gc.new_zeros((1, 2, 1)),
                                   row_status=gs.new_zeros((1, 2, 1)), bisect_iters=65)
     assert sa.lib().specattn_select_topp(C.byref(a), None) == -3
+
+
+@pytest.mark.parametrize("chunk,per_step,iters", [(16, False, 0), (16, True, 0), (16, False, 10), (4, True, 10),
+                                                  (64, False, 0), (8, True, 0), (32, False, 5)])
+def test_chunk_granular_selection_matches_oracle(chunk, per_step, iters):
+    import paper_2510_27641_b200 as sa
+    # lengths that are not multiples of the chunk; rows that span a cluster; per-group head sets
+    cases = [(3, 8, 5, 4096, np.array([4096, 1000, 2731], np.int32), 2),
+             (2, 3, 4, 40000, np.array([40000, 33333], np.int32), 1),
+             (2, 2, 2, 64, np.array([3, 64], np.int32), 1)]
+    for B, H, gamma, Ls, kv_len, G in cases:
+        probs = [wl.draft_probs(13, u, kv_len, H, gamma, Ls, sink=6.0, slope=0.004) for u in range(2)]
+        hg = None if G == 1 else (np.arange(H) * G // H).astype(np.int32)
+        for p in (0.8, 0.95):
+            gi, gc, gs, _ = sa.select_topp([to_dev(x) for x in probs], to_dev(kv_len), [1, 0], p, n_groups=G,
+                                           head_group=None if hg is None else hg.tolist(),
+                                           per_step=per_step, bisect_iters=iters, chunk=chunk)
+            torch.cuda.synchronize()
+            oi, oc, os_, od = oracle.select_variant(probs, [1, 0], kv_len, p, per_step=per_step, n_iters=iters,
+                                                    chunk=chunk, n_groups=G, head_group=hg)
+            assert _compare_variant(gi, gc, gs, oi, oc, os_, od) == 2 * B * G
+            # whole chunks only (the last one cut at kv_len)
+            g_idx, g_cnt = gi.cpu().numpy(), gc.cpu().numpy()
+            for b in range(B):
+                kept = np.zeros(int(kv_len[b]), bool)
+                kept[g_idx[0, b, 0, :g_cnt[0, b, 0]]] = True
+                for j in range(0, int(kv_len[b]), chunk):
+                    assert kept[j:j + chunk].all() or not kept[j:j + chunk].any()
+
+
+def test_chunk_selection_overflow_single_row_and_arguments():
+    import paper_2510_27641_b200 as sa
+    kv = np.array([5000], np.int32)
+    probs = wl.draft_probs(14, 0, kv, 2, 2, 5000, sink=6.0, slope=0.004)
+    # the list is cut to idx_stride positions (in the middle of a chunk), the count stays true
+    gi, gc, gs, _ = sa.select_topp([to_dev(probs)], to_dev(kv), [0], 0.99, chunk=16, idx_stride=40)
+    oi, oc, os_, od = oracle.select_variant([probs], [0], kv, 0.99, chunk=16, idx_stride=40)
+    assert gc.item() == oc.item() > 40 and gs.item() == os_.item() == sa.ROW_OVERFLOW
+    assert np.array_equal(gi.cpu().numpy()[0, 0, 0], oi[0, 0, 0])
+    # one long row: chunked selection does not take the in-place path
+    row = wl.topp_rows("zipf", 1, 65536, 5).reshape(1, 1, 1, 65536)
+    kv1 = np.array([65530], np.int32)
+    gi, gc, gs, _ = sa.select_topp([to_dev(row)], to_dev(kv1), [0], 0.9, chunk=16)
+    oi, oc, os_, od = oracle.select_variant([row], [0], kv1, 0.9, chunk=16)
+    _compare_variant(gi, gc, gs, oi, oc, os_, od)
+    for bad_chunk in (2, 3, 12, 128, -1):
+        a, keep = sa.make_select_args([to_dev(probs)], to_dev(kv), [0], 0.9, idx=gi.new_zeros((1, 1, 1, 8)),
+                                      counts=gc.new_zeros((1, 1, 1)), row_status=gs.new_zeros((1, 1, 1)), chunk=bad_chunk)
+        assert sa.lib().specattn_select_topp(C.byref(a), None) == -3
