@@ -276,12 +276,18 @@ int specattn_sparse_verify_static(const specattn_verify_args* args, void* cuda_s
  *
  * Alg. 1, blocks "Sparse Attention Mask Creation" and "Verification with Sparse Attention":
  * one select over the mapped draft layers, then one sparse verify per target layer, with the
- * step's inputs and results crossing PCIe inside the call.  In stream order it
- *   1. copies draft_probs_host[u] -> select.draft_probs[u] for every mapped draft layer,
- *   2. runs specattn_select_topp(select),
- *   3. for each target layer j: copies q_host[j] -> verify[j].q, runs
- *      specattn_sparse_verify(verify[j]) and copies verify[j].out / .lse -> out_host[j] /
- *      lse_host[j].
+ * step's inputs and results crossing PCIe inside the call.  It
+ *   1. copies q_host[j] -> verify[j].q for every target layer and draft_probs_host[u] ->
+ *      select.draft_probs[u] for every mapped draft layer, on a copy stream of its own,
+ *   2. on the caller's stream runs specattn_select_topp for a draft layer as soon as its rows
+ *      have landed (one launch per mapped draft layer) and then specattn_sparse_verify(verify[j])
+ *      of the target layers mapped to it, while later draft layers are still being copied,
+ *   3. copies verify[j].out / .lse -> out_host[j] / lse_host[j] on a second copy stream as each
+ *      layer finishes,
+ * and finally makes the caller's stream wait for both copy streams: work enqueued on that
+ * stream afterwards sees the step complete.  The two copy streams and the events between the
+ * lanes are created on the first call per device and kept; one call at a time enqueues per
+ * device.  select.n_target_layers must equal n_target_layers.
  * `select` and `verify[j]` are complete device-side argument structs (their device buffers,
  * including the staging buffers the copies land in, are the caller's); verify[j].idx/counts
  * must already point at the lists of layer_map[j] (or dense be set where layer_map[j] < 0).
