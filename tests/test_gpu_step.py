@@ -134,8 +134,20 @@ def test_host_buffer_step_matches_device_resident_step():
     out_host = [torch.zeros(o.shape, dtype=torch.float32).pin_memory() for o in step.out]
     lse_host = [torch.zeros(l.shape, dtype=torch.float32).pin_memory() for l in step.lse]
     step.run_host(dp_host, q_host, out_host, lse_host)
+    # work enqueued on the caller's stream afterwards sees the step complete (the call joins its
+    # copy lanes back into that stream): a device-side copy of the last layer's output, taken
+    # without any synchronisation in between
+    seen = step.out[3].clone()
     torch.cuda.synchronize()
-    assert torch.equal(step.counts, ref_cnt)
+    assert torch.equal(step.counts, ref_cnt) and torch.equal(seen, ref_out[3])
+    for j in range(4):
+        assert torch.equal(out_host[j], ref_out[j].cpu()) and torch.equal(lse_host[j], ref_lse[j].cpu())
+    # two steps back to back reuse the lanes and their events
+    for t in out_host:
+        t.zero_()
+    step.run_host(dp_host, q_host, out_host, lse_host)
+    step.run_host(dp_host, q_host, out_host, lse_host)
+    torch.cuda.synchronize()
     for j in range(4):
         assert torch.equal(out_host[j], ref_out[j].cpu()) and torch.equal(lse_host[j], ref_lse[j].cpu())
 
