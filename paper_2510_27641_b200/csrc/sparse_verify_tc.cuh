@@ -10,8 +10,8 @@
 //   S^T[128 keys x N]  = K[128 x 128] Q^T          A = K tile, B = Q tile, both K-major in smem
 //   O^T[128 dims x N] += V^T[128 x 128 keys] P^T   A = V tile (MN-major), B = P^T (MN-major)
 // No tensor work is spent on padding rows, and -- because a TMEM lane is a key (or an output
-// dimension) -- the four softmax warps, one per lane quadrant and hence one per SM
-// sub-partition, each own 32 keys of every tile.  P = exp2(S - m) is written as two bf16
+// dimension) -- the softmax warps are spread over the four lane quadrants, i.e. over the four SM
+// sub-partitions: a warp owns 32 keys of every tile (and half of the query rows).  P = exp2(S - m) is written as two bf16
 // terms (P = P_hi + P_lo) into the shared-memory bytes of the K tile it was computed from,
 // which are dead once S^T is complete; the stage is released when the P V product has read it.
 //
@@ -20,10 +20,10 @@
 // bf16 terms and fp32 accumulation); only a tile that exceeds it takes the slow path (row
 // maxima over the 128 keys by warp butterflies and a small shared-memory exchange, then a
 // rescale of the O^T columns in tensor memory).  Whether a tile takes it is agreed per tile
-// through one named barrier of the four softmax warps.
+// through one named barrier of the softmax warps.
 //
-// Warps: 0-3 softmax (TMEM lane quadrant = warp index), 4 = MMA issue (one thread),
-// 5-8 = producers: two warps per tile, 64 keys each, 16-byte cp.async straight into the
+// Warps: 0-7 softmax (TMEM lane quadrant = warp % 4, half of the query rows = warp / 4, so every
+// SM sub-partition runs two of them), 8 = MMA issue (one thread), 9-12 = producers: two warps per tile, 64 keys each, 16-byte cp.async straight into the
 // 128-byte-swizzled operand layout, then fence.proxy.async before the arrival.
 #pragma once
 
@@ -32,9 +32,9 @@ constexpr int kTcTileBytes = kTcTile * 256;      // one K or V tile (32 KB)
 constexpr int kTcStages = 3;
 constexpr int kTcRec = 130 * 32;                 // floats of a record per 32 query rows
 constexpr float kTcRaise = 8.f;                  // raise the reference maximum beyond 2^8
-constexpr int kTcThreads = 9 * 32;
-constexpr int kTcMmaWarp = 4;
-constexpr int kTcSoftmaxThreads = 128;
+constexpr int kTcThreads = 13 * 32;
+constexpr int kTcMmaWarp = 8;
+constexpr int kTcSoftmaxThreads = 256;
 
 // byte offset of 16-byte chunk `c` (0..15) of row `r` in a tile of `rows` rows of 256 bytes: two
 // 128-byte halves per row, chunks XOR-swizzled with the row index (UMMA 128-byte swizzle)
@@ -89,6 +89,16 @@ __device__ __forceinline__ void tc_st16(uint32_t addr, const uint32_t (&r)[16]) 
       "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
+__device__ __forceinline__ void tc_ld8(uint32_t (&r)[8], uint32_t addr) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(addr));
+}
+__device__ __forceinline__ void tc_st8(uint32_t addr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(addr), "r"(r[0]),
+               "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
 // named barrier that also ORs a predicate over its participants: everyone gets the same answer,
 // so a group that must leave together can decide to leave on it
 __device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool pred) {
@@ -118,6 +128,15 @@ __device__ __forceinline__ void tc_lds16(int (&d)[16], const int* p) {
     const int4 v = reinterpret_cast<const int4*>(p)[i];
     d[4 * i] = v.x; d[4 * i + 1] = v.y; d[4 * i + 2] = v.z; d[4 * i + 3] = v.w;
   }
+}
+
+__device__ __forceinline__ void tc_lds8(float (&d)[8], const float* p) {
+  const float4 v0 = reinterpret_cast<const float4*>(p)[0], v1 = reinterpret_cast<const float4*>(p)[1];
+  d[0] = v0.x; d[1] = v0.y; d[2] = v0.z; d[3] = v0.w; d[4] = v1.x; d[5] = v1.y; d[6] = v1.z; d[7] = v1.w;
+}
+__device__ __forceinline__ void tc_lds8(int (&d)[8], const int* p) {
+  const int4 v0 = reinterpret_cast<const int4*>(p)[0], v1 = reinterpret_cast<const int4*>(p)[1];
+  d[0] = v0.x; d[1] = v0.y; d[2] = v0.z; d[3] = v0.w; d[4] = v1.x; d[5] = v1.y; d[6] = v1.z; d[7] = v1.w;
 }
 
 // Butterfly reduce-scatter over the 32 lanes of a warp: v[i] is this lane's value for row i;
@@ -168,7 +187,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   constexpr int NS = kTcStages;
   constexpr int NTH = kTcThreads;
   constexpr int NBLK = (N + 31) / 32;
-  constexpr bool kKeepS = true;  // scores stay in registers between the two passes
   extern __shared__ __align__(1024) unsigned char smem_raw_tc[];
   TcShared& sh =
       *reinterpret_cast<TcShared*>((reinterpret_cast<uintptr_t>(smem_raw_tc) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -194,11 +212,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
     mbar_init(&sh.q_empty, 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sh.s_full[i], 1);
-      mbar_init(&sh.s_free[i], 4);
-      mbar_init(&sh.p_full[i], 4);
+      mbar_init(&sh.s_free[i], 8);   // one arrival per softmax warp
+      mbar_init(&sh.p_full[i], 8);
       mbar_init(&sh.pv_done[i], 1);
     }
-    mbar_init(&sh.o_free, 4);
+    mbar_init(&sh.o_free, 8);
     mbar_fence_init();
     sh.abort_flag = 0;
     sh.raise_tile[0] = sh.raise_tile[1] = 0;
@@ -285,7 +303,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   __syncthreads();
   const long long NP = aligned ? sh.part_start[U] : ((NA < G) ? NA : static_cast<long long>(G));
 
-  const bool is_softmax = warp < 4;
+  const bool is_softmax = warp < 8;
   const bool is_mma = (warp == kTcMmaWarp);
   if (is_softmax) {
     // the only warps that write global memory: the previous kernel is complete from here on
@@ -353,7 +371,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   if (!is_softmax && !is_mma) {
     // =============================== producer warps ===============================================
     // tile i is filled by warps 2 (i & 1) and 2 (i & 1) + 1: keys 0..63 and 64..127 of the tile
-    const int pw = warp - 5;
+    const int pw = warp - 9;
     const int tpar = pw >> 1, half = pw & 1;
     int it = 0, seg = 0;
     int a = a0, u = u_first;
@@ -544,8 +562,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
     __syncwarp();
   } else {
     // =============================== softmax warps ==============================================
-    const int key_lane = tid;  // key of the tile / output dimension = TMEM lane
-    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
+    // warp = (row half, lane quadrant): 32 keys of the tile against half of the query rows
+    constexpr int RW = N / 2;   // query rows of this warp
+    constexpr int NO = NT;      // ... in groups of eight
+    const int quad = warp & 3, r0 = (warp >> 2) * RW;
+    const int key_lane = quad * 32 + lane;  // key of the tile / output dimension = TMEM lane
+    const uint32_t lane_sel = static_cast<uint32_t>(quad * 32) << 16;
     constexpr int kBar = 1;
     bool fail = false;
     int it = 0, seg = 0;
@@ -571,9 +593,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
       const int c_list = ucnt - P.tail;
       const int ntiles = (tok_hi - tok_lo + kTcTile - 1) / kTcTile;
       if (tid < N) sh.m_ref[tid] = -INFINITY;
-      float l_part[N];
+      float l_part[RW];
 #pragma unroll
-      for (int r = 0; r < N; ++r) l_part[r] = 0.f;
+      for (int r = 0; r < RW; ++r) l_part[r] = 0.f;
       if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
 
       for (int n = 0; n < ntiles; ++n) {
@@ -589,29 +611,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         const bool tail_tile = P.tail && (t0 + kTcTile > c_list);
         // ---- pass 1: does any visible score exceed its row's reference maximum by 2^8? --------
         bool exceed = false;
-        uint32_t sv[NT][16];  // this key's scores against every query row
+        uint32_t sv[NO][8];  // this key's scores against this warp's query rows
         if (!__any_sync(0xffffffffu, fail)) {
 #pragma unroll
-          for (int c = 0; c < NT; ++c) tc_ld16(sv[c], tmem + sb * N + lane_sel + c * 16);
+          for (int o = 0; o < NO; ++o) tc_ld8(sv[o], tmem + sb * N + lane_sel + r0 + o * 8);
           tc_wait_ld();
-          if (!kKeepS) {  // the scores are read again in pass 2; until then the registers are free
-            tc_fence_before();
-          }
 #pragma unroll
-          for (int c = 0; c < NT; ++c) {
-            float mr[16];
-            tc_lds16(mr, sh.m_ref + c * 16);
+          for (int o = 0; o < NO; ++o) {
+            float mr[8];
+            tc_lds8(mr, sh.m_ref + r0 + o * 8);
             if (!tail_tile) {
 #pragma unroll
-              for (int j = 0; j < 16; ++j)
-                exceed |= !(fmaf(__uint_as_float(sv[c][j]), P.scale_log2, -mr[j]) <= kTcRaise);
+              for (int j = 0; j < 8; ++j)
+                exceed |= !(fmaf(__uint_as_float(sv[o][j]), P.scale_log2, -mr[j]) <= kTcRaise);
             } else {
-              int lim[16];
-              tc_lds16(lim, sh.row_lim + c * 16);
+              int lim[8];
+              tc_lds8(lim, sh.row_lim + r0 + o * 8);
 #pragma unroll
-              for (int j = 0; j < 16; ++j)
+              for (int j = 0; j < 8; ++j)
                 exceed |= ((jt < 0) | (jt <= lim[j])) &
-                          !(fmaf(__uint_as_float(sv[c][j]), P.scale_log2, -mr[j]) <= kTcRaise);
+                          !(fmaf(__uint_as_float(sv[o][j]), P.scale_log2, -mr[j]) <= kTcRaise);
             }
           }
           exceed &= kvalid;
@@ -620,26 +639,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
         if (sh.raise_tile[sb] == i + 1) {
           // ---- slow path: new row maxima, rescale of the sums and of O^T ----------------------
-#pragma unroll
-          for (int blk = 0; blk < NBLK; ++blk) {
+          {
             float v[32];
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-              if (blk * 2 + c < NT) {
-                int lim[16];
-                tc_lds16(lim, sh.row_lim + (blk * 2 + c) * 16);
+            for (int j = 0; j < 32; ++j) v[j] = -INFINITY;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                  const bool vis = kvalid & (!tail_tile | (jt < 0) | (jt <= lim[j]));
-                  v[c * 16 + j] = vis ? __uint_as_float(sv[blk * 2 + c][j]) * P.scale_log2 : -INFINITY;
-                }
-              } else {
+            for (int o = 0; o < NO; ++o) {
+              int lim[8];
+              tc_lds8(lim, sh.row_lim + r0 + o * 8);
 #pragma unroll
-                for (int j = 0; j < 16; ++j) v[c * 16 + j] = -INFINITY;
+              for (int j = 0; j < 8; ++j) {
+                const bool vis = kvalid & (!tail_tile | (jt < 0) | (jt <= lim[j]));
+                v[o * 8 + j] = vis ? __uint_as_float(sv[o][j]) * P.scale_log2 : -INFINITY;
               }
             }
             const float wm = tc_reduce_scatter<true>(v, lane);
-            if (blk * 32 + lane < N) sh.wred[warp][blk * 32 + lane] = wm;
+            if (lane < RW) sh.wred[quad][r0 + lane] = wm;
           }
           if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
           if (tid < N) {
@@ -655,25 +670,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
             tc_fence_after();
             if (!__any_sync(0xffffffffu, fail)) {
 #pragma unroll
-              for (int c = 0; c < 2 * NT; ++c) {  // the P_hi and the P_lo half of O^T
-                uint32_t ov[16];
-                tc_ld16(ov, col_o + lane_sel + c * 16);
-                float al[16];
-                tc_lds16(al, sh.alpha + (c % NT) * 16);
+              for (int c = 0; c < 2 * NO; ++c) {  // this warp's rows in the P_hi and the P_lo part of O^T
+                const int col = (c / NO) * N + r0 + (c % NO) * 8;
+                uint32_t ov[8];
+                tc_ld8(ov, col_o + lane_sel + col);
+                float al[8];
+                tc_lds8(al, sh.alpha + r0 + (c % NO) * 8);
                 tc_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 16; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * al[j]);
-                tc_st16(col_o + lane_sel + c * 16, ov);
+                for (int j = 0; j < 8; ++j) ov[j] = __float_as_uint(__uint_as_float(ov[j]) * al[j]);
+                tc_st8(col_o + lane_sel + col, ov);
               }
               tc_wait_st();
             }
           }
 #pragma unroll
-          for (int c = 0; c < NT; ++c) {
-            float al[16];
-            tc_lds16(al, sh.alpha + c * 16);
+          for (int o = 0; o < NO; ++o) {
+            float al[8];
+            tc_lds8(al, sh.alpha + r0 + o * 8);
 #pragma unroll
-            for (int j = 0; j < 16; ++j) l_part[c * 16 + j] *= al[j];
+            for (int j = 0; j < 8; ++j) l_part[o * 8 + j] *= al[j];
           }
         }
         // ---- pass 2: P = exp2(S - m) as two bf16 terms, into the dead K tile ------------------
@@ -684,43 +700,40 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.s_free[sb]);
 #pragma unroll
-          for (int c = 0; c < NT; ++c) {
-            float mr[16];
-            tc_lds16(mr, sh.m_ref + c * 16);
-            float p[16];
+          for (int o = 0; o < NO; ++o) {
+            float mr[8];
+            tc_lds8(mr, sh.m_ref + r0 + o * 8);
+            float p[8];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) p[j] = ex2(fmaf(__uint_as_float(sv[c][j]), P.scale_log2, -mr[j]));
+            for (int j = 0; j < 8; ++j) p[j] = ex2(fmaf(__uint_as_float(sv[o][j]), P.scale_log2, -mr[j]));
             if (tail_tile) {
-              int lim[16];
-              tc_lds16(lim, sh.row_lim + c * 16);
+              int lim[8];
+              tc_lds8(lim, sh.row_lim + r0 + o * 8);
 #pragma unroll
-              for (int j = 0; j < 16; ++j) p[j] = ((jt < 0) | (jt <= lim[j])) ? p[j] : 0.f;
+              for (int j = 0; j < 8; ++j) p[j] = ((jt < 0) | (jt <= lim[j])) ? p[j] : 0.f;
             }
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
+            for (int j = 0; j < 8; ++j) {
               p[j] = kvalid ? p[j] : 0.f;
-              l_part[c * 16 + j] += p[j];
+              l_part[o * 8 + j] += p[j];
             }
+            // P = P_hi + P_lo in bf16 on the integer / FMA pipes: P_hi keeps the upper 16 bits
+            // (truncation), P_lo is the exact remainder rounded to nearest (P >= 0, so adding
+            // half an ulp to the bit pattern rounds): |P - P_hi - P_lo| <= 2^-16 P, unbiased
+            uint32_t hi[4], lo[4];
 #pragma unroll
-            for (int g8 = 0; g8 < 2; ++g8) {
-              // P = P_hi + P_lo in bf16 on the integer / FMA pipes: P_hi keeps the upper 16 bits
-              // (truncation), P_lo is the exact remainder rounded to nearest (P >= 0, so adding
-              // half an ulp to the bit pattern rounds): |P - P_hi - P_lo| <= 2^-16 P, unbiased
-              uint32_t hi[4], lo[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                const uint32_t b0 = __float_as_uint(p[g8 * 8 + 2 * e]), b1 = __float_as_uint(p[g8 * 8 + 2 * e + 1]);
-                hi[e] = __byte_perm(b0, b1, 0x7632);
-                const uint32_t d0 = __float_as_uint(__uint_as_float(b0) - __uint_as_float(b0 & 0xffff0000u)) + 0x8000u;
-                const uint32_t d1 = __float_as_uint(__uint_as_float(b1) - __uint_as_float(b1 & 0xffff0000u)) + 0x8000u;
-                lo[e] = __byte_perm(d0, d1, 0x7632);
-              }
-              // B operand [P_hi^T | P_lo^T]: 2N columns, 16-byte chunk ch of a key's row at
-              // (ch / 8) * 16 KB + ((ch % 8) ^ (key % 8)) * 16
-              const int ch_hi = c * 2 + g8, ch_lo = ch_hi + N / 8;
-              st_shared_v4(pb + (ch_hi >> 3) * 16384 + (((ch_hi & 7) ^ (key_lane & 7)) << 4), hi[0], hi[1], hi[2], hi[3]);
-              st_shared_v4(pb + (ch_lo >> 3) * 16384 + (((ch_lo & 7) ^ (key_lane & 7)) << 4), lo[0], lo[1], lo[2], lo[3]);
+            for (int e = 0; e < 4; ++e) {
+              const uint32_t b0 = __float_as_uint(p[2 * e]), b1 = __float_as_uint(p[2 * e + 1]);
+              hi[e] = __byte_perm(b0, b1, 0x7632);
+              const uint32_t d0 = __float_as_uint(__uint_as_float(b0) - __uint_as_float(b0 & 0xffff0000u)) + 0x8000u;
+              const uint32_t d1 = __float_as_uint(__uint_as_float(b1) - __uint_as_float(b1 & 0xffff0000u)) + 0x8000u;
+              lo[e] = __byte_perm(d0, d1, 0x7632);
             }
+            // B operand [P_hi^T | P_lo^T]: 2N columns, 16-byte chunk ch of a key's row at
+            // (ch / 8) * 16 KB + ((ch % 8) ^ (key % 8)) * 16
+            const int ch_hi = (r0 >> 3) + o, ch_lo = ch_hi + N / 8;
+            st_shared_v4(pb + (ch_hi >> 3) * 16384 + (((ch_hi & 7) ^ (key_lane & 7)) << 4), hi[0], hi[1], hi[2], hi[3]);
+            st_shared_v4(pb + (ch_lo >> 3) * 16384 + (((ch_lo & 7) ^ (key_lane & 7)) << 4), lo[0], lo[1], lo[2], lo[3]);
           }
           fence_proxy_async();  // P^T is read by the tensor core through the async proxy
           __syncwarp();
@@ -731,13 +744,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
       if (fail) sh.abort_flag = 1;
 
       // ---- end of the unit's share: row sums over all keys, O^T out of tensor memory ------------
-#pragma unroll
-      for (int blk = 0; blk < NBLK; ++blk) {
+      {
         float v[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = (blk * 32 + j < N) ? l_part[(blk * 32 + j < N) ? blk * 32 + j : 0] : 0.f;
+        for (int j = 0; j < 32; ++j) v[j] = (j < RW) ? l_part[(j < RW) ? j : 0] : 0.f;
         const float ws = tc_reduce_scatter<false>(v, lane);
-        if (blk * 32 + lane < N) sh.wred[warp][blk * 32 + lane] = ws;
+        if (lane < RW) sh.wred[quad][r0 + lane] = ws;
       }
       if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
       if (tid < N) sh.lsum[tid] = (sh.wred[0][tid] + sh.wred[1][tid]) + (sh.wred[2][tid] + sh.wred[3][tid]);
@@ -750,14 +762,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
       const int d = key_lane;  // this thread's output dimension
       if (whole) {
 #pragma unroll
-        for (int c = 0; c < NT; ++c) {
-          uint32_t ov[16], ow[16];
-          tc_ld16(ov, col_o + lane_sel + c * 16);
-          tc_ld16(ow, col_o + lane_sel + N + c * 16);
+        for (int o = 0; o < NO; ++o) {
+          uint32_t ov[8], ow[8];
+          tc_ld8(ov, col_o + lane_sel + r0 + o * 8);
+          tc_ld8(ow, col_o + lane_sel + N + r0 + o * 8);
           tc_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int r = c * 16 + j;
+          for (int j = 0; j < 8; ++j) {
+            const int r = r0 + o * 8 + j;
             if (r < P.M) {
               const float l = sh.lsum[r];
               P.out[(obase + sh.row_off[r]) * kD + d] =
@@ -773,14 +785,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         // publish this CTA's share ([row][dim] sums, then m, then l), then see who arrived last
         float* rec = P.partials + static_cast<size_t>(2 * blockIdx.x + (a == a0 ? 0 : 1)) * NBLK * kTcRec;
 #pragma unroll
-        for (int c = 0; c < NT; ++c) {
-          uint32_t ov[16], ow[16];
-          tc_ld16(ov, col_o + lane_sel + c * 16);
-          tc_ld16(ow, col_o + lane_sel + N + c * 16);
+        for (int o = 0; o < NO; ++o) {
+          uint32_t ov[8], ow[8];
+          tc_ld8(ov, col_o + lane_sel + r0 + o * 8);
+          tc_ld8(ow, col_o + lane_sel + N + r0 + o * 8);
           tc_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
-            __stcg(rec + (c * 16 + j) * kD + d, __uint_as_float(ov[j]) + __uint_as_float(ow[j]));
+          for (int j = 0; j < 8; ++j)
+            __stcg(rec + (r0 + o * 8 + j) * kD + d, __uint_as_float(ov[j]) + __uint_as_float(ow[j]));
         }
         if (tid < N) {
           __stcg(rec + N * kD + tid, sh.m_ref[tid]);
@@ -797,30 +809,31 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         if (named_bar_or(kBar, kTcSoftmaxThreads, fail)) { fail = true; break; }
         if (sh.last_arriver) {
           __threadfence();
-          // merge every contributor's record in CTA order, 16 query rows at a time
+          // merge every contributor's record in CTA order, eight query rows at a time
           auto rec_of = [&](int i) {
             return P.partials + static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, NA, NP) >= us) ? 0 : 1)) *
                                     NBLK * kTcRec;
           };
 #pragma unroll 1
-          for (int c = 0; c < NT; ++c) {
-            // one pass with a running maximum: the 48 loads of a contributor are independent,
+          for (int o = 0; o < NO; ++o) {
+            // one pass with a running maximum: the 24 loads of a contributor are independent,
             // and two contributors are in flight at a time
-            float mx[16], acc[16], ls[16];
+            const int rb = r0 + o * 8;
+            float mx[8], acc[8], ls[8];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) { mx[j] = -INFINITY; acc[j] = 0.f; ls[j] = 0.f; }
+            for (int j = 0; j < 8; ++j) { mx[j] = -INFINITY; acc[j] = 0.f; ls[j] = 0.f; }
 #pragma unroll 2
             for (int i = i_lo; i <= i_hi; ++i) {
               const float* r2 = rec_of(i);
-              float mi[16], li[16], oi[16];
+              float mi[8], li[8], oi[8];
 #pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                mi[j] = __ldcg(r2 + N * kD + c * 16 + j);
-                li[j] = __ldcg(r2 + N * kD + N + c * 16 + j);
-                oi[j] = __ldcg(r2 + (c * 16 + j) * kD + d);
+              for (int j = 0; j < 8; ++j) {
+                mi[j] = __ldcg(r2 + N * kD + rb + j);
+                li[j] = __ldcg(r2 + N * kD + N + rb + j);
+                oi[j] = __ldcg(r2 + (rb + j) * kD + d);
               }
 #pragma unroll
-              for (int j = 0; j < 16; ++j) {
+              for (int j = 0; j < 8; ++j) {
                 float mn, ao, ai;
                 merge_scales(mx[j], mi[j], mn, ao, ai);
                 mx[j] = mn;
@@ -829,8 +842,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
               }
             }
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const int r = c * 16 + j;
+            for (int j = 0; j < 8; ++j) {
+              const int r = rb + j;
               if (r < P.M) {
                 P.out[(obase + sh.row_off[r]) * kD + d] = acc[j] * ((ls[j] > 0.f) ? 1.f / ls[j] : 0.f);
                 if (d == 0) P.lse[obase + sh.row_off[r]] = (ls[j] > 0.f) ? (mx[j] + log2f(ls[j])) * kLn2 : -INFINITY;
@@ -856,7 +869,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
 
   // ---- release tensor memory once every warp that touches it is done -----------------------------
   tc_fence_before();
-  named_bar_sync(2, 5 * 32);  // warps 0..4
+  named_bar_sync(2, 9 * 32);  // warps 0..8
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
