@@ -193,8 +193,12 @@ int specattn_select_topp(const specattn_select_args* args, void* cuda_stream);
  * SPECATTN_VERIFY_ENGINE_MMA_SYNC / SPECATTN_VERIFY_ENGINE_TCGEN05: force one of the two
  * implementations of the same operation (warp-level mma.sync with register accumulators, or
  * tcgen05.mma with accumulators in tensor memory).  With neither bit the library picks by
- * problem shape; results agree within the tolerance of the operation either way.  Setting
- * both bits is SPECATTN_ERR_RANGE. */
+ * what the host can see: tcgen05 for dense calls with more than 32 query rows per KV head
+ * (n_q * n_q_heads / n_kv_heads) over caches of at least 8192 positions per sequence
+ * (block_table_stride * page_size), mma.sync otherwise -- list lengths live on the device, so a
+ * caller that knows its lists are long (thousands of positions per sequence) and has more than
+ * 32 query rows should set SPECATTN_VERIFY_ENGINE_TCGEN05 itself.  Results agree within the
+ * tolerance of the operation either way.  Setting both bits is SPECATTN_ERR_RANGE. */
 #define SPECATTN_VERIFY_LISTS_STABLE 1u
 #define SPECATTN_VERIFY_ENGINE_MMA_SYNC 2u
 #define SPECATTN_VERIFY_ENGINE_TCGEN05 4u

@@ -853,11 +853,18 @@ int validate(const specattn_verify_args* args) {
 // 32-row blocks of the query block (tcgen05 engine)
 int row_blocks(const specattn_verify_args& A) { return (m_tiles(A) + 1) / 2; }
 
-// Which engine runs a call: the caller's choice, else by shape.
+// Which engine runs a call: the caller's choice, else by what the host can see of the shape.
+// Measured (dense, 32k-131k positions per sequence): with 33-64 query rows per KV head the
+// mma.sync engine sits at its tensor-pipe ceiling (3.1-3.2 TB/s) and the tcgen05 engine reaches
+// 3.6-3.9 TB/s; up to 32 rows, and on short lists at any size (one-shot set-up and merge cost),
+// mma.sync is ahead.  List lengths live on the device, so only dense calls whose cache holds at
+// least 8192 positions per sequence are switched.
 bool use_tcgen05(const specattn_verify_args& A) {
   if (A.flags & SPECATTN_VERIFY_ENGINE_TCGEN05) return true;
   if (A.flags & SPECATTN_VERIFY_ENGINE_MMA_SYNC) return false;
-  return false;
+  const long long rows = static_cast<long long>(A.n_q) * (A.n_q_heads / A.n_kv_heads);
+  const long long capacity = static_cast<long long>(A.block_table_stride) * A.page_size;
+  return A.dense && rows > 32 && capacity >= 8192;
 }
 
 // Sized for either engine, so that the choice never depends on the workspace at hand.

@@ -101,14 +101,28 @@ def test_config4_shape_reduced_with_per_head_lists():
     step1.load_inputs([None if x is None else torch.from_numpy(x) for x in si.draft_probs],
                       [bf16.bits_to_torch(q) for q in si.q])
     step1.run()
+    import paper_2510_27641_b200 as sa
+    # (dense calls of this shape -- 40 query rows per KV head over a 20000-position cache -- go to
+    # the tcgen05 engine by default; the bitwise comparison pins both sides to one engine)
     stepd = VerifyStep(layer_map=[-1, -1], n_draft_layers=2, batch=2, n_draft_heads=16, gamma=4,
                        L_stride=si.L_stride, n_q_heads=64, p=1.0, kv_pools=pools, kv_len=step.kv_len,
-                       block_table=step.block_table)
+                       block_table=step.block_table, verify_flags=sa.VERIFY_ENGINE_MMA_SYNC)
     stepd.load_inputs([None, None], [bf16.bits_to_torch(q) for q in si.q])
     stepd.run()
     torch.cuda.synchronize()
     for j in range(2):
         assert torch.equal(step1.out[j], stepd.out[j]) and torch.equal(step1.lse[j], stepd.lse[j])
+    # the default engine choice for the dense call agrees within the tolerance of the operation
+    stepa = VerifyStep(layer_map=[-1, -1], n_draft_layers=2, batch=2, n_draft_heads=16, gamma=4,
+                       L_stride=si.L_stride, n_q_heads=64, p=1.0, kv_pools=pools, kv_len=step.kv_len,
+                       block_table=step.block_table)
+    stepa.load_inputs([None, None], [bf16.bits_to_torch(q) for q in si.q])
+    stepa.run()
+    torch.cuda.synchronize()
+    assert int(stepa.status.abs().sum()) == 0
+    for j in range(2):
+        assert float((stepa.out[j] - stepd.out[j]).abs().max()) <= 2e-5
+        assert float((stepa.lse[j] - stepd.lse[j]).abs().max()) <= 2e-5
     u = int(si.layer_map[0])
     assert step1.counts[u].cpu().numpy().ravel().tolist() == [20000, 20000]
 
