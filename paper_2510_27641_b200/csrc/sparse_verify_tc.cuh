@@ -112,7 +112,9 @@ __device__ __forceinline__ bool named_bar_or(int id, int nthreads, bool pred) {
   return r != 0;
 }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+  // (no memory clobber: the target bytes are only ever touched through such stores and by the
+  // tensor core, and ordinary loads may move across them; the proxy fence that follows orders them)
+  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d));
 }
 
 __device__ __forceinline__ void tc_lds16(float (&d)[16], const float* p) {
@@ -620,17 +622,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           for (int o = 0; o < NO; ++o) {
             float mr[8];
             tc_lds8(mr, sh.m_ref + r0 + o * 8);
+            // from here on sv holds x = s * scale - m, the exponent of P
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              sv[o][j] = __float_as_uint(fmaf(__uint_as_float(sv[o][j]), P.scale_log2, -mr[j]));
             if (!tail_tile) {
 #pragma unroll
-              for (int j = 0; j < 8; ++j)
-                exceed |= !(fmaf(__uint_as_float(sv[o][j]), P.scale_log2, -mr[j]) <= kTcRaise);
+              for (int j = 0; j < 8; ++j) exceed |= !(__uint_as_float(sv[o][j]) <= kTcRaise);
             } else {
               int lim[8];
               tc_lds8(lim, sh.row_lim + r0 + o * 8);
 #pragma unroll
               for (int j = 0; j < 8; ++j)
-                exceed |= ((jt < 0) | (jt <= lim[j])) &
-                          !(fmaf(__uint_as_float(sv[o][j]), P.scale_log2, -mr[j]) <= kTcRaise);
+                exceed |= ((jt < 0) | (jt <= lim[j])) & !(__uint_as_float(sv[o][j]) <= kTcRaise);
             }
           }
           exceed &= kvalid;
@@ -643,6 +647,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
             float v[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = -INFINITY;
+            // the raw scores again (the S^T buffer is still this tile's)
+#pragma unroll
+            for (int o = 0; o < NO; ++o) tc_ld8(sv[o], tmem + sb * N + lane_sel + r0 + o * 8);
+            tc_wait_ld();
 #pragma unroll
             for (int o = 0; o < NO; ++o) {
               int lim[8];
@@ -686,10 +694,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           }
 #pragma unroll
           for (int o = 0; o < NO; ++o) {
-            float al[8];
+            float al[8], mr[8];
             tc_lds8(al, sh.alpha + r0 + o * 8);
+            tc_lds8(mr, sh.m_ref + r0 + o * 8);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) l_part[o * 8 + j] *= al[j];
+            for (int j = 0; j < 8; ++j) {
+              l_part[o * 8 + j] *= al[j];
+              sv[o][j] = __float_as_uint(fmaf(__uint_as_float(sv[o][j]), P.scale_log2, -mr[j]));  // against the new m
+            }
           }
         }
         // ---- pass 2: P = exp2(S - m) as two bf16 terms, into the dead K tile ------------------
@@ -701,11 +713,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           if (lane == 0) mbar_arrive(&sh.s_free[sb]);
 #pragma unroll
           for (int o = 0; o < NO; ++o) {
-            float mr[8];
-            tc_lds8(mr, sh.m_ref + r0 + o * 8);
             float p[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) p[j] = ex2(fmaf(__uint_as_float(sv[o][j]), P.scale_log2, -mr[j]));
+            for (int j = 0; j < 8; ++j) p[j] = ex2(__uint_as_float(sv[o][j]));
             if (tail_tile) {
               int lim[8];
               tc_lds8(lim, sh.row_lim + r0 + o * 8);
