@@ -296,6 +296,25 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     return in_place ? __float_as_uint(__ldg(A + i) + 0.f) : __float_as_uint(a[i]);
   };
   const int n4 = (n_loc + 3) >> 2;
+  // In-place passes read the row from global memory (L2) with four independent 16-byte loads per
+  // thread in flight: with one dependent load per iteration a CTA moved ~4 GB/s (latency-bound).
+  constexpr int kIpUnroll = 4;
+  auto load_keys4 = [&](int i4, unsigned int (&key)[4]) -> bool {  // keys of positions 4*i4 .. 4*i4+3
+    const bool act = i4 < n4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (act) {
+      v = __ldg(reinterpret_cast<const float4*>(A) + i4);
+      const int left = n_loc - 4 * i4;
+      if (left < 4) v.w = 0.f;
+      if (left < 3) v.z = 0.f;
+      if (left < 2) v.y = 0.f;
+    }
+    key[0] = __float_as_uint(v.x + 0.f);  // -0.0 reads as +0.0
+    key[1] = __float_as_uint(v.y + 0.f);
+    key[2] = __float_as_uint(v.z + 0.f);
+    key[3] = __float_as_uint(v.w + 0.f);
+    return act;
+  };
   const int n_pos4 = n4 * 4;                       // slice length rounded up to whole float4s
   const int n_chunks = (n_pos4 + kChunk - 1) / kChunk;
   // selection at chunk granularity: the searched row (one score per chunk) is built after the
@@ -333,26 +352,22 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   bool bad = false;
   if (in_place) {
     // single contributing row: one pass over the slice for validity and the level-1 histogram
-    for (int base = 0; base < n4; base += kThreads) {
-      const int i4 = base + tid;
-      const bool act = i4 < n4;
-      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (act) {
-        v = __ldg(reinterpret_cast<const float4*>(A) + i4);
-        const int left = n_loc - 4 * i4;
-        if (left < 4) v.w = 0.f;
-        if (left < 3) v.z = 0.f;
-        if (left < 2) v.y = 0.f;
-        bad |= !(v.x >= 0.f && v.x <= FLT_MAX) | !(v.y >= 0.f && v.y <= FLT_MAX) |
-               !(v.z >= 0.f && v.z <= FLT_MAX) | !(v.w >= 0.f && v.w <= FLT_MAX);
-      }
-      const float vals[4] = {v.x + 0.f, v.y + 0.f, v.z + 0.f, v.w + 0.f};
-      if (kVariant && !chunked) vmax = fmaxf(vmax, fmaxf(fmaxf(vals[0], vals[1]), fmaxf(vals[2], vals[3])));
+    for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
+      unsigned int key[kIpUnroll][4];
+      bool act[kIpUnroll];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const unsigned int key = __float_as_uint(vals[e]);
-        const bool take = act && (4 * i4 + e < n_loc) && key != 0u && !(key >> 31) && !chunked;
-        hist_add(h1, take, static_cast<int>(key >> 20), mantissa_of(key));
+      for (int uu = 0; uu < kIpUnroll; ++uu) act[uu] = load_keys4(base + uu * kThreads + tid, key[uu]);
+#pragma unroll
+      for (int uu = 0; uu < kIpUnroll; ++uu) {
+        const int i4 = base + uu * kThreads + tid;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float x = __uint_as_float(key[uu][e]);
+          bad |= act[uu] && !(x >= 0.f && x <= FLT_MAX);  // negative, NaN or infinite
+          if (kVariant && !chunked) vmax = fmaxf(vmax, x);
+          const bool take = act[uu] && (4 * i4 + e < n_loc) && key[uu][e] != 0u && !(key[uu][e] >> 31) && !chunked;
+          hist_add(h1, take, static_cast<int>(key[uu][e] >> 20), mantissa_of(key[uu][e]));
+        }
       }
     }
   } else
@@ -535,6 +550,23 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     if (searching) {
       // only the elements inside the threshold bin take part
       const Hist hr = {lb, lb + kL23Bins};
+      if (in_place) {
+        for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
+          unsigned int key[kIpUnroll][4];
+          bool act[kIpUnroll];
+#pragma unroll
+          for (int uu = 0; uu < kIpUnroll; ++uu) act[uu] = load_keys4(base + uu * kThreads + tid, key[uu]);
+#pragma unroll
+          for (int uu = 0; uu < kIpUnroll; ++uu) {
+            const int i4 = base + uu * kThreads + tid;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const bool take = act[uu] && (4 * i4 + e < n_loc) && (key[uu][e] >> (shift + 10)) == prefix;
+              hist_add(hr, take, static_cast<int>((key[uu][e] >> shift) & 1023u), mantissa_of(key[uu][e]));
+            }
+          }
+        }
+      } else
       for (int base = 0; base < n_srch; base += kThreads) {
         const int i = base + tid;
         unsigned int key = 0u;
@@ -614,8 +646,30 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     return key_at(i) >= theta_key;
   };
   auto n_pos = [&](int i) -> int { return chunked ? min(P.chunk, n_loc - i * P.chunk) : 1; };
+  // a row read in place: per-warp ranges of whole float4s, four loads per lane in flight
+  const int wchunk4 = (((n4 + kWarps - 1) / kWarps) + 31) & ~31;
+  const int w4_lo = min(n4, warp * wchunk4);
+  const int w4_hi = min(n4, w4_lo + wchunk4);
   int wc = 0;
-  if (!invalid) {
+  if (!invalid && in_place) {
+    for (int i0 = w4_lo; i0 < w4_hi; i0 += 32 * kIpUnroll) {
+      unsigned int key[kIpUnroll][4];
+      bool act[kIpUnroll];
+#pragma unroll
+      for (int uu = 0; uu < kIpUnroll; ++uu) {
+        const int i4 = i0 + uu * 32 + lane;
+        act[uu] = load_keys4(i4 < w4_hi ? i4 : n4, key[uu]);
+      }
+      int c = 0;
+#pragma unroll
+      for (int uu = 0; uu < kIpUnroll; ++uu) {
+        const int i4 = i0 + uu * 32 + lane;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) c += (act[uu] && 4 * i4 + e < n_loc && key[uu][e] >= theta_key) ? 1 : 0;
+      }
+      wc += __reduce_add_sync(kFull, c);
+    }
+  } else if (!invalid) {
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
       const int i = i0 + lane;
       const bool keep = i < w_hi && kept(i);
@@ -641,7 +695,43 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     if (r < rank) offset += c;
     count += c;
   }
-  if (!invalid) {
+  if (!invalid && in_place) {
+    int* out = P.idx + out_list * P.idx_stride;
+    long long pos = offset + sh.warp_cnt[warp];
+    const unsigned int lt = (1u << lane) - 1u;
+    for (int i0 = w4_lo; i0 < w4_hi; i0 += 32 * kIpUnroll) {
+      unsigned int key[kIpUnroll][4];
+      bool act[kIpUnroll];
+#pragma unroll
+      for (int uu = 0; uu < kIpUnroll; ++uu) {
+        const int i4 = i0 + uu * 32 + lane;
+        act[uu] = load_keys4(i4 < w4_hi ? i4 : n4, key[uu]);
+      }
+#pragma unroll
+      for (int uu = 0; uu < kIpUnroll; ++uu) {
+        // 128 consecutive positions, four per lane: ascending order is lane-major
+        const int i4 = i0 + uu * 32 + lane;
+        bool keep[4];
+        unsigned int before = 0, total_kept = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          keep[e] = act[uu] && 4 * i4 + e < n_loc && key[uu][e] >= theta_key;
+          const unsigned int m = __ballot_sync(kFull, keep[e]);
+          before += __popc(m & lt);
+          total_kept += __popc(m);
+        }
+        long long my = pos + before;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (keep[e]) {
+            if (my < P.idx_stride) out[my] = lo + 4 * i4 + e;
+            ++my;
+          }
+        }
+        pos += total_kept;
+      }
+    }
+  } else if (!invalid) {
     int* out = P.idx + out_list * P.idx_stride;
     long long pos = offset + sh.warp_cnt[warp];
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
@@ -765,7 +855,15 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   P.chunk = (A.chunk > 1) ? A.chunk : 1;
   if (P.chunk > 1) P.single_row = 0;  // chunk scores live in the shared-memory slice
   const bool variant = P.per_step || P.bisect_iters > 0 || P.chunk > 1;
-  const int cs = specattn::pick_cluster(A.L_stride, n_lists);
+  int cs = specattn::pick_cluster(A.L_stride, n_lists);
+  if (P.single_row) {
+    // A row read in place needs no shared-memory slice, so the cluster only has to keep a slice
+    // below 2^16 positions (the 16-bit halves of the mantissa sums must not wrap) and to fill
+    // the GPU: with hundreds of rows, one or two CTAs per row avoid most cluster barriers.
+    cs = 1;
+    while (cs < 8 && (A.L_stride + cs - 1) / cs > 65536) cs *= 2;
+    while (cs < 8 && n_lists * cs < 296) cs *= 2;
+  }
   const long long s_align = (P.chunk > 4) ? P.chunk : 4;
   const long long slice = P.single_row ? 0 : (((A.L_stride + cs - 1) / cs) + s_align - 1) / s_align * s_align;
   if (slice > specattn::kSliceCap) return SPECATTN_ERR_UNSUPPORTED;
