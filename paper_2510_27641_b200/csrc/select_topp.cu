@@ -95,7 +95,6 @@ struct Hist {
 struct Shared {
   unsigned int h_lo[kL1Bins];  // level-1 histogram of this CTA
   unsigned int h_hi[kL1Bins];
-  long long row_off[SPECATTN_MAX_ROWS_PER_LIST];  // element offset of each contributing row, in add order
   double grp_mass[kL1Bins / kGroup];
   int warp_cnt[kWarps];
   int n_rows;
@@ -256,7 +255,11 @@ template <bool kInPlace, bool kVariant>
 __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel(const __grid_constant__ SelectParams P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   Shared& sh = *reinterpret_cast<Shared*>(smem_raw);
-  float* a = reinterpret_cast<float*>(smem_raw + ((sizeof(Shared) + 127) / 128) * 128);
+  // behind the fixed part: the element offset of each contributing row, in add order (a row
+  // read in place is its list's only row, at offset 0, and has no such table), then the slice
+  long long* const row_off = reinterpret_cast<long long*>(smem_raw + ((sizeof(Shared) + 127) / 128) * 128);
+  float* a = reinterpret_cast<float*>(smem_raw + ((sizeof(Shared) + 127) / 128) * 128 +
+                                      (kInPlace ? 0 : SPECATTN_MAX_ROWS_PER_LIST * sizeof(long long)));
 
   cg::cluster_group cluster = cg::this_cluster();
   const int cs = static_cast<int>(cluster.num_blocks());
@@ -296,9 +299,9 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     return in_place ? __float_as_uint(__ldg(A + i) + 0.f) : __float_as_uint(a[i]);
   };
   const int n4 = (n_loc + 3) >> 2;
-  // In-place passes read the row from global memory (L2) with four independent 16-byte loads per
+  // In-place passes read the row from global memory (L2) with eight independent 16-byte loads per
   // thread in flight: with one dependent load per iteration a CTA moved ~4 GB/s (latency-bound).
-  constexpr int kIpUnroll = 4;
+  constexpr int kIpUnroll = 8;
   auto load_keys4 = [&](int i4, unsigned int (&key)[4]) -> bool {  // keys of positions 4*i4 .. 4*i4+3
     const bool act = i4 < n4;
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -333,12 +336,16 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   // contributing rows in the order that defines the aggregated value
   if (tid == 0) {
     int n = 0;
-    for (int h = 0; h < P.H; ++h) {
-      if (P.has_groups && P.head_group[h] != g) continue;
-      if (kVariant && P.per_step) {
-        sh.row_off[n++] = static_cast<long long>(h * P.gamma + step) * P.L_stride;
-      } else {
-        for (int s = 0; s < P.gamma; ++s) sh.row_off[n++] = static_cast<long long>(h * P.gamma + s) * P.L_stride;
+    if (kInPlace) {
+      n = 1;
+    } else {
+      for (int h = 0; h < P.H; ++h) {
+        if (P.has_groups && P.head_group[h] != g) continue;
+        if (kVariant && P.per_step) {
+          row_off[n++] = static_cast<long long>(h * P.gamma + step) * P.L_stride;
+        } else {
+          for (int s = 0; s < P.gamma; ++s) row_off[n++] = static_cast<long long>(h * P.gamma + s) * P.L_stride;
+        }
       }
     }
     sh.n_rows = n;
@@ -383,7 +390,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     auto issue = [&]() {
       if (ic < n_chunks) {
         const int len4 = min(kChunk, n_pos4 - ic * kChunk) >> 2;
-        const float* src = src0 + sh.row_off[ir] + ic * kChunk;
+        const float* src = src0 + row_off[ir] + ic * kChunk;
         const uint32_t dst = ring_addr + islot * (kChunk * 4);
 #pragma unroll
         for (int k = 0; k < 2; ++k)
@@ -870,7 +877,8 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   // shared memory: fixed part, the aggregated slice, then the per-thread staging ring
   // (kDepth pieces of 8 KB; it later hosts the scan arrays).  Small slices leave room for two
   // CTAs per SM.
-  const size_t fixed = ((sizeof(specattn::Shared) + 127) / 128) * 128;
+  const size_t fixed = ((sizeof(specattn::Shared) + 127) / 128) * 128 +
+                       (P.single_row ? 0 : SPECATTN_MAX_ROWS_PER_LIST * sizeof(long long));
   const size_t slice_bytes = static_cast<size_t>((slice + 31) / 32 * 32) * sizeof(float);
   // (a single-row list keeps nothing but the 32 KB of scan arrays behind the fixed part)
   const size_t smem = fixed + slice_bytes +
