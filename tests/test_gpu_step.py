@@ -212,3 +212,41 @@ def test_full_size_sampled_outputs(which):
         gl = step.lse[j][b, :, hk * grp:(hk + 1) * grp].reshape(-1)
         check_attention(go, gl, ro, rl)
     assert int(step.status.abs().sum()) == 0
+
+
+@pytest.mark.parametrize("engine", ["default", "mma_sync"])
+def test_full_size_dense_baseline_of_config4(engine):
+    """Config 4's p = 1 baseline at full size: 4 sequences x 131072 positions, 64 q / 8 kv heads,
+    gamma = 4 (40 query rows per KV head).  The default engine choice for this shape is the
+    tcgen05 kernel; the other run forces mma.sync.  Sampled (sequence, kv head) units are
+    recomputed by the oracle over all 131072 positions, with K/V regenerated on the CPU."""
+    import paper_2510_27641_b200 as sa
+    from paper_2510_27641_b200.step import VerifyStep
+    cfg = wl.config4(n_target_layers=1, p=1.0)
+    si = wl.make_step_inputs(cfg)
+    pools = [wl.kv_pool(cfg.seed, 0, si.n_pages, cfg.page_size, cfg.n_kv_heads, cfg.head_dim, device=dev())]
+    flags = 0 if engine == "default" else sa.VERIFY_ENGINE_MMA_SYNC
+    step = VerifyStep(layer_map=[-1], n_draft_layers=cfg.n_draft_layers, batch=cfg.batch,
+                      n_draft_heads=cfg.n_draft_heads, gamma=cfg.gamma, L_stride=si.L_stride,
+                      n_q_heads=cfg.n_q_heads, p=1.0, kv_pools=pools, kv_len=to_dev(si.kv_len),
+                      block_table=to_dev(si.block_table), pages_per_seq=si.pages_per_seq, verify_flags=flags)
+    step.load_inputs([None] * cfg.n_draft_layers, [bf16.bits_to_torch(si.q[0])])
+    step.run()
+    torch.cuda.synchronize()
+    assert int(step.status.abs().sum()) == 0
+    sp, sk, ss, sh = wl.kv_strides(cfg.page_size, cfg.n_kv_heads, cfg.head_dim)
+    grp, d, L = cfg.n_q_heads // cfg.n_kv_heads, cfg.head_dim, cfg.ctx
+    rng = np.random.default_rng(1)
+    for _ in range(2):
+        b, hk = int(rng.integers(0, cfg.batch)), int(rng.integers(0, cfg.n_kv_heads))
+        pos = np.arange(L, dtype=np.int64)
+        page = si.block_table[b, pos // cfg.page_size].astype(np.int64)
+        base = page * sp + (pos % cfg.page_size) * ss + hk * sh
+        flat = torch.from_numpy(base)[:, None] + torch.arange(d)[None, :]
+        K = bf16.torch_to_bits(wl.kv_values(cfg.seed, 0, flat))
+        V = bf16.torch_to_bits(wl.kv_values(cfg.seed, 0, flat + sk))
+        qrows = si.q[0][b][:, hk * grp:(hk + 1) * grp, :].reshape(-1, d)
+        ro, rl = oracle.attend_rows(qrows, K, V)
+        go = step.out[0][b, :, hk * grp:(hk + 1) * grp, :].reshape(-1, d)
+        gl = step.lse[0][b, :, hk * grp:(hk + 1) * grp].reshape(-1)
+        check_attention(go, gl, ro, rl)
