@@ -122,6 +122,13 @@ __device__ __forceinline__ bool mbar_wait_cluster(unsigned long long* bar, uint3
   }
   return false;
 }
+// The two halves of a cluster barrier: arrive early, wait only where the peer's state is needed.
+__device__ __forceinline__ void cluster_arrive() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait() {
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }

@@ -292,9 +292,12 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   }
   fence_proxy_async();
   __syncthreads();
-  // launched as CTA pairs: the peer's barrier must exist before anyone can arrive on it
+  // Launched as CTA pairs: the peer's barrier must exist before anyone can arrive on it.  Only
+  // the arrival happens here; every thread waits for the peer's arrival where it first needs
+  // it (the consumers before their first combine, everybody else before leaving), so that the
+  // barrier costs nothing on the way to the first copy.
   const bool paired = (MT <= 2) && (cluster_num_ctas() == 2);
-  if (paired) cluster_sync_all();
+  if (paired) cluster_arrive();
   if (warp == 0) {  // inclusive scan of the atom counts, 32 at a time
     int carry = 0;
     for (int base = 0; base < U; base += 32) {
@@ -329,10 +332,10 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     if (atoms > 0) {
 #pragma unroll
       for (int c = 0; c < kCandidates; ++c) {
-        // share_c = (N / G) * (1 + c / 16)
-        const long long num = static_cast<long long>(atoms) * G * 16;
-        const long long den = N * (16 + c);
-        int k = static_cast<int>((2 * num + den) / (2 * den));  // round to nearest
+        // share_c = (N / G) * (1 + c / 16); 32-bit: atoms <= 12288, G ~ 148, N <= 2048 * 12288
+        const unsigned int num = static_cast<unsigned int>(atoms) * G * 16u;
+        const unsigned int den = static_cast<unsigned int>(N) * (16u + c);
+        int k = static_cast<int>((2u * num + den) / (2u * den));  // round to nearest
         if (k < 1) k = 1;
         if (k > atoms) k = atoms;
         atomicAdd(&sh.cand_parts[c], k);
@@ -358,9 +361,9 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       if (u < U) {
         const int atoms = sh.unit_start[u + 1] - sh.unit_start[u];
         if (atoms > 0) {
-          const long long num = static_cast<long long>(atoms) * G * 16;
-          const long long den = N * (16 + cand);
-          k = static_cast<int>((2 * num + den) / (2 * den));
+          const unsigned int num = static_cast<unsigned int>(atoms) * G * 16u;
+          const unsigned int den = static_cast<unsigned int>(N) * (16u + cand);
+          k = static_cast<int>((2u * num + den) / (2u * den));
           if (k < 1) k = 1;
           if (k > atoms) k = atoms;
         }
@@ -393,7 +396,10 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       }
     }
   }
-  if (static_cast<long long>(blockIdx.x) >= NP) return;
+  if (static_cast<long long>(blockIdx.x) >= NP) {
+    if (paired) cluster_wait();
+    return;
+  }
   int a0, a1;
   if (aligned) {
     int lo = 0, hi = U - 1;  // unit whose CTA range holds this CTA
@@ -403,9 +409,9 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     }
     const int k = sh.part_start[lo + 1] - sh.part_start[lo];
     const int j = static_cast<int>(blockIdx.x) - sh.part_start[lo];
-    const long long atoms = sh.unit_start[lo + 1] - sh.unit_start[lo];
-    a0 = sh.unit_start[lo] + static_cast<int>(j * atoms / k);
-    a1 = sh.unit_start[lo] + static_cast<int>((j + 1) * atoms / k);
+    const int atoms = sh.unit_start[lo + 1] - sh.unit_start[lo];  // j < k <= G: the products fit 32 bits
+    a0 = sh.unit_start[lo] + j * atoms / k;
+    a1 = sh.unit_start[lo] + (j + 1) * atoms / k;
   } else {
     a0 = cta_first_atom(blockIdx.x, N, NP);
     a1 = cta_first_atom(blockIdx.x + 1, N, NP);
@@ -545,6 +551,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       // give this warp's last copies a bounded chance to land before the CTA retires
       mbar_wait(&sh.full[last_it % kStages], (last_it / kStages) & 1u, nullptr);
     }
+    if (paired) cluster_wait();
     return;
   }
 
@@ -565,6 +572,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   int it = 0, seg = 0;
   int a = a0, u = u_first;
   bool ok = true;
+  bool peer_seen = false;
   while (a < a1) {
     const int us = sh.unit_start[u], ue = sh.unit_start[u + 1];
     const int seg_hi = min(a1, ue);
@@ -618,6 +626,10 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     }
 
     // ---- end of the segment: row sums across the quad, then combine the slab's warps ---------
+    if (paired && !peer_seen) {  // the peer's arrival at kernel start: long past by now
+      cluster_wait();
+      peer_seen = true;
+    }
     float m0 = st.m0, m1 = st.m1, l0 = st.l0, l1 = st.l1;
     float (&acc)[16][4] = st.acc;
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
@@ -785,6 +797,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       while (u < U && sh.unit_start[u + 1] == sh.unit_start[u]) ++u;
     }
   }
+  if (paired && !peer_seen) cluster_wait();
   if (!ok && P.status && lane == 0) atomicOr(P.status, SPECATTN_ROW_TIMEOUT);
 }
 
