@@ -231,6 +231,7 @@ typedef struct specattn_verify_args {
   size_t workspace_bytes;
   uint32_t flags;        /* SPECATTN_VERIFY_* bits, 0 for none */
   int32_t tail_len;      /* in-flight tokens attended causally after the list, 0 <= tail_len <= 64 */
+  const void* plan;      /* optional: a work partition made by specattn_verify_plan, or NULL */
 } specattn_verify_args;
 
 /* Bytes of workspace specattn_sparse_verify needs for these shapes on the current device
@@ -242,6 +243,21 @@ size_t specattn_verify_workspace_bytes(const specattn_verify_args* args);
 int specattn_verify_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 int specattn_sparse_verify(const specattn_verify_args* args, void* cuda_stream);
+
+/* specattn_verify_plan -- the work partition of a verify launch, computed ahead of it.
+ *
+ * Not an operation of the paper: an engineering shortcut of this implementation.  How the kernel
+ * deals its (sequence, kv head) lists to the SMs depends only on the list lengths (counts, or
+ * kv_len for dense calls), tail_len, the shapes and the GPU -- not on q, the K/V pool or the
+ * outputs.  Target layers that share a draft layer's lists therefore share the partition, and a
+ * verify kernel that finds a matching plan in args->plan skips computing it (a few microseconds
+ * of start-up per launch).  `plan` is a device buffer of specattn_verify_plan_bytes(args) bytes,
+ * 16-byte aligned, written by a small kernel on the stream (after whatever produces counts /
+ * kv_len, e.g. specattn_select_topp) and valid until those change.  A kernel given a plan that
+ * does not fit its launch (other batch, heads, tail_len, dense flag or GPU) ignores it.  Only
+ * the mma.sync engine reads plans. */
+size_t specattn_verify_plan_bytes(const specattn_verify_args* args);
+int specattn_verify_plan(const specattn_verify_args* args, void* plan, size_t plan_bytes, void* cuda_stream);
 
 /* ========================================================================================
  * specattn_sparse_verify_static -- specattn_sparse_verify for callers that cannot allocate.
@@ -291,7 +307,8 @@ int specattn_sparse_verify_static(const specattn_verify_args* args, void* cuda_s
  * and finally makes the caller's stream wait for both copy streams: work enqueued on that
  * stream afterwards sees the step complete.  The two copy streams and the events between the
  * lanes are created on the first call per device and kept; one call at a time enqueues per
- * device.  select.n_target_layers must equal n_target_layers.
+ * device.  select.n_target_layers must equal n_target_layers.  Where verify[j].plan is set, the
+ * call runs specattn_verify_plan into it before the first layer that points at it.
  * `select` and `verify[j]` are complete device-side argument structs (their device buffers,
  * including the staging buffers the copies land in, are the caller's); verify[j].idx/counts
  * must already point at the lists of layer_map[j] (or dense be set where layer_map[j] < 0).

@@ -16,7 +16,8 @@ __all__ = ["select_topp", "sparse_verify", "sparse_verify_static", "verify_works
            "verify_step_host", "status_string", "kernel_launch_count", "library_path",
            "SelectArgs", "VerifyArgs", "StepHostArgs", "lib", "SpecAttnError",
            "ROW_OK", "ROW_INVALID_PROB", "ROW_OVERFLOW", "ROW_BAD_INDEX", "ROW_TIMEOUT",
-           "VERIFY_LISTS_STABLE", "VERIFY_ENGINE_MMA_SYNC", "VERIFY_ENGINE_TCGEN05"]
+           "VERIFY_LISTS_STABLE", "VERIFY_ENGINE_MMA_SYNC", "VERIFY_ENGINE_TCGEN05", "verify_plan",
+           "verify_plan_buffer"]
 
 ROW_OK, ROW_INVALID_PROB, ROW_OVERFLOW, ROW_BAD_INDEX, ROW_TIMEOUT = 0, 1, 2, 4, 8
 VERIFY_LISTS_STABLE = 1
@@ -56,7 +57,7 @@ class VerifyArgs(C.Structure):
                 ("idx_stride", C.c_int64), ("counts", C.c_void_p), ("sm_scale", C.c_float),
                 ("out", C.c_void_p), ("lse", C.c_void_p), ("status", C.c_void_p),
                 ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("flags", C.c_uint32),
-                ("tail_len", C.c_int32)]
+                ("tail_len", C.c_int32), ("plan", C.c_void_p)]
 
 
 class StepHostArgs(C.Structure):
@@ -86,6 +87,10 @@ def lib() -> C.CDLL:
         L.specattn_verify_workspace_bytes.restype = C.c_size_t
         L.specattn_verify_workspace_init.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
         L.specattn_verify_workspace_init.restype = C.c_int
+        L.specattn_verify_plan_bytes.argtypes = [C.POINTER(VerifyArgs)]
+        L.specattn_verify_plan_bytes.restype = C.c_size_t
+        L.specattn_verify_plan.argtypes = [C.POINTER(VerifyArgs), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.specattn_verify_plan.restype = C.c_int
         L.specattn_sparse_verify_static.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
         L.specattn_sparse_verify_static.restype = C.c_int
         L.specattn_verify_step_host.argtypes = [C.POINTER(StepHostArgs), C.c_void_p]
@@ -269,6 +274,24 @@ def sparse_verify(q: torch.Tensor, kv_pages: torch.Tensor, kv_len: torch.Tensor,
     if rc != 0:
         raise SpecAttnError(rc, "specattn_sparse_verify")
     return out, lse, status
+
+
+def verify_plan_buffer(args: VerifyArgs, device=None) -> torch.Tensor:
+    """A device buffer large enough for the work partition of launches shaped like ``args``."""
+    n = int(lib().specattn_verify_plan_bytes(C.byref(args)))
+    if n == 0:
+        raise SpecAttnError(-6, "specattn_verify_plan_bytes")
+    dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+    return torch.zeros((n + 3) // 4, dtype=torch.int32, device=dev)
+
+
+def verify_plan(args: VerifyArgs, plan: torch.Tensor, stream=None) -> None:
+    """specattn_verify_plan: computes the work partition of launches shaped like ``args`` (same
+    lists / kv_len, tail_len, shapes) into ``plan``; point ``args.plan`` at it afterwards."""
+    rc = lib().specattn_verify_plan(C.byref(args), plan.data_ptr(), plan.numel() * plan.element_size(),
+                                    _stream_ptr(stream))
+    if rc != 0:
+        raise SpecAttnError(rc, "specattn_verify_plan")
 
 
 def sparse_verify_static(args: VerifyArgs, stream=None) -> None:

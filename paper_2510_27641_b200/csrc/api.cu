@@ -195,6 +195,8 @@ extern "C" int specattn_verify_step_host(const specattn_step_host_args* args, vo
   // the caller's stream: selection per draft layer when first needed, then the verify launches
   if (!ok(cudaStreamWaitEvent(stream, pipe.q_in, 0))) return SPECATTN_ERR_CUDA;
   bool selected[SPECATTN_MAX_DRAFT_LAYERS] = {false};
+  const void* planned[SPECATTN_MAX_DRAFT_LAYERS + 1];
+  int n_planned = 0;
   for (int j = 0; j < S.n_target_layers; ++j) {
     const int u = sel.layer_map[j];
     if (u >= 0 && !selected[u]) {
@@ -208,6 +210,16 @@ extern "C" int specattn_verify_step_host(const specattn_step_host_args* args, vo
       if (rc != SPECATTN_OK) return rc;
     }
     const specattn_verify_args& v = S.verify[j];
+    // a work partition that several layers share is computed before its first user
+    if (v.plan != nullptr) {
+      bool done = false;
+      for (int k = 0; k < n_planned && !done; ++k) done = planned[k] == v.plan;
+      if (!done) {
+        const int prc = specattn_verify_plan(&v, const_cast<void*>(v.plan), specattn_verify_plan_bytes(&v), cuda_stream);
+        if (prc != SPECATTN_OK) return prc;
+        if (n_planned < SPECATTN_MAX_DRAFT_LAYERS + 1) planned[n_planned++] = v.plan;
+      }
+    }
     const int rc = specattn_sparse_verify(&v, cuda_stream);
     if (rc != SPECATTN_OK) return rc;
     // lane "out"

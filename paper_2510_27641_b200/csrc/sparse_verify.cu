@@ -80,6 +80,7 @@ struct VerifyParams {
   int lists_stable;  // SPECATTN_VERIFY_LISTS_STABLE
   int tail;          // in-flight tokens appended to every unit, attended causally
   int tail_off;      // tail - T: query t may see tail tokens j <= t + tail_off
+  const int* plan;   // precomputed work partition (specattn_verify_plan) or nullptr
 };
 
 // WPM = consumer warps per 16-row slab: 4 -> (stage parity, 32-key half), 2 -> (stage parity).
@@ -134,6 +135,152 @@ __device__ __forceinline__ void merge_scales(float m, float im, float& mn, float
   const float base = (mn == -INFINITY) ? 0.f : mn;
   a_old = ex2(m - base);   // ex2(-inf) = 0
   a_in = ex2(im - base);
+}
+
+// ---- precomputed work partition ("plan") ------------------------------------------------------
+// The partition of a launch depends only on the list lengths, the shapes and the grid: target
+// layers that share a draft layer's lists share it.  A plan holds, as int32:
+//   [0] magic  [1] U  [2] grid  [3] aligned  [4] NP  [5] N (atoms)  [6] tail  [7] dense
+//   unit_start[U + 1], unit_cnt[U], part_start[U + 1], then (a0, a1, u_first) per CTA
+// A kernel whose launch does not match the header ignores the plan and partitions itself.
+constexpr int kPlanMagic = 0x5a17a9e1;
+constexpr int kPlanHeader = 8;
+__host__ __device__ inline size_t plan_ints(int U, int grid) {
+  return static_cast<size_t>(kPlanHeader) + (U + 1) + U + (U + 1) + 3 * static_cast<size_t>(grid);
+}
+
+// One CTA computes what every CTA of a verify launch would compute for itself at start-up.
+__global__ void __launch_bounds__(256, 1) verify_plan_kernel(const __grid_constant__ VerifyParams P, int* plan, int G) {
+  __shared__ int unit_start[kMaxUnits + 1];
+  __shared__ int part_start[kAlignedMaxUnits + 1];
+  __shared__ int cand_parts[kCandidates], cand_max[kCandidates];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int U = P.B * P.Hkv;
+  pdl_wait();              // the lists are the previous kernel's output
+  pdl_launch_dependents();
+  int* const p_us = plan + kPlanHeader;
+  int* const p_cnt = p_us + (U + 1);
+  int* const p_ps = p_cnt + U;
+  int* const p_cta = p_ps + (U + 1);
+  if (tid == 0) unit_start[0] = 0;
+  for (int u = tid; u < U; u += 256) {
+    const int c = unit_count(P, u);
+    p_cnt[u] = c;
+    unit_start[u + 1] = (c + kAtom - 1) / kAtom;
+  }
+  if (tid < kCandidates) { cand_parts[tid] = 0; cand_max[tid] = 0; }
+  __syncthreads();
+  if (warp == 0) {
+    int carry = 0;
+    for (int base = 0; base < U; base += 32) {
+      const int u = base + lane;
+      int v = (u < U) ? unit_start[u + 1] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += n;
+      }
+      if (u < U) unit_start[u + 1] = v + carry;
+      carry += __shfl_sync(0xffffffffu, v, 31);
+    }
+  }
+  __syncthreads();
+  const long long N = unit_start[U];
+  const bool try_aligned = (U <= kAlignedMaxUnits) && (N > 0);
+  if (try_aligned && tid < U) {
+    const int atoms = unit_start[tid + 1] - unit_start[tid];
+    if (atoms > 0) {
+      for (int c = 0; c < kCandidates; ++c) {
+        const unsigned int num = static_cast<unsigned int>(atoms) * G * 16u;
+        const unsigned int den = static_cast<unsigned int>(N) * (16u + c);
+        int k = static_cast<int>((2u * num + den) / (2u * den));
+        if (k < 1) k = 1;
+        if (k > atoms) k = atoms;
+        atomicAdd(&cand_parts[c], k);
+        atomicMax(&cand_max[c], (atoms + k - 1) / k);
+      }
+    }
+  }
+  __syncthreads();
+  int cand = -1;
+  if (try_aligned) {
+    for (int c = 0; c < kCandidates; ++c)
+      if (cand_parts[c] <= G) { cand = c; break; }
+    if (cand >= 0 && static_cast<long long>(cand_max[cand]) * G > N + 24ll * G) cand = -1;
+  }
+  const bool aligned = cand >= 0;
+  if (aligned && warp == 0) {
+    int carry = 0;
+    for (int base = 0; base < U; base += 32) {
+      const int u = base + lane;
+      int k = 0;
+      if (u < U) {
+        const int atoms = unit_start[u + 1] - unit_start[u];
+        if (atoms > 0) {
+          const unsigned int num = static_cast<unsigned int>(atoms) * G * 16u;
+          const unsigned int den = static_cast<unsigned int>(N) * (16u + cand);
+          k = static_cast<int>((2u * num + den) / (2u * den));
+          if (k < 1) k = 1;
+          if (k > atoms) k = atoms;
+        }
+      }
+      int v = k;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += n;
+      }
+      if (u < U) part_start[u + 1] = v + carry;
+      if (base == 0 && lane == 0) part_start[0] = 0;
+      carry += __shfl_sync(0xffffffffu, v, 31);
+    }
+  }
+  __syncthreads();
+  const long long NP = aligned ? part_start[U] : ((N < G) ? N : static_cast<long long>(G));
+  for (int u = tid; u <= U; u += 256) {
+    p_us[u] = unit_start[u];
+    p_ps[u] = aligned ? part_start[u] : 0;
+  }
+  for (int i = tid; i < G; i += 256) {
+    int a0 = 0, a1 = 0, u_first = 0;
+    if (i < NP) {
+      if (aligned) {
+        int lo = 0, hi = U - 1;
+        while (lo < hi) {
+          const int mid = (lo + hi + 1) >> 1;
+          if (part_start[mid] <= i) lo = mid; else hi = mid - 1;
+        }
+        const int k = part_start[lo + 1] - part_start[lo];
+        const int j = i - part_start[lo];
+        const int atoms = unit_start[lo + 1] - unit_start[lo];
+        a0 = unit_start[lo] + j * atoms / k;
+        a1 = unit_start[lo] + (j + 1) * atoms / k;
+      } else {
+        a0 = cta_first_atom(i, N, NP);
+        a1 = cta_first_atom(i + 1, N, NP);
+      }
+      int lo = 0, hi = U - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (unit_start[mid] <= a0) lo = mid; else hi = mid - 1;
+      }
+      u_first = lo;
+      while (unit_start[u_first + 1] <= a0) ++u_first;
+    }
+    p_cta[3 * i] = a0;
+    p_cta[3 * i + 1] = a1;
+    p_cta[3 * i + 2] = u_first;
+  }
+  if (tid == 0) {
+    plan[1] = U;
+    plan[2] = G;
+    plan[3] = aligned ? 1 : 0;
+    plan[4] = static_cast<int>(NP);
+    plan[5] = static_cast<int>(N);
+    plan[6] = P.tail;
+    plan[7] = P.dense;
+    plan[0] = kPlanMagic;
+  }
 }
 
 // Online-softmax state of one warp: rows g and g+8 of its 16-row slab, 128 output columns.
@@ -285,10 +432,26 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     sh.abort_flag = 0;
     sh.unit_start[0] = 0;
   }
-  for (int u = tid; u < U; u += NT) {
-    const int c = unit_count(P, u);
-    sh.unit_cnt[u] = c;
-    sh.unit_start[u + 1] = (c + kAtom - 1) / kAtom;
+  // A plan made for this launch (same units, grid, tail, dense flag) replaces the whole
+  // partition below by one coalesced copy.
+  const int* const plan = P.plan;
+  const bool planned = plan != nullptr && plan[0] == kPlanMagic && plan[1] == U &&
+                       plan[2] == static_cast<int>(gridDim.x) && plan[6] == P.tail && plan[7] == P.dense;
+  if (planned) {
+    const int* const p_us = plan + kPlanHeader;
+    const int* const p_cnt = p_us + (U + 1);
+    const int* const p_ps = p_cnt + U;
+    for (int u = tid; u <= U; u += NT) {
+      sh.unit_start[u] = p_us[u];
+      if (u < U) sh.unit_cnt[u] = p_cnt[u];
+      if (u <= kAlignedMaxUnits) sh.part_start[u] = p_ps[u];
+    }
+  } else {
+    for (int u = tid; u < U; u += NT) {
+      const int c = unit_count(P, u);
+      sh.unit_cnt[u] = c;
+      sh.unit_start[u + 1] = (c + kAtom - 1) / kAtom;
+    }
   }
   fence_proxy_async();
   __syncthreads();
@@ -298,6 +461,20 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   // barrier costs nothing on the way to the first copy.
   const bool paired = (MT <= 2) && (cluster_num_ctas() == 2);
   if (paired) cluster_arrive();
+  long long N;        // atoms of all units
+  bool aligned;       // which of the two partitions
+  long long NP;       // CTAs that get work
+  int a0 = 0, a1 = 0, u_first = 0;  // this CTA's atom range and the unit holding its first atom
+  const int G = static_cast<int>(gridDim.x);
+  if (planned) {
+    N = plan[5];
+    aligned = plan[3] != 0;
+    NP = plan[4];
+    const int* const p_cta = plan + kPlanHeader + (U + 1) + U + (U + 1) + 3 * blockIdx.x;
+    a0 = p_cta[0];
+    a1 = p_cta[1];
+    u_first = p_cta[2];
+  } else {
   if (warp == 0) {  // inclusive scan of the atom counts, 32 at a time
     int carry = 0;
     for (int base = 0; base < U; base += 32) {
@@ -321,8 +498,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   // largest exceeds the ideal share by no more than 24 atoms.  Otherwise "contiguous": the atoms of all units
   // laid end to end and cut into gridDim equal ranges, which balances any mix of list lengths
   // at the price of CTAs that straddle unit boundaries.
-  const long long N = sh.unit_start[U];
-  const int G = static_cast<int>(gridDim.x);
+  N = sh.unit_start[U];
   if (tid < kCandidates) { sh.cand_parts[tid] = 0; sh.cand_max[tid] = 0; }
   if (tid == 0) sh.aligned = 0;
   __syncthreads();
@@ -352,7 +528,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     // fixed few microseconds of extra merging, an oversized part costs time per atom
     if (cand >= 0 && static_cast<long long>(sh.cand_max[cand]) * G > N + 24ll * G) cand = -1;
   }
-  const bool aligned = cand >= 0;
+  aligned = cand >= 0;
   if (aligned && warp == 0) {  // first CTA of every unit: exclusive scan of k_u
     int carry = 0;
     for (int base = 0; base < U; base += 32) {
@@ -380,7 +556,8 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     }
   }
   __syncthreads();
-  const long long NP = aligned ? sh.part_start[U] : ((N < G) ? N : static_cast<long long>(G));
+  NP = aligned ? sh.part_start[U] : ((N < G) ? N : static_cast<long long>(G));
+  }  // !planned
   if (warp < NC) {
     // consumers are the only writers of global memory: from here on the previous kernel's
     // results (and its use of the shared workspace) are complete
@@ -400,7 +577,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     if (paired) cluster_wait();
     return;
   }
-  int a0, a1;
+  if (!planned) {
   if (aligned) {
     int lo = 0, hi = U - 1;  // unit whose CTA range holds this CTA
     while (lo < hi) {
@@ -418,7 +595,6 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   }
 
   // unit holding atom a0
-  int u_first;
   {
     int lo = 0, hi = U - 1;
     while (lo < hi) {
@@ -428,6 +604,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     u_first = lo;
     while (sh.unit_start[u_first + 1] <= a0) ++u_first;  // skip empty units that share the start
   }
+  }  // !planned
 
   if (warp >= NC) {
     // =========================== producer warps ===========================================
@@ -892,6 +1069,53 @@ size_t workspace_bytes_for(const specattn_verify_args& A, int n_ctas) {
 
 using specattn::VerifyParams;
 
+namespace specattn {
+namespace {
+// The kernel-side view of the arguments (everything except the workspace).
+VerifyParams make_params(const specattn_verify_args& A) {
+  VerifyParams P;
+  memset(&P, 0, sizeof(P));
+  P.B = A.batch;
+  P.T = A.n_q;
+  P.Hq = A.n_q_heads;
+  P.Hkv = A.n_kv_heads;
+  P.grp = A.n_q_heads / A.n_kv_heads;
+  P.M = P.T * P.grp;
+  P.G = A.n_groups;
+  P.dense = A.dense ? 1 : 0;
+  P.page_size = A.page_size;
+  P.page_shift = -1;
+  for (int s = 0; s < 31; ++s)
+    if ((1 << s) == A.page_size) P.page_shift = s;
+  P.q = static_cast<const __nv_bfloat16*>(A.q);
+  P.kv = static_cast<const __nv_bfloat16*>(A.kv_pages);
+  P.n_pages = A.n_pages;
+  P.s_page = A.stride_page;
+  P.s_kv = A.stride_kv;
+  P.s_slot = A.stride_slot;
+  P.s_head = A.stride_head;
+  P.bt = A.block_table;
+  P.bt_stride = A.block_table_stride;
+  P.kv_len = A.kv_len;
+  P.idx = A.idx;
+  P.idx_stride = A.idx_stride;
+  P.counts = A.counts;
+  const float scale = (A.sm_scale != 0.f) ? A.sm_scale : 1.0f / sqrtf(static_cast<float>(A.head_dim));
+  P.scale_log2 = scale * specattn::kLog2e;
+  P.out = A.out;
+  P.lse = A.lse;
+  P.status = A.status;
+  P.lists_stable = (A.flags & SPECATTN_VERIFY_LISTS_STABLE) ? 1 : 0;
+  P.tail = A.tail_len;
+  P.tail_off = A.tail_len - A.n_q;
+
+  P.plan = static_cast<const int*>(A.plan);
+  return P;
+}
+}  // namespace
+}  // namespace specattn
+
+
 extern "C" size_t specattn_verify_workspace_bytes(const specattn_verify_args* args) {
   if (specattn::validate(args) != SPECATTN_OK) return 0;
   const int n = specattn::device_sm_count();
@@ -926,42 +1150,8 @@ extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cu
   if (n_ctas <= 0) return SPECATTN_ERR_CUDA;
   if (A.workspace_bytes < specattn::workspace_bytes_for(A, n_ctas)) return SPECATTN_ERR_WORKSPACE;
 
-  VerifyParams P;
-  memset(&P, 0, sizeof(P));
-  P.B = A.batch;
-  P.T = A.n_q;
-  P.Hq = A.n_q_heads;
-  P.Hkv = A.n_kv_heads;
-  P.grp = A.n_q_heads / A.n_kv_heads;
-  P.M = P.T * P.grp;
-  P.G = A.n_groups;
-  P.dense = A.dense ? 1 : 0;
-  P.page_size = A.page_size;
-  P.page_shift = -1;
-  for (int s = 0; s < 31; ++s)
-    if ((1 << s) == A.page_size) P.page_shift = s;
-  P.q = static_cast<const __nv_bfloat16*>(A.q);
-  P.kv = static_cast<const __nv_bfloat16*>(A.kv_pages);
-  P.n_pages = A.n_pages;
-  P.s_page = A.stride_page;
-  P.s_kv = A.stride_kv;
-  P.s_slot = A.stride_slot;
-  P.s_head = A.stride_head;
-  P.bt = A.block_table;
-  P.bt_stride = A.block_table_stride;
-  P.kv_len = A.kv_len;
-  P.idx = A.idx;
-  P.idx_stride = A.idx_stride;
-  P.counts = A.counts;
-  const float scale = (A.sm_scale != 0.f) ? A.sm_scale : 1.0f / sqrtf(static_cast<float>(A.head_dim));
-  P.scale_log2 = scale * specattn::kLog2e;
-  P.out = A.out;
-  P.lse = A.lse;
-  P.status = A.status;
+  VerifyParams P = specattn::make_params(A);
   P.counters = static_cast<unsigned int*>(A.workspace);
-  P.lists_stable = (A.flags & SPECATTN_VERIFY_LISTS_STABLE) ? 1 : 0;
-  P.tail = A.tail_len;
-  P.tail_off = A.tail_len - A.n_q;
   P.partials = reinterpret_cast<float*>(static_cast<unsigned char*>(A.workspace) + specattn::kCounterBytes);
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -982,6 +1172,44 @@ extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cu
     }
   }
   if (err != cudaSuccess) return SPECATTN_ERR_CUDA;
+  specattn::g_launch_count.fetch_add(1, std::memory_order_relaxed);
+  return SPECATTN_OK;
+}
+
+extern "C" size_t specattn_verify_plan_bytes(const specattn_verify_args* args) {
+  if (specattn::validate(args) != SPECATTN_OK) return 0;
+  const int n = specattn::device_sm_count();
+  if (n <= 0) return 0;
+  return specattn::plan_ints(args->batch * args->n_kv_heads, n) * sizeof(int);
+}
+
+extern "C" int specattn_verify_plan(const specattn_verify_args* args, void* plan, size_t plan_bytes,
+                                    void* cuda_stream) {
+  const int v = specattn::validate(args);
+  if (v != SPECATTN_OK) return v;
+  const specattn_verify_args& A = *args;
+  if (plan == nullptr || !A.kv_len) return SPECATTN_ERR_NULL;
+  if (!A.dense && !A.counts) return SPECATTN_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(plan) % 16 != 0) return SPECATTN_ERR_ALIGN;
+  const int n_ctas = specattn::device_sm_count();
+  if (n_ctas <= 0) return SPECATTN_ERR_CUDA;
+  if (plan_bytes < specattn::plan_ints(A.batch * A.n_kv_heads, n_ctas) * sizeof(int)) return SPECATTN_ERR_WORKSPACE;
+  if (A.batch == 0) return SPECATTN_OK;
+  VerifyParams P = specattn::make_params(A);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(1, 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = static_cast<cudaStream_t>(cuda_stream);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, specattn::verify_plan_kernel, P, static_cast<int*>(plan), n_ctas) != cudaSuccess) {
+    cudaGetLastError();
+    return SPECATTN_ERR_CUDA;
+  }
   specattn::g_launch_count.fetch_add(1, std::memory_order_relaxed);
   return SPECATTN_OK;
 }

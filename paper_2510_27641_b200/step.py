@@ -11,6 +11,7 @@ from typing import Sequence
 import torch
 
 from . import (SelectArgs, VerifyArgs, SpecAttnError, VERIFY_LISTS_STABLE, lib, make_select_args, make_verify_args,
+               verify_plan, verify_plan_buffer,
                verify_step_host, verify_workspace, _stream_ptr)
 
 __all__ = ["VerifyStep"]
@@ -22,7 +23,8 @@ class VerifyStep:
                  kv_pools: Sequence[torch.Tensor], kv_len: torch.Tensor,
                  block_table: torch.Tensor | None, pages_per_seq: int | None = None,
                  n_groups: int = 1, head_group: Sequence[int] | None = None,
-                 idx_stride: int | None = None, sm_scale: float = 0.0, verify_flags: int = 0, device=None):
+                 idx_stride: int | None = None, sm_scale: float = 0.0, verify_flags: int = 0,
+                 use_plans: bool = True, device=None):
         dev = device or kv_pools[0].device
         self.layer_map = [int(x) for x in layer_map]
         self.n_layers = len(self.layer_map)
@@ -50,6 +52,7 @@ class VerifyStep:
                 idx=self.idx, counts=self.counts, row_status=self.row_status, diag=self.diag)
         self.verify_args: list[VerifyArgs] = []
         self.workspace = None
+        self.plans: dict[int, tuple[torch.Tensor, int]] = {}   # draft layer (-1: dense) -> (plan, a layer using it)
         for j, u in enumerate(self.layer_map):
             a = make_verify_args(self.q[j], kv_pools[j], kv_len, block_table=block_table,
                                  pages_per_seq=pages_per_seq,
@@ -62,6 +65,11 @@ class VerifyStep:
             if self.workspace is None:
                 self.workspace = verify_workspace(a, dev)
             a.workspace, a.workspace_bytes = self.workspace.data_ptr(), self.workspace.numel()
+            # target layers that share a draft layer's lists (or are dense) share a work partition
+            if use_plans:
+                if u not in self.plans:
+                    self.plans[u] = (verify_plan_buffer(a, dev), j)
+                a.plan = self.plans[u][0].data_ptr()
             self.verify_args.append(a)
 
     # ---- inputs -------------------------------------------------------------------------------
@@ -80,6 +88,11 @@ class VerifyStep:
         if rc != 0:
             raise SpecAttnError(rc, "specattn_select_topp")
 
+    def run_plans(self, stream=None):
+        """One small launch per distinct list set: the work partition its verify launches share."""
+        for plan, j in self.plans.values():
+            verify_plan(self.verify_args[j], plan, stream)
+
     def run_verify(self, j: int, stream=None):
         rc = lib().specattn_sparse_verify(C.byref(self.verify_args[j]), _stream_ptr(stream))
         if rc != 0:
@@ -90,6 +103,7 @@ class VerifyStep:
         sp = _stream_ptr(stream)
         L = lib()
         self.run_select(stream)
+        self.run_plans(stream)
         for a in self.verify_args:
             rc = L.specattn_sparse_verify(C.byref(a), sp)
             if rc != 0:
@@ -102,4 +116,4 @@ class VerifyStep:
 
     @property
     def launches_per_step(self) -> int:
-        return (1 if self.select_args is not None else 0) + self.n_layers
+        return (1 if self.select_args is not None else 0) + len(self.plans) + self.n_layers
