@@ -225,3 +225,59 @@ def test_back_to_back_launches_with_many_segments_per_cta():
     torch.cuda.synchronize()
     assert int(st.abs().sum()) == 0
     assert torch.equal(o, out) and torch.equal(l, lse)
+
+
+def test_precomputed_work_partition_gives_the_same_results_and_is_ignored_when_it_does_not_fit():
+    import ctypes as C
+    import paper_2510_27641_b200 as sa
+    if _ENGINE["flags"] != sa.VERIFY_ENGINE_MMA_SYNC:
+        pytest.skip("only the mma.sync engine reads plans")
+    rng = np.random.default_rng(5)
+    lens = rng.integers(1, 5000, size=10).tolist()
+    case = _make_case(70, 10, 5, 32, 8, 16, lens)
+    kv_d = case["kv"].to(dev())
+    q_d, len_d, bt_d = bf16_to_dev(case["q"]), to_dev(case["lens"]), to_dev(case["bt"])
+    idx_d, cnt_d = to_dev(case["idx"]), to_dev(case["cnt"])
+    ref_o, ref_l, _ = _run(case)
+
+    def run(plan, tail_len=0, cnt=cnt_d):
+        o = torch.full_like(ref_o, float("nan"))
+        l = torch.full_like(ref_l, float("nan"))
+        a = sa.make_verify_args(q_d, kv_d, len_d, block_table=bt_d, idx=idx_d, counts=cnt, out=o, lse=l,
+                                flags=_ENGINE["flags"], tail_len=tail_len)
+        a.workspace_t = sa.verify_workspace(a)
+        a.workspace, a.workspace_bytes = a.workspace_t.data_ptr(), a.workspace_t.numel()
+        a.plan = None if plan is None else plan.data_ptr()
+        rc = sa.lib().specattn_sparse_verify(C.byref(a), None)
+        assert rc == 0
+        torch.cuda.synchronize()
+        return o, l, a
+
+    o0, l0, a0 = run(None)
+    plan = sa.verify_plan_buffer(a0)
+    sa.verify_plan(a0, plan)
+    torch.cuda.synchronize()
+    hdr = plan[:8].cpu().tolist()
+    assert hdr[1] == 10 * 8 and hdr[6] == 0 and hdr[7] == 0 and hdr[4] >= 1
+    o1, l1, _ = run(plan)
+    assert torch.equal(o0, o1) and torch.equal(l0, l1) and torch.equal(o0, ref_o)
+    # a plan made for other lists of the same shape is the caller's mistake; one whose header
+    # does not fit the launch (here: another tail_len) is ignored and the kernel partitions itself
+    case_t = _make_case(70, 10, 5, 32, 8, 16, lens, tail=3)
+    ref_t = _oracle(case_t)
+    kv_t = case_t["kv"].to(dev())
+    o = torch.empty_like(ref_o)
+    l = torch.empty_like(ref_l)
+    at = sa.make_verify_args(bf16_to_dev(case_t["q"]), kv_t, to_dev(case_t["lens"]), block_table=to_dev(case_t["bt"]),
+                             idx=to_dev(case_t["idx"]), counts=to_dev(case_t["cnt"]), out=o, lse=l,
+                             flags=_ENGINE["flags"], tail_len=3)
+    ws = sa.verify_workspace(at)
+    at.workspace, at.workspace_bytes = ws.data_ptr(), ws.numel()
+    at.plan = plan.data_ptr()
+    assert sa.lib().specattn_sparse_verify(C.byref(at), None) == 0
+    torch.cuda.synchronize()
+    check_attention(o, l, *ref_t)
+    # argument errors
+    small = torch.zeros(4, dtype=torch.int32, device=dev())
+    assert sa.lib().specattn_verify_plan(C.byref(a0), small.data_ptr(), 16, None) == -5
+    assert sa.lib().specattn_verify_plan(C.byref(a0), None, 1 << 20, None) == -1
