@@ -419,7 +419,8 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--topp-sweep", action="store_true", help="also run the 256-row selection micro-benchmark")
+    ap.add_argument("--topp-sweep", action="store_true", help="(default on) the 256-row selection micro-benchmark of config 2")
+    ap.add_argument("--no-topp-sweep", action="store_true", help="skip the selection micro-benchmark")
     ap.add_argument("--verify-micro", action="store_true", help="only run the sparse_verify micro-benchmark")
     ap.add_argument("--verify-engine", default="auto", choices=["auto", "mma_sync", "tcgen05"],
                     help="force one implementation of sparse_verify (default: the library picks by shape)")
@@ -539,7 +540,7 @@ def main():
                        "global_batch": cfg.batch * world, "ctx": cfg.ctx, "page_size": cfg.page_size,
                        "gamma": cfg.gamma, "p": cfg.p, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
                        "head_dim": cfg.head_dim, "parallelism": f"batch-sharded x{world}, no collective",
-                       "launch": "CUDA graph of 1 select + 32 verify launches",
+                       "launch": f"CUDA graph of 1 select + {len(step.plans)} plan + {step.n_layers} verify launches",
                        "l2": "inputs exceed L2: 252 MB of draft rows and 1.3 GB of gathered K/V per step"},
             "e2e": {"value": round(us_e2e, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(n_step * args.steps),
@@ -560,9 +561,16 @@ def main():
         us_cpu, sample = smp.step_us()
         line["cpu_baseline"] = {"value": round(us_cpu, 1), "unit": UNIT, "cores": smp.cores, "kind": "oracle",
                                 "sample": sample}
-    if rank == 0 and args.topp_sweep:
+    if rank == 0 and not args.no_topp_sweep:
         del g_step, g_verify, g_select
-        line["extra"]["topp_sweep"] = topp_sweep(dev)
+        sweep = topp_sweep(dev)
+        line["extra"]["topp_sweep"] = sweep
+        # the second half of the metric: rows/s of the selection alone, per row length (geometric
+        # mean over the three families and three p of config 2)
+        by_n = {}
+        for k, v in sweep.items():
+            by_n.setdefault(k.split("/")[1], []).append(v["rows_per_s"])
+        line["extra"]["topp_rows_per_s"] = {n: round(float(np.exp(np.mean(np.log(v))))) for n, v in by_n.items()}
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
