@@ -267,6 +267,10 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int warp = tid >> 5;
+  // a one-CTA "cluster" needs no hardware cluster barrier (~0.7 us each, seven per list)
+  auto csync = [&]() {
+    if (cs > 1) cluster.sync(); else __syncthreads();
+  };
 
   const int list = blockIdx.y;  // (used slot, sequence, group)
   const int g = list % P.G;
@@ -512,7 +516,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   __syncthreads();
 
   // ---- 3: threshold search --------------------------------------------------------------------
-  cluster.sync();  // every CTA's level-1 histogram and invalid count are complete
+  csync();  // every CTA's level-1 histogram and invalid count are complete
   int n_bad = 0;
   for (int r = 0; r < cs; ++r) n_bad += *cluster.map_shared_rank(&sh.n_invalid, r);
 
@@ -532,7 +536,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       r_mass[bin] = static_cast<double>((mh << 16) + ml) * pow2_double(max(bin >> 3, 1) - 150);
     }
   }
-  cluster.sync();  // every owner's range is reduced
+  csync();  // every owner's range is reduced
   if (searching) {
     const int per_bins = kL1Bins / cs;
     for (int bin = tid; bin < kL1Bins; bin += kThreads) {
@@ -585,7 +589,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
         hist_add(hr, take, static_cast<int>((key >> shift) & 1023u), mantissa_of(key));
       }
     }
-    cluster.sync();  // every CTA's histogram of this level is complete
+    csync();  // every CTA's histogram of this level is complete
     if (searching) {
       const double scale = pow2_double(e1);
       for (int bin = tid; bin < kL23Bins; bin += kThreads) {
@@ -635,7 +639,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       }
       // the next query's row overwrites the slice and the staging ring, which peers may still
       // be reading (their scans of this CTA's last histogram)
-      cluster.sync();
+      csync();
     }
   }
   }  // for step
@@ -695,7 +699,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     }
     sh.local_kept = s;
   }
-  cluster.sync();  // local_kept of every CTA is visible
+  csync();  // local_kept of every CTA is visible
   long long offset = 0, count = 0;
   for (int r = 0; r < cs; ++r) {
     const int c = *cluster.map_shared_rank(&sh.local_kept, r);
@@ -776,7 +780,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       d[3] = m_ge;
     }
   }
-  cluster.sync();  // nobody leaves while its shared memory may still be read remotely
+  csync();  // nobody leaves while its shared memory may still be read remotely
 }
 
 int pick_cluster(long long L_stride, long long n_lists) {
