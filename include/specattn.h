@@ -104,8 +104,16 @@ extern "C" {
  * multiple of 4 and <= SPECATTN_MAX_KV_LEN; every draft_probs[u] 16-byte aligned;
  * 0 <= kv_len[b] <= L_stride (larger values are clamped); 0 < p (NaN rejected);
  * n_groups >= 1; head_group (HOST, may be NULL = every head feeds every group) values in
- * [0, n_groups).  No workspace is needed: each list is held in the shared memory of one
- * thread-block cluster.
+ * [0, n_groups).
+ *
+ * workspace (optional, device, 16-byte aligned, specattn_select_workspace_bytes() bytes; no
+ * counterpart in the paper): without it each list is aggregated and searched inside the shared
+ * memory of one thread-block cluster (at most 8 CTAs per list, one launch).  With it, and for
+ * the default selection (no variant) over rows of >= 2048 positions, the call runs two
+ * launches: every list's rows are summed by CTAs of 1024 positions each -- in the same order,
+ * so a[] has the same bits -- into the workspace, and the search then reads a[] from there; the
+ * lists are the same, the GPU is filled whatever the number of lists.  The workspace holds no
+ * state between calls; two calls that may overlap on the GPU need separate workspaces.
  * ======================================================================================== */
 typedef struct specattn_select_args {
   uint32_t struct_size;
@@ -133,9 +141,16 @@ typedef struct specattn_select_args {
   int32_t bisect_iters; /* 0 = exact threshold, else 1..64 */
   int32_t chunk;        /* 0 | 1 = per position, else 4, 8, 16, 32 or 64 */
   int32_t reserved;     /* 0 */
+  void* workspace;          /* device, or NULL */
+  uint64_t workspace_bytes; /* size of *workspace */
 } specattn_select_args;
 
 int specattn_select_topp(const specattn_select_args* args, void* cuda_stream);
+
+/* Bytes of workspace that let specattn_select_topp(args) take its two-launch form (0 when the
+ * call would not use one: a variant, single-row lists, rows shorter than 2048 positions, or
+ * invalid arguments).  Reads only the scalar fields and layer_map of args. */
+size_t specattn_select_workspace_bytes(const specattn_select_args* args);
 
 /* ========================================================================================
  * specattn_sparse_verify -- sparse attention of one target layer.

@@ -43,7 +43,7 @@ class SelectArgs(C.Structure):
                 ("p", C.c_float), ("idx", C.c_void_p), ("idx_stride", C.c_int64),
                 ("counts", C.c_void_p), ("row_status", C.c_void_p), ("diag", C.c_void_p),
                 ("per_step", C.c_int32), ("bisect_iters", C.c_int32), ("chunk", C.c_int32),
-                ("reserved", C.c_int32)]
+                ("reserved", C.c_int32), ("workspace", C.c_void_p), ("workspace_bytes", C.c_uint64)]
 
 
 class VerifyArgs(C.Structure):
@@ -81,6 +81,8 @@ def lib() -> C.CDLL:
         L = C.CDLL(str(_LIB_PATH))
         L.specattn_select_topp.argtypes = [C.POINTER(SelectArgs), C.c_void_p]
         L.specattn_select_topp.restype = C.c_int
+        L.specattn_select_workspace_bytes.argtypes = [C.POINTER(SelectArgs)]
+        L.specattn_select_workspace_bytes.restype = C.c_size_t
         L.specattn_sparse_verify.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
         L.specattn_sparse_verify.restype = C.c_int
         L.specattn_verify_workspace_bytes.argtypes = [C.POINTER(VerifyArgs)]
@@ -126,9 +128,11 @@ def make_select_args(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.T
                      head_group: Sequence[int] | None = None, idx: torch.Tensor,
                      counts: torch.Tensor, row_status: torch.Tensor,
                      diag: torch.Tensor | None = None, per_step: bool = False, bisect_iters: int = 0,
-                     chunk: int = 1):
+                     chunk: int = 1, workspace: torch.Tensor | bool | None = True):
     """Fills a SelectArgs.  Returns (args, keepalive) -- keepalive holds the host arrays the
-    struct points at and must outlive the call."""
+    struct points at and must outlive the call.  workspace: a uint8 CUDA tensor, True (allocate
+    what specattn_select_workspace_bytes asks for, if anything) or None / False (none: the
+    one-launch cluster form)."""
     n_d = len(draft_probs)
     ref = next(t for t in draft_probs if t is not None)
     B, H, gamma, Ls = ref.shape
@@ -153,7 +157,15 @@ def make_select_args(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.T
     a.counts, a.row_status = counts.data_ptr(), row_status.data_ptr()
     a.diag = None if diag is None else diag.data_ptr()
     a.per_step, a.bisect_iters, a.chunk = int(bool(per_step)), int(bisect_iters), int(chunk)
-    return a, (ptrs, lm, hg, draft_probs, kv_len, idx, counts, row_status, diag)
+    if workspace is True:
+        need = int(lib().specattn_select_workspace_bytes(C.byref(a)))
+        workspace = torch.empty((need,), dtype=torch.uint8, device=ref.device) if need > 0 else None
+    elif workspace is False:
+        workspace = None
+    if workspace is not None:
+        assert workspace.dtype == torch.uint8 and workspace.is_contiguous()
+        a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    return a, (ptrs, lm, hg, draft_probs, kv_len, idx, counts, row_status, diag, workspace)
 
 
 def select_topp(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.Tensor,
@@ -162,7 +174,7 @@ def select_topp(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.Tensor
                 idx: torch.Tensor | None = None, counts: torch.Tensor | None = None,
                 row_status: torch.Tensor | None = None, diag: torch.Tensor | None = None,
                 want_diag: bool = False, per_step: bool = False, bisect_iters: int = 0, chunk: int = 1,
-                stream=None):
+                workspace: torch.Tensor | bool | None = True, stream=None):
     """specattn_select_topp.  draft_probs: per draft layer a float32 CUDA tensor
     [B, H_d, gamma, L_stride] (None for layers no target layer maps to).  Returns
     (idx [n_d,B,G,idx_stride] int32, counts [n_d,B,G], row_status [n_d,B,G], diag or None)."""
@@ -182,10 +194,12 @@ def select_topp(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.Tensor
     args, keep = make_select_args(draft_probs, kv_len, layer_map, p, n_groups=n_groups,
                                   head_group=head_group, idx=idx, counts=counts,
                                   row_status=row_status, diag=diag, per_step=per_step,
-                                  bisect_iters=bisect_iters, chunk=chunk)
+                                  bisect_iters=bisect_iters, chunk=chunk, workspace=workspace)
     rc = lib().specattn_select_topp(C.byref(args), _stream_ptr(stream))
     if rc != 0:
         raise SpecAttnError(rc, "specattn_select_topp")
+    if keep[-1] is not None and stream is not None and workspace is True:
+        keep[-1].record_stream(stream)   # allocated here, used on the caller's stream
     del keep
     return idx, counts, row_status, diag
 

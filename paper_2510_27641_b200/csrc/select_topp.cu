@@ -81,6 +81,7 @@ struct SelectParams {
   int per_step;    // Alg. 2 as printed: one nucleus per speculated query, unioned
   int bisect_iters;  // > 0: the threshold is the last midpoint of that many bisection steps
   int chunk;         // > 1: selection over per-chunk sums (power of two, 4..64); kept chunks keep all positions
+  const float* agg;  // two-launch form: the aggregated rows, [list][L_stride], written by aggregate_rows_kernel
 };
 
 // A histogram of exact mantissa sums, kept as two 32-bit words: `lo` sums the low 16 mantissa
@@ -296,7 +297,9 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   unsigned int* const lvl_base = reinterpret_cast<unsigned int*>(ring + 4096);  // 2 levels x (lo, hi) x 1024
   const Hist h1 = {sh.h_lo, sh.h_hi};
 
-  const float* A = P.probs[slot] + static_cast<long long>(b) * P.H * P.gamma * P.L_stride + lo;
+  const float* A = (kInPlace && P.agg != nullptr)
+                       ? P.agg + static_cast<long long>(list) * P.L_stride + lo
+                       : P.probs[slot] + static_cast<long long>(b) * P.H * P.gamma * P.L_stride + lo;
   constexpr bool in_place = kInPlace;
   // bit pattern of aggregated position i of the slice (-0.0 reads as +0.0)
   auto key_at = [&](int i) -> unsigned int {
@@ -356,6 +359,8 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   }
   for (int i = tid; i < kL1Bins; i += kThreads) sh.h_hi[i] = sh.h_lo[i] = 0u;
   __syncthreads();
+  // two-launch form: this kernel was allowed to start while the aggregation still ran
+  if (kInPlace && P.agg != nullptr) pdl_wait();
   const int R = sh.n_rows;
   float vmax = 0.f;  // largest aggregated value of this thread's positions (literal bisection)
 
@@ -783,6 +788,102 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   csync();  // nobody leaves while its shared memory may still be read remotely
 }
 
+// First launch of the two-launch form: a[i] = +0 + the contributing rows in order, for 1024
+// positions per CTA, so that the number of CTAs streaming the rows from HBM does not depend on
+// the number of lists.  The adds are the ones of the cluster kernel (binary32, same order), so
+// the bits of a[] are the same.  A negative input, which a sum could hide, poisons its
+// position with NaN: the search then reports the list as invalid like the cluster kernel does.
+constexpr int kAggPositions = kThreads * 4;
+constexpr int kAggUnroll = 8;
+__global__ void __launch_bounds__(kThreads) aggregate_rows_kernel(const __grid_constant__ SelectParams P,
+                                                                  float* __restrict__ out) {
+  __shared__ long long row_off[SPECATTN_MAX_ROWS_PER_LIST];
+  __shared__ int n_rows;
+  pdl_launch_dependents();  // the search kernel may take its place on the SMs; it waits for this grid
+  const int tid = threadIdx.x;
+  const int list = blockIdx.y;
+  const int g = list % P.G;
+  const int b = (list / P.G) % P.B;
+  const int slot = list / (P.G * P.B);
+  long long Lll = P.kv_len[b];
+  if (Lll < 0) Lll = 0;
+  if (Lll > P.L_stride) Lll = P.L_stride;
+  const int L = static_cast<int>(Lll);
+  const int pos = blockIdx.x * kAggPositions + 4 * tid;
+  if (blockIdx.x * kAggPositions >= L) return;
+  if (tid == 0) {
+    int n = 0;
+    for (int h = 0; h < P.H; ++h) {
+      if (P.has_groups && P.head_group[h] != g) continue;
+      for (int s = 0; s < P.gamma; ++s) row_off[n++] = static_cast<long long>(h * P.gamma + s) * P.L_stride;
+    }
+    n_rows = n;
+  }
+  __syncthreads();
+  if (pos >= L) return;
+  const int R = n_rows;
+  const int cut = L - pos;  // positions of this float4 that are inputs
+  const float* src = P.probs[slot] + static_cast<long long>(b) * P.H * P.gamma * P.L_stride + pos;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), mn = acc;
+  for (int r0 = 0; r0 < R; r0 += kAggUnroll) {
+    float4 x[kAggUnroll];
+#pragma unroll
+    for (int k = 0; k < kAggUnroll; ++k)
+      if (r0 + k < R) x[k] = __ldcs(reinterpret_cast<const float4*>(src + row_off[r0 + k]));
+#pragma unroll
+    for (int k = 0; k < kAggUnroll; ++k) {
+      if (r0 + k < R) {
+        float4 v = x[k];
+        if (cut < 4) {  // values beyond kv_len are not inputs
+          v.w = 0.f;
+          if (cut < 3) v.z = 0.f;
+          if (cut < 2) v.y = 0.f;
+        }
+        mn.x = fminf(mn.x, v.x);
+        mn.y = fminf(mn.y, v.y);
+        mn.z = fminf(mn.z, v.z);
+        mn.w = fminf(mn.w, v.w);
+        acc.x = acc.x + v.x;
+        acc.y = acc.y + v.y;
+        acc.z = acc.z + v.z;
+        acc.w = acc.w + v.w;
+      }
+    }
+  }
+  const float nan = __uint_as_float(0x7fc00000u);
+  if (mn.x < 0.f) acc.x = nan;
+  if (mn.y < 0.f) acc.y = nan;
+  if (mn.z < 0.f) acc.z = nan;
+  if (mn.w < 0.f) acc.w = nan;
+  *reinterpret_cast<float4*>(out + static_cast<long long>(list) * P.L_stride + pos) = acc;
+}
+
+// Number of index lists of a call (0 on invalid arguments) -- shared by the entry point and
+// the workspace query.
+long long count_lists(const specattn_select_args& A) {
+  if (A.n_draft_layers < 1 || A.n_draft_layers > SPECATTN_MAX_DRAFT_LAYERS || A.n_target_layers < 0 ||
+      A.batch < 0 || A.n_groups < 1 || A.layer_map == nullptr)
+    return 0;
+  bool used[SPECATTN_MAX_DRAFT_LAYERS] = {false};
+  int n_used = 0;
+  for (int j = 0; j < A.n_target_layers; ++j) {
+    const int u = A.layer_map[j];
+    if (u < -1 || u >= A.n_draft_layers) return 0;
+    if (u >= 0 && !used[u]) {
+      used[u] = true;
+      ++n_used;
+    }
+  }
+  return static_cast<long long>(n_used) * A.batch * A.n_groups;
+}
+
+// The two-launch form applies to the default selection over multi-row lists of >= 2048 positions.
+bool two_launch_shape(const specattn_select_args& A) {
+  const bool variant = (A.per_step && A.gamma > 1) || A.bisect_iters > 0 || A.chunk > 1;
+  return !variant && static_cast<long long>(A.n_draft_heads) * A.gamma > 1 && A.L_stride >= 2048 &&
+         A.L_stride % 4 == 0;
+}
+
 int pick_cluster(long long L_stride, long long n_lists) {
   int cs = 1;
   while (cs < 8 && (L_stride + cs - 1) / cs > 8192) cs *= 2;
@@ -794,6 +895,12 @@ int pick_cluster(long long L_stride, long long n_lists) {
 }  // namespace specattn
 
 using specattn::SelectParams;
+
+extern "C" size_t specattn_select_workspace_bytes(const specattn_select_args* args) {
+  if (args == nullptr || args->struct_size != sizeof(specattn_select_args)) return 0;
+  if (!specattn::two_launch_shape(*args)) return 0;
+  return static_cast<size_t>(specattn::count_lists(*args)) * static_cast<size_t>(args->L_stride) * sizeof(float);
+}
 
 extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda_stream) {
   if (args == nullptr) return SPECATTN_ERR_NULL;
@@ -861,6 +968,15 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   // single-row lists are read in place once the rows are long enough for the extra CTAs per
   // SM to pay for re-reading them from L2 (measured cross-over between 8k and 64k positions)
   P.single_row = (static_cast<long long>(A.n_draft_heads) * A.gamma == 1 && A.L_stride >= 2048) ? 1 : 0;
+  // two-launch form: the rows are summed into the workspace first and the search reads that sum
+  // in place like a single-row list
+  const bool two_launch = A.workspace != nullptr && specattn::two_launch_shape(A) &&
+                          A.workspace_bytes >= static_cast<uint64_t>(n_lists) * A.L_stride * sizeof(float);
+  if (two_launch) {
+    if (reinterpret_cast<uintptr_t>(A.workspace) % 16 != 0) return SPECATTN_ERR_ALIGN;
+    P.single_row = 1;
+    P.agg = static_cast<const float*>(A.workspace);
+  }
   P.per_step = (A.per_step && A.gamma > 1) ? 1 : 0;  // with one query the union is the single nucleus
   P.bisect_iters = A.bisect_iters;
   P.chunk = (A.chunk > 1) ? A.chunk : 1;
@@ -926,13 +1042,24 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   cfg.blockDim = dim3(specattn::kThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = static_cast<cudaStream_t>(cuda_stream);
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = static_cast<unsigned>(cs);
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (two_launch) {
+    const dim3 grid(static_cast<unsigned>((A.L_stride + specattn::kAggPositions - 1) / specattn::kAggPositions),
+                    static_cast<unsigned>(n_lists), 1);
+    specattn::aggregate_rows_kernel<<<grid, specattn::kThreads, 0, cfg.stream>>>(P, static_cast<float*>(A.workspace));
+    if (cudaGetLastError() != cudaSuccess) return SPECATTN_ERR_CUDA;
+    specattn::g_launch_count.fetch_add(1, std::memory_order_relaxed);
+    // the search may be scheduled while the aggregation drains; it waits before reading a[]
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
+  }
   if (variant)
     err = P.single_row ? cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<true, true>, P)
                        : cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<false, true>, P);

@@ -24,7 +24,7 @@ class VerifyStep:
                  block_table: torch.Tensor | None, pages_per_seq: int | None = None,
                  n_groups: int = 1, head_group: Sequence[int] | None = None,
                  idx_stride: int | None = None, sm_scale: float = 0.0, verify_flags: int = 0,
-                 use_plans: bool = True, device=None):
+                 use_plans: bool = True, select_workspace: bool = True, device=None):
         dev = device or kv_pools[0].device
         self.layer_map = [int(x) for x in layer_map]
         self.n_layers = len(self.layer_map)
@@ -49,7 +49,8 @@ class VerifyStep:
         if used:   # a step whose layers are all dense has nothing to select
             self.select_args, self._keep = make_select_args(
                 self.draft_probs, kv_len, self.layer_map, p, n_groups=n_groups, head_group=head_group,
-                idx=self.idx, counts=self.counts, row_status=self.row_status, diag=self.diag)
+                idx=self.idx, counts=self.counts, row_status=self.row_status, diag=self.diag,
+                workspace=select_workspace)
         self.verify_args: list[VerifyArgs] = []
         self.workspace = None
         self.plans: dict[int, tuple[torch.Tensor, int]] = {}   # draft layer (-1: dense) -> (plan, a layer using it)
@@ -116,4 +117,7 @@ class VerifyStep:
 
     @property
     def launches_per_step(self) -> int:
-        return (1 if self.select_args is not None else 0) + len(self.plans) + self.n_layers
+        n_select = 0
+        if self.select_args is not None:
+            n_select = 2 if self.select_args.workspace else 1   # aggregation + search, or the cluster form
+        return n_select + len(self.plans) + self.n_layers

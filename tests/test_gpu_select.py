@@ -16,6 +16,16 @@ from gpu_util import compare_lists, dev, to_dev
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=["two_launch", "cluster"], autouse=True)
+def form(request, monkeypatch):
+    """Every case runs once per form of the call: with a workspace (aggregation launch + search
+    launch, where the shape allows it) and without (one cluster per list)."""
+    import functools
+    import paper_2510_27641_b200 as sa
+    monkeypatch.setattr(sa, "select_topp", functools.partial(sa.select_topp, workspace=request.param == "two_launch"))
+    return request.param
+
+
 def _run_rows(rows: np.ndarray, kv_len, p, idx_stride=None):
     """R = 1: each row is its own list.  rows [n_rows, L_stride] float32."""
     import paper_2510_27641_b200 as sa
@@ -299,3 +309,38 @@ def test_chunk_selection_overflow_single_row_and_arguments():
         a, keep = sa.make_select_args([to_dev(probs)], to_dev(kv), [0], 0.9, idx=gi.new_zeros((1, 1, 1, 8)),
                                       counts=gc.new_zeros((1, 1, 1)), row_status=gs.new_zeros((1, 1, 1)), chunk=bad_chunk)
         assert sa.lib().specattn_select_topp(C.byref(a), None) == -3
+
+
+def test_both_forms_give_the_same_bits_and_flag_hidden_negative_inputs(form):
+    """Multi-row lists: the two-launch form (workspace) and the cluster form must agree bit for
+    bit (lists, counts, status, diag), also for ragged lengths, head groups and invalid inputs --
+    a negative input that the sum hides, NaN, Inf, and garbage beyond kv_len."""
+    import paper_2510_27641_b200 as sa
+    B, H, gamma, Ls = 5, 6, 3, 6144
+    kv_len = np.array([6144, 2049, 5000, 6144, 3000], np.int32)
+    probs = wl.draft_probs(11, 0, kv_len, H, gamma, Ls, sink=6.0, slope=0.004)
+    probs[1, 2, 1, 700] = -1e-30        # hidden by the other 17 rows' mass
+    probs[2, 0, 0, 4999] = np.nan
+    probs[3, 5, 2, 6143] = np.inf
+    probs[4, :, :, 3000:] = -5.0        # beyond kv_len: not inputs
+    hg = (np.arange(H) * 2 // H).astype(np.int32)
+    d = to_dev(probs)
+    res = {}
+    for ws in (True, False):
+        gi, gc, gs, gd = sa.select_topp.func([d], to_dev(kv_len), [0], 0.9, n_groups=2, head_group=hg.tolist(),
+                                             want_diag=True, workspace=ws)
+        torch.cuda.synchronize()
+        res[ws] = (gi.cpu().numpy(), gc.cpu().numpy(), gs.cpu().numpy(), gd.cpu().numpy())
+    (i1, c1, s1, d1), (i0, c0, s0, d0) = res[True], res[False]
+    assert np.array_equal(c1, c0) and np.array_equal(s1, s0)
+    ok = s0 == 0
+    assert np.array_equal(d1[ok], d0[ok])
+    for b in range(B):
+        for g in range(2):
+            assert np.array_equal(i1[0, b, g, :c0[0, b, g]], i0[0, b, g, :c0[0, b, g]])
+    bad = sa.ROW_INVALID_PROB
+    assert s0[0, :, 0].tolist() == [0, bad if hg[2] == 0 else 0, bad, 0, 0]
+    assert s0[0, :, 1].tolist() == [0, bad if hg[2] == 1 else 0, 0, bad, 0]
+    oi, oc, os_, od = oracle.select_topp([probs], np.zeros(1, np.int32), kv_len, 0.9, n_groups=2, head_group=hg)
+    assert np.array_equal(os_, s0)
+    assert np.array_equal(oc[os_ == 0], c0[os_ == 0])
