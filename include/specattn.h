@@ -109,7 +109,8 @@ extern "C" {
  * workspace (optional, device, 16-byte aligned, specattn_select_workspace_bytes() bytes; no
  * counterpart in the paper): without it each list is aggregated and searched inside the shared
  * memory of one thread-block cluster (at most 8 CTAs per list, one launch).  With it, and for
- * the default selection (no variant) over rows of >= 2048 positions, the call runs two
+ * the default selection (no variant) over rows of >= 2048 positions when the lists are so few
+ * that one cluster each would leave SMs idle (lists x CTAs per cluster < 148), the call runs two
  * launches: every list's rows are summed by CTAs of 1024 positions each -- in the same order,
  * so a[] has the same bits -- into the workspace, and the search then reads a[] from there; the
  * lists are the same, the GPU is filled whatever the number of lists.  The workspace holds no
@@ -148,8 +149,8 @@ typedef struct specattn_select_args {
 int specattn_select_topp(const specattn_select_args* args, void* cuda_stream);
 
 /* Bytes of workspace that let specattn_select_topp(args) take its two-launch form (0 when the
- * call would not use one: a variant, single-row lists, rows shorter than 2048 positions, or
- * invalid arguments).  Reads only the scalar fields and layer_map of args. */
+ * call would not use one: a variant, single-row lists, rows shorter than 2048 positions, enough
+ * lists to fill the GPU with one cluster each, or invalid arguments).  Reads only the scalar fields and layer_map of args. */
 size_t specattn_select_workspace_bytes(const specattn_select_args* args);
 
 /* ========================================================================================

@@ -27,12 +27,18 @@
 //      Every CTA scans the reduced bins with the same warp-shuffle suffix scan in binary64,
 //      so all arrive at the same bin without a broadcast.  (Remote atomics into one CTA's
 //      histogram were measured first and cost ~11 us per level on tie-free rows.)
+//      When the level-1 threshold bin holds at most 512 values (its exact mantissa sum bounds
+//      their number) levels 2 and 3 are replaced by a short cut: every CTA collects its keys of
+//      that bin, all CTAs fetch all of them and pick the threshold key directly.
 //   4. after three levels the threshold is known bit-exactly; each CTA compacts its kept
 //      positions in ascending order behind the counts of the lower-ranked CTAs.
 // When a list has a single contributing row (one draft head, gamma = 1: the selection
 // micro-benchmark) of 32k positions or more there is nothing to aggregate and the row is not
 // copied to shared memory at all but re-read from global memory (L2) by the later passes,
-// which shrinks a CTA to ~57 KB of shared memory so that four of them share an SM.
+// which shrinks a CTA to ~51 KB of shared memory so that four of them share an SM.
+// With a workspace and few lists the call becomes two launches: aggregate_rows_kernel sums the
+// rows with 1024 positions per CTA (the whole GPU streams, however few the lists) and the
+// search runs in place over that sum.
 #include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <float.h>
@@ -61,6 +67,7 @@ constexpr int kL23Bins = 1024;           // 10 mantissa bits per later level
 constexpr int kGroup = 32;               // bins per scan group (one warp-wide scan)
 constexpr int kSliceCap = 24576;         // positions per CTA
 constexpr unsigned int kFull = 0xffffffffu;
+constexpr int kCandCap = 512;           // keys of the threshold bin that the short cut below can hold
 
 struct SelectParams {
   const float* probs[SPECATTN_MAX_DRAFT_LAYERS];  // per used slot
@@ -103,6 +110,10 @@ struct Shared {
   float warp_max[kWarps];   // largest aggregated value seen by each warp (literal bisection only)
   float cta_max;            // read by the other CTAs of the cluster
   int local_kept;           // read by the other CTAs of the cluster
+  int n_cand;               // keys this CTA found in the level-1 threshold bin (read by the cluster)
+  unsigned int cand[kCandCap];
+  unsigned int red_key[2 * kWarps];
+  unsigned long long red_sum[2 * kWarps];
   // result of a scan (written by warp 0)
   int found_bin;
   double mass_above;        // mass strictly above the found bin (incl. carry)
@@ -146,6 +157,20 @@ __device__ __forceinline__ void hist_add(const Hist& h, bool take, int bin, unsi
   } else if (take) {
     hist_bump(h, bin, mant & 0xffffu, mant >> 16);
   }
+}
+
+// Appends the keys of the taking lanes to the CTA's candidate list (all 32 lanes call this
+// together); slots beyond the capacity are counted but not stored.
+__device__ __forceinline__ void cand_add(Shared& sh, bool take, unsigned int key) {
+  const unsigned takers = __ballot_sync(kFull, take);
+  if (takers == 0) return;
+  const int lane = threadIdx.x & 31;
+  const int leader = __ffs(takers) - 1;
+  int base = 0;
+  if (lane == leader) base = atomicAdd(&sh.n_cand, __popc(takers));
+  base = __shfl_sync(kFull, base, leader);
+  const int slot = base + __popc(takers & ((1u << lane) - 1u));
+  if (take && slot < kCandCap) sh.cand[slot] = key;
 }
 
 __device__ __forceinline__ double shfl_down_f64(double v, int d) { return __shfl_down_sync(kFull, v, d); }
@@ -356,6 +381,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       }
     }
     sh.n_rows = n;
+    sh.n_cand = 0;
   }
   for (int i = tid; i < kL1Bins; i += kThreads) sh.h_hi[i] = sh.h_lo[i] = 0u;
   __syncthreads();
@@ -560,6 +586,112 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   unsigned int prefix = searching ? static_cast<unsigned int>(sh.found_bin) : 0u;
   const int e1 = max(static_cast<int>(prefix >> 3), 1) - 150;
   double carry_m = searching ? sh.mass_above : 0.0;
+  bool short_cut = false;  // the threshold was found among the gathered keys of the level-1 bin
+  // Short cut: the threshold bin of level 1 usually holds few values (tens to hundreds for
+  // attention rows).  Its mantissa sum S bounds their number (a normal mantissa is >= 2^23); when
+  // at most kCandCap fit, every CTA collects its keys of that bin, fetches everybody's, and
+  // finds the threshold among them directly -- the sums of their mantissas are exact integers,
+  // so every CTA decides alike -- instead of two more rounds of histogram, cluster reduction
+  // and scan (~6 us each, all latency).
+  if (searching && (prefix >> 3) >= 1u) {
+    const unsigned long long S = static_cast<unsigned long long>(r_mass[prefix] * pow2_double(-e1));
+    short_cut = (S >> 23) <= static_cast<unsigned long long>(kCandCap);
+  }
+  if (short_cut) {
+    if (in_place) {
+      for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
+        unsigned int key[kIpUnroll][4];
+        bool act[kIpUnroll];
+#pragma unroll
+        for (int uu = 0; uu < kIpUnroll; ++uu) act[uu] = load_keys4(base + uu * kThreads + tid, key[uu]);
+#pragma unroll
+        for (int uu = 0; uu < kIpUnroll; ++uu) {
+          const int i4 = base + uu * kThreads + tid;
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            cand_add(sh, act[uu] && (4 * i4 + e < n_loc) && (key[uu][e] >> 20) == prefix, key[uu][e]);
+        }
+      }
+    } else {
+      for (int base = 0; base < n_srch; base += kThreads) {
+        const int i = base + tid;
+        const unsigned int key = (i < n_srch) ? key_at(i) : 0u;
+        cand_add(sh, i < n_srch && (key >> 20) == prefix, key);
+      }
+    }
+    csync();  // every CTA's candidate list is complete
+    int cnt_r[8];
+    int M = 0;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      cnt_r[r] = (r < cs) ? min(*cluster.map_shared_rank(&sh.n_cand, r), kCandCap) : 0;
+      M += cnt_r[r];
+    }
+    M = min(M, kCandCap);  // (the bound on S guarantees it)
+    unsigned int* const all = reinterpret_cast<unsigned int*>(r_mass);
+    int off = 0;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      if (r < cs) {
+        const unsigned int* src = cluster.map_shared_rank(sh.cand, r);
+        for (int i = tid; i < cnt_r[r] && off + i < kCandCap; i += kThreads) all[off + i] = src[i];
+        off += cnt_r[r];
+      }
+    }
+    __syncthreads();
+    const double scale = pow2_double(e1);
+    // highest key whose suffix (itself, its ties and everything above) reaches the target
+    unsigned int best = 0u, lowest = 0xffffffffu;
+    for (int i = tid; i < M; i += kThreads) {
+      const unsigned int ki = all[i];
+      unsigned long long s_ge = 0ull;
+      for (int j = 0; j < M; ++j) {
+        const unsigned int kj = all[j];
+        s_ge += (kj >= ki) ? mantissa_of(kj) : 0u;
+      }
+      if (carry_m + static_cast<double>(s_ge) * scale >= target) best = max(best, ki);
+      lowest = min(lowest, ki);
+    }
+    best = __reduce_max_sync(kFull, best);
+    lowest = __reduce_min_sync(kFull, lowest);
+    if (lane == 0) {
+      sh.red_key[warp] = best;
+      sh.red_key[kWarps + warp] = lowest;
+    }
+    __syncthreads();
+    best = 0u;
+    lowest = 0xffffffffu;
+    for (int w = 0; w < kWarps; ++w) {
+      best = max(best, sh.red_key[w]);
+      lowest = min(lowest, sh.red_key[kWarps + w]);
+    }
+    // (no key reaches it only through rounding between two summation orders: keep the bin)
+    const unsigned int theta = (best != 0u) ? best : lowest;
+    unsigned long long s_ge = 0ull, s_gt = 0ull;
+    for (int j = tid; j < M; j += kThreads) {
+      const unsigned int kj = all[j];
+      s_ge += (kj >= theta) ? mantissa_of(kj) : 0u;
+      s_gt += (kj > theta) ? mantissa_of(kj) : 0u;
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+      s_ge += __shfl_xor_sync(kFull, s_ge, o);
+      s_gt += __shfl_xor_sync(kFull, s_gt, o);
+    }
+    if (lane == 0) {
+      sh.red_sum[warp] = s_ge;
+      sh.red_sum[kWarps + warp] = s_gt;
+    }
+    __syncthreads();
+    s_ge = s_gt = 0ull;
+    for (int w = 0; w < kWarps; ++w) {
+      s_ge += sh.red_sum[w];
+      s_gt += sh.red_sum[kWarps + w];
+    }
+    theta_key = theta;
+    m_gt = carry_m + static_cast<double>(s_gt) * scale;
+    m_ge = carry_m + static_cast<double>(s_ge) * scale;
+  } else
   for (int level = 0; level < 2; ++level) {
     const int shift = (level == 0) ? 10 : 0;
     unsigned int* lb = lvl_base + level * 2 * kL23Bins;
@@ -612,7 +744,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       carry_m = sh.mass_above;
     }
   }
-  if (searching) {
+  if (searching && !short_cut) {
     theta_key = prefix;
     m_gt = sh.mass_above;
     m_ge = sh.mass_ge;
@@ -877,18 +1009,25 @@ long long count_lists(const specattn_select_args& A) {
   return static_cast<long long>(n_used) * A.batch * A.n_groups;
 }
 
-// The two-launch form applies to the default selection over multi-row lists of >= 2048 positions.
-bool two_launch_shape(const specattn_select_args& A) {
-  const bool variant = (A.per_step && A.gamma > 1) || A.bisect_iters > 0 || A.chunk > 1;
-  return !variant && static_cast<long long>(A.n_draft_heads) * A.gamma > 1 && A.L_stride >= 2048 &&
-         A.L_stride % 4 == 0;
-}
-
 int pick_cluster(long long L_stride, long long n_lists) {
   int cs = 1;
   while (cs < 8 && (L_stride + cs - 1) / cs > 8192) cs *= 2;
   while (cs < 8 && n_lists * cs < 296 && L_stride / cs > 2048) cs *= 2;
   return cs;
+}
+
+// The two-launch form applies to the default selection over multi-row lists of >= 2048
+// positions, and pays when one cluster per list would leave SMs without a CTA: a CTA streams
+// ~35 GB/s, so the cluster kernel is bound by (bytes per list) / (8 x 35 GB/s) however few the
+// lists, while the search launch adds ~25 us of its own.  Measured (us, cluster / two-launch):
+// 4 lists x 64 rows x 131072: 121 / 94; 16 such lists: 237 / 152; 32 lists x 60 rows x 32768
+// (256 CTAs): 71 / 94.
+bool two_launch_shape(const specattn_select_args& A) {
+  const bool variant = (A.per_step && A.gamma > 1) || A.bisect_iters > 0 || A.chunk > 1;
+  if (variant || static_cast<long long>(A.n_draft_heads) * A.gamma <= 1 || A.L_stride < 2048 || A.L_stride % 4 != 0)
+    return false;
+  const long long n_lists = count_lists(A);
+  return n_lists > 0 && n_lists * pick_cluster(A.L_stride, n_lists) < 148;
 }
 
 }  // namespace

@@ -327,9 +327,11 @@ def test_both_forms_give_the_same_bits_and_flag_hidden_negative_inputs(form):
     d = to_dev(probs)
     res = {}
     for ws in (True, False):
+        n0 = sa.lib().specattn_kernel_launch_count()
         gi, gc, gs, gd = sa.select_topp.func([d], to_dev(kv_len), [0], 0.9, n_groups=2, head_group=hg.tolist(),
                                              want_diag=True, workspace=ws)
         torch.cuda.synchronize()
+        assert sa.lib().specattn_kernel_launch_count() - n0 == (2 if ws else 1)   # the form asked for ran
         res[ws] = (gi.cpu().numpy(), gc.cpu().numpy(), gs.cpu().numpy(), gd.cpu().numpy())
     (i1, c1, s1, d1), (i0, c0, s0, d0) = res[True], res[False]
     assert np.array_equal(c1, c0) and np.array_equal(s1, s0)
@@ -344,3 +346,25 @@ def test_both_forms_give_the_same_bits_and_flag_hidden_negative_inputs(form):
     oi, oc, os_, od = oracle.select_topp([probs], np.zeros(1, np.int32), kv_len, 0.9, n_groups=2, head_group=hg)
     assert np.array_equal(os_, s0)
     assert np.array_equal(oc[os_ == 0], c0[os_ == 0])
+
+
+@pytest.mark.parametrize("n", [1024, 4096, 40000])
+@pytest.mark.parametrize("n_bin", [1, 37, 512, 513])
+def test_threshold_bin_population_around_the_short_cut_capacity(n, n_bin):
+    """The search takes a short cut when the level-1 threshold bin can hold at most 512 values
+    (it gathers them instead of refining with two more histogram levels).  Rows whose threshold
+    bin holds exactly n_bin distinct values just above 2^-10 (so the bin's mantissa sum >> 23
+    equals n_bin), for populations on both sides of that capacity, in a shared-memory slice
+    (n = 1024), a row read in place by one CTA and one read by a cluster."""
+    rng = np.random.default_rng(n + n_bin)
+    rows = np.full((3, n), 1e-9, np.float32)
+    for r in range(3):
+        pos = rng.permutation(n)
+        rows[r, pos[:n_bin]] = (np.float32(2.0 ** -10) * (1 + np.arange(n_bin, dtype=np.float64) * 2.0 ** -23)).astype(np.float32)
+        rows[r, pos[n_bin:n_bin + 4]] = 0.1
+    bin_mass = n_bin * 2.0 ** -10
+    total = 0.4 + bin_mass + (n - n_bin - 4) * 1e-9
+    for frac in (0.01, 0.5, 0.999):       # threshold at the top, in the middle and at the bottom of the bin
+        p = (0.4 + frac * bin_mass) / total
+        st, gd, od = _run_rows(rows, n, float(p))
+        assert st["n"] == 3
