@@ -931,7 +931,6 @@ __global__ void __launch_bounds__(kThreads) aggregate_rows_kernel(const __grid_c
                                                                   float* __restrict__ out) {
   __shared__ long long row_off[SPECATTN_MAX_ROWS_PER_LIST];
   __shared__ int n_rows;
-  pdl_launch_dependents();  // the search kernel may take its place on the SMs; it waits for this grid
   const int tid = threadIdx.x;
   const int list = blockIdx.y;
   const int g = list % P.G;
@@ -988,6 +987,9 @@ __global__ void __launch_bounds__(kThreads) aggregate_rows_kernel(const __grid_c
   if (mn.z < 0.f) acc.z = nan;
   if (mn.w < 0.f) acc.w = nan;
   *reinterpret_cast<float4*>(out + static_cast<long long>(list) * P.L_stride + pos) = acc;
+  // the search kernel's CTAs may move in as this grid drains (earlier, they would take thread
+  // slots from CTAs that still stream); it waits for the whole grid before reading a[]
+  pdl_launch_dependents();
 }
 
 // Number of index lists of a call (0 on invalid arguments) -- shared by the entry point and
@@ -1147,7 +1149,6 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
                       (P.single_row ? static_cast<size_t>(32 * 1024) : static_cast<size_t>(specattn::kRingFloats) * sizeof(float)) +
                       (P.per_step ? static_cast<size_t>(specattn::kSliceCap / 8) : 0);  // the union's bit mask
   if (smem > 224 * 1024) return SPECATTN_ERR_UNSUPPORTED;
-
   // Opt in to large dynamic shared memory once per device, so that later calls issue nothing
   // but the launch.
   cudaError_t err = cudaSuccess;
@@ -1198,6 +1199,45 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.numAttrs = 2;
+  }
+  // Few clusters: ask for more shared memory than needed, so that an SM takes fewer CTAs and the
+  // clusters spread over the GPU instead of filling every slot of a few SMs (co-resident CTAs
+  // slow one another's passes: 32 CTAs took 79 us packed, 62 us spread) -- but only as far as
+  // all clusters still run at once (clusters are placed GPC by GPC; 16 clusters of 8 do not fit
+  // at one CTA per SM, and a second wave costs far more).  The limits are asked of the runtime
+  // once per cluster size and cached.
+  {
+    const void* fn = variant ? (P.single_row ? (const void*)specattn::select_topp_kernel<true, true>
+                                             : (const void*)specattn::select_topp_kernel<false, true>)
+                             : (P.single_row ? (const void*)specattn::select_topp_kernel<true, false>
+                                             : (const void*)specattn::select_topp_kernel<false, false>);
+    static const size_t pads[3] = {120 * 1024, 100 * 1024, 70 * 1024};
+    static std::atomic<int> fit[64][4][4][3];  // [device][kernel][log2 cs][pad]: clusters + 1, 0 = unknown
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const int kidx = (variant ? 2 : 0) + (P.single_row ? 1 : 0);
+    int lcs = 0;
+    while ((1 << lcs) < cs) ++lcs;
+    for (int k = 0; k < 3 && dev >= 0 && dev < 64; ++k) {
+      if (pads[k] <= smem) break;
+      int known = fit[dev][kidx][lcs][k].load(std::memory_order_relaxed);
+      if (known == 0) {
+        cudaLaunchConfig_t q = cfg;
+        q.dynamicSmemBytes = pads[k];
+        q.gridDim = dim3(static_cast<unsigned>(cs), 1024, 1);
+        int n_fit = 0;
+        if (cudaOccupancyMaxActiveClusters(&n_fit, fn, &q) != cudaSuccess) {
+          cudaGetLastError();
+          n_fit = 0;
+        }
+        known = n_fit + 1;
+        fit[dev][kidx][lcs][k].store(known, std::memory_order_relaxed);
+      }
+      if (known - 1 >= n_lists) {
+        cfg.dynamicSmemBytes = pads[k];
+        break;
+      }
+    }
   }
   if (variant)
     err = P.single_row ? cudaLaunchKernelEx(&cfg, specattn::select_topp_kernel<true, true>, P)
