@@ -681,11 +681,6 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         } else {
           bad = resolve(t0, off);
         }
-        // Resolve this warp's next tile of the segment now, so that its two dependent loads
-        // are in flight while the warp waits for the slot: the slot's turnaround then holds
-        // only the copy itself.
-        t0_next = t0 + kProdWarps * kStageTok;
-        if (t0_next < tok_hi) bad_next = resolve(t0_next, off_next); else t0_next = -1;
         if (!mbar_wait(&sh.empty[s], ph ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
         const int ntok = min(kStageTok, tok_hi - t0);
         // The tail of a segment is padded to a whole 32-key block with copies of its last
@@ -714,6 +709,11 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           q_pending = false;
           if (!load_q()) { sh.abort_flag = 1; dead = true; break; }
         }
+        // Resolve this warp's next tile of the segment right after the copies went out (not
+        // before: while the ring still has free slots the two dependent loads would delay
+        // them by ~1.3 us), so that a slot's turnaround holds only the copy itself.
+        t0_next = t0 + kProdWarps * kStageTok;
+        if (t0_next < tok_hi) bad_next = resolve(t0_next, off_next); else t0_next = -1;
         if (bad && P.status) atomicOr(P.status + b, SPECATTN_ROW_BAD_INDEX);
         last_it = it;
       }
