@@ -134,7 +134,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------
-def build_step(cfg, dev, verify_flags=0):
+def build_step(cfg, dev, verify_flags=0, select_workspace=True):
     import torch
     import workloads as wl
     from paper_2510_27641_b200.step import VerifyStep
@@ -147,7 +147,7 @@ def build_step(cfg, dev, verify_flags=0):
                       n_q_heads=cfg.n_q_heads, p=cfg.p, kv_pools=pools,
                       kv_len=torch.from_numpy(si.kv_len).to(dev),
                       block_table=None if si.block_table is None else torch.from_numpy(si.block_table).to(dev),
-                      pages_per_seq=si.pages_per_seq, verify_flags=verify_flags)
+                      pages_per_seq=si.pages_per_seq, verify_flags=verify_flags, select_workspace=select_workspace)
     dp_host = [None if x is None else torch.from_numpy(x).pin_memory() for x in si.draft_probs]
     q_host = [bf16.bits_to_torch(q).pin_memory() for q in si.q]
     step.load_inputs(dp_host, q_host)
@@ -487,6 +487,8 @@ def main():
     ap.add_argument("--no-long-context", action="store_true", help="skip the config-4 (ctx 131072) measurements")
     ap.add_argument("--layers", type=int, default=0, help="override the number of target layers (debug)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-select-workspace", action="store_true",
+                    help="selection without its optional workspace: one cluster per list whatever their number")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -522,7 +524,8 @@ def main():
 
     # every rank owns a batch of its own (batch sharding): same shapes, rank-specific seed
     cfg_r = rank_config(cfg, rank, world)
-    si, pools, step, dp_host, q_host = build_step(cfg_r, dev, verify_flags=vflags)
+    si, pools, step, dp_host, q_host = build_step(cfg_r, dev, verify_flags=vflags,
+                                                  select_workspace=not args.no_select_workspace)
     step.run()
     torch.cuda.synchronize()
     counts = step.counts.cpu().numpy()
