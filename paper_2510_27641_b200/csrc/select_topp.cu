@@ -186,10 +186,20 @@ __device__ void scan_bins(Shared& sh, const double* mass, int nbins, double carr
   const int groups = nbins / kGroup;
   const int tid = threadIdx.x;
   const int lane = tid & 31;
-  if (tid < groups) {
+  // group sums: four threads per group add eight bins each (top bin first), then combine; the
+  // order is fixed, and consecutive threads read consecutive 64-byte pieces (a thread per group
+  // walking its 256 bytes put all lanes of a warp on one bank)
+  {
+    const int grp = tid >> 2, part = tid & 3;
     double s = 0.0;
-    for (int b = kGroup - 1; b >= 0; --b) s += mass[tid * kGroup + b];
-    sh.grp_mass[tid] = s;
+    if (grp < groups) {
+      const double* m8 = mass + grp * kGroup + part * 8;
+#pragma unroll
+      for (int b = 7; b >= 0; --b) s += m8[b];
+    }
+    const double s1 = s + __shfl_xor_sync(kFull, s, 1);      // (0+1), (2+3)
+    const double s2 = s1 + __shfl_xor_sync(kFull, s1, 2);    // all four quarters
+    if (grp < groups && part == 0) sh.grp_mass[grp] = s2;
   }
   __syncthreads();
   if (tid < 32) {
