@@ -250,3 +250,15 @@ def test_full_size_dense_baseline_of_config4(engine):
         go = step.out[0][b, :, hk * grp:(hk + 1) * grp, :].reshape(-1, d)
         gl = step.lse[0][b, :, hk * grp:(hk + 1) * grp].reshape(-1)
         check_attention(go, gl, ro, rl)
+
+
+def test_graft_entry_smoke_runs():
+    """The repository's smoke entry point (one small step checked against the oracle) stays in
+    working order as the launch plan of a step changes."""
+    import importlib
+    import sys
+    from pathlib import Path
+    root = str(Path(__file__).resolve().parents[1])
+    if root not in sys.path:
+        sys.path.insert(0, root)
+    importlib.import_module("__graft_entry__").smoke()
