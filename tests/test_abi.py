@@ -87,3 +87,33 @@ def test_product_path_never_imports_the_oracle():
     for f in (ROOT / "oracle").rglob("*"):
         if f.suffix in (".py", ".cpp"):
             assert "paper_2510_27641_b200" not in f.read_text(), f
+
+
+def test_select_workspace_query_follows_the_documented_rule(sa):
+    """specattn_select_workspace_bytes reads host fields only: a workspace is asked for exactly
+    when the default selection runs over multi-row lists of >= 2048 positions that are too few to
+    give every SM a CTA with one cluster each."""
+    L = sa.lib()
+
+    def need(n_target, batch, heads, gamma, Ls, **kw):
+        a = sa.SelectArgs()
+        a.struct_size = C.sizeof(sa.SelectArgs)
+        lm = (C.c_int32 * n_target)(*[j % 4 for j in range(n_target)])
+        a.n_draft_layers, a.n_target_layers, a.batch = 4, n_target, batch
+        a.n_draft_heads, a.gamma, a.n_groups, a.L_stride = heads, gamma, 1, Ls
+        a.layer_map = lm
+        for k, v in kw.items():
+            setattr(a, k, v)
+        return int(L.specattn_select_workspace_bytes(C.byref(a)))
+
+    assert need(1, 4, 16, 4, 131072) == 4 * 131072 * 4            # 4 lists x 8 CTAs: underfilled
+    assert need(8, 4, 16, 4, 131072) == 16 * 131072 * 4           # 16 lists x 8 = 128 < 148
+    assert need(32, 8, 12, 5, 32768) == 0                          # 32 lists x 8 CTAs fill the GPU
+    assert need(1, 4, 1, 1, 131072) == 0                           # single-row lists are read in place
+    assert need(1, 4, 16, 4, 1024) == 0                            # short rows
+    assert need(1, 4, 16, 4, 131072, per_step=1) == 0              # variants keep the cluster form
+    assert need(1, 4, 16, 4, 131072, chunk=16) == 0
+    assert need(1, 4, 16, 4, 131072, bisect_iters=10) == 0
+    assert L.specattn_select_workspace_bytes(None) == 0
+    bad = sa.SelectArgs()
+    assert L.specattn_select_workspace_bytes(C.byref(bad)) == 0   # struct_size not set
