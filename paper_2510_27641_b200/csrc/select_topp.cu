@@ -808,6 +808,9 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   const int wchunk4 = (((n4 + kWarps - 1) / kWarps) + 31) & ~31;
   const int w4_lo = min(n4, warp * wchunk4);
   const int w4_hi = min(n4, w4_lo + wchunk4);
+  // (in place) the kept positions as ballot words, four per 128 positions; the scan array is
+  // idle by now and no peer reads it after the level-1 gather
+  unsigned int* const keep_words = reinterpret_cast<unsigned int*>(r_mass);
   int wc = 0;
   if (!invalid && in_place) {
     for (int i0 = w4_lo; i0 < w4_hi; i0 += 32 * kIpUnroll) {
@@ -818,14 +821,21 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
         const int i4 = i0 + uu * 32 + lane;
         act[uu] = load_keys4(i4 < w4_hi ? i4 : n4, key[uu]);
       }
-      int c = 0;
 #pragma unroll
       for (int uu = 0; uu < kIpUnroll; ++uu) {
+        // 128 consecutive positions, four per lane: one ballot word per position-in-float4.
+        // The words are kept (lane e stores word e), so the write pass below never reads the
+        // row again.
         const int i4 = i0 + uu * 32 + lane;
+        unsigned int mine = 0u;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) c += (act[uu] && 4 * i4 + e < n_loc && key[uu][e] >= theta_key) ? 1 : 0;
+        for (int e = 0; e < 4; ++e) {
+          const unsigned int m = __ballot_sync(kFull, act[uu] && 4 * i4 + e < n_loc && key[uu][e] >= theta_key);
+          wc += __popc(m);
+          if (lane == e) mine = m;
+        }
+        if (lane < 4 && i0 + uu * 32 < w4_hi) keep_words[((i0 + uu * 32) >> 5) * 4 + lane] = mine;
       }
-      wc += __reduce_add_sync(kFull, c);
     }
   } else if (!invalid) {
     for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
@@ -857,37 +867,27 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     int* out = P.idx + out_list * P.idx_stride;
     long long pos = offset + sh.warp_cnt[warp];
     const unsigned int lt = (1u << lane) - 1u;
-    for (int i0 = w4_lo; i0 < w4_hi; i0 += 32 * kIpUnroll) {
-      unsigned int key[kIpUnroll][4];
-      bool act[kIpUnroll];
+    __syncwarp();  // this warp's ballot words are complete
+    for (int g4 = w4_lo; g4 < w4_hi; g4 += 32) {
+      // 128 consecutive positions, four per lane: ascending order is lane-major
+      const int i4 = g4 + lane;
+      const uint4 words = *reinterpret_cast<const uint4*>(keep_words + (g4 >> 5) * 4);
+      const unsigned int mw[4] = {words.x, words.y, words.z, words.w};
+      unsigned int before = 0, total_kept = 0;
 #pragma unroll
-      for (int uu = 0; uu < kIpUnroll; ++uu) {
-        const int i4 = i0 + uu * 32 + lane;
-        act[uu] = load_keys4(i4 < w4_hi ? i4 : n4, key[uu]);
+      for (int e = 0; e < 4; ++e) {
+        before += __popc(mw[e] & lt);
+        total_kept += __popc(mw[e]);
       }
+      long long my = pos + before;
 #pragma unroll
-      for (int uu = 0; uu < kIpUnroll; ++uu) {
-        // 128 consecutive positions, four per lane: ascending order is lane-major
-        const int i4 = i0 + uu * 32 + lane;
-        bool keep[4];
-        unsigned int before = 0, total_kept = 0;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          keep[e] = act[uu] && 4 * i4 + e < n_loc && key[uu][e] >= theta_key;
-          const unsigned int m = __ballot_sync(kFull, keep[e]);
-          before += __popc(m & lt);
-          total_kept += __popc(m);
+      for (int e = 0; e < 4; ++e) {
+        if ((mw[e] >> lane) & 1u) {
+          if (my < P.idx_stride) out[my] = lo + 4 * i4 + e;
+          ++my;
         }
-        long long my = pos + before;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (keep[e]) {
-            if (my < P.idx_stride) out[my] = lo + 4 * i4 + e;
-            ++my;
-          }
-        }
-        pos += total_kept;
       }
+      pos += total_kept;
     }
   } else if (!invalid) {
     int* out = P.idx + out_list * P.idx_stride;
