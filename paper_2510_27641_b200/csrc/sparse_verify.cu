@@ -735,7 +735,11 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   // =============================== consumer warps ===========================================
   const int mt = warp / WPM;            // 16-row slab of the query block
   const int wr = warp % WPM;            // role inside the slab
-  const int parity = (WPM == 4) ? (wr >> 1) : wr;   // which stages (it % 2) this warp reads
+  // which tiles (it % 2) this warp reads.  Warps w and w + 4 share an SM sub-partition: they take
+  // opposite parities, so that one is in its tensor phase while the other waits, exponentiates
+  // or loads fragments (with equal parities both wait for the same tile and collide in every
+  // phase: the tensor pipe was 47 % busy)
+  const int parity = ((WPM == 4) ? (wr >> 1) : wr) ^ ((warp >> 2) & 1);
   const int g = lane >> 2, tq = lane & 3;
   const int lm = lane >> 3, lr = lane & 7;  // ldmatrix: matrix id, row within it
   const uint32_t q_addr = smem_u32(sh.q) + (mt * 16 + (lm & 1) * 8 + lr) * kPitch + (lm >> 1) * 16;
