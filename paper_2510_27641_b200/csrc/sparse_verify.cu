@@ -293,7 +293,8 @@ struct WarpState {
 // `valid` = number of existing keys in the block (>= 1; rows beyond it hold finite padding).
 // `tail_begin` = index inside the block of the first in-flight token (>= 32: none); rows g and
 // g+8 of the slab may see in-flight tokens j <= lim0 / lim1 only (causal among themselves).
-__device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&qf)[8][4], uint32_t k_addr,
+template <bool kQReload>
+__device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&qf)[8][4], uint32_t q_addr, uint32_t k_addr,
                                                uint32_t v_addr, int valid, float scale_log2, int tq,
                                                int tail_begin, int lim0, int lim1) {
   float sc[4][4];
@@ -301,13 +302,21 @@ __device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&q
   for (int n = 0; n < 4; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
 #pragma unroll
   for (int kk = 0; kk < 8; ++kk) {
-    uint32_t k0[4], k1[4];
+    uint32_t qa[4], k0[4], k1[4];
+    if (kQReload) {
+      ldmatrix_x4(qa, q_addr + kk * 32);
+    } else {
+      qa[0] = qf[kk][0];
+      qa[1] = qf[kk][1];
+      qa[2] = qf[kk][2];
+      qa[3] = qf[kk][3];
+    }
     ldmatrix_x4(k0, k_addr + kk * 32);
     ldmatrix_x4(k1, k_addr + 16 * kPitch + kk * 32);
-    mma_bf16(sc[0], qf[kk], k0[0], k0[1]);
-    mma_bf16(sc[1], qf[kk], k0[2], k0[3]);
-    mma_bf16(sc[2], qf[kk], k1[0], k1[1]);
-    mma_bf16(sc[3], qf[kk], k1[2], k1[3]);
+    mma_bf16(sc[0], qa, k0[0], k0[1]);
+    mma_bf16(sc[1], qa, k0[2], k0[3]);
+    mma_bf16(sc[2], qa, k1[0], k1[1]);
+    mma_bf16(sc[3], qa, k1[2], k1[3]);
   }
   // raw scores stay unscaled: exp2(s * c - m * c) is one fused multiply-add per element
   if (valid < 32) {  // only the last block of a segment has missing keys
@@ -766,13 +775,20 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     const int lim1 = (mt * 16 + g + 8) / P.grp + P.tail_off;
 
     // query fragments of this unit
+    // With two warps per slab (query blocks of more than 32 rows) the query fragments are
+    // re-read from shared memory for every block instead of being held in 32 registers: the
+    // compiler spends those on fragment prefetch (dense, 40 rows: 3.11 -> 3.37 TB/s); with
+    // four warps per slab the same change loses 3 %.
+    constexpr bool kQReload = (WPM == 2);
     uint32_t qf[8][4];
     ok = mbar_wait(&sh.q_full, seg & 1u, &sh.abort_flag);
     if (!ok) sh.abort_flag = 1;
+    if (!kQReload) {
 #pragma unroll
-    for (int kk = 0; kk < 8; ++kk) ldmatrix_x4(qf[kk], q_addr + kk * 32);
-    __syncwarp();
-    if (ok && lane == 0) mbar_arrive(&sh.q_empty);
+      for (int kk = 0; kk < 8; ++kk) ldmatrix_x4(qf[kk], q_addr + kk * 32);
+      __syncwarp();
+      if (ok && lane == 0) mbar_arrive(&sh.q_empty);
+    }
 
     WarpState st;
 #pragma unroll
@@ -794,18 +810,22 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       if (WPM == 4) {
         const int key0 = (wr & 1) * 32;
         if (key0 < ntok)
-          attend_block32(st, qf, k_base + key0 * kPitch, v_base + key0 * kPitch, ntok - key0, P.scale_log2, tq,
+          attend_block32<kQReload>(st, qf, q_addr, k_base + key0 * kPitch, v_base + key0 * kPitch, ntok - key0, P.scale_log2, tq,
                          tb - key0, lim0, lim1);
       } else {
-        attend_block32(st, qf, k_base, v_base, ntok, P.scale_log2, tq, tb, lim0, lim1);
+        attend_block32<kQReload>(st, qf, q_addr, k_base, v_base, ntok, P.scale_log2, tq, tb, lim0, lim1);
         if (32 < ntok)
-          attend_block32(st, qf, k_base + 32 * kPitch, v_base + 32 * kPitch, ntok - 32, P.scale_log2, tq,
+          attend_block32<kQReload>(st, qf, q_addr, k_base + 32 * kPitch, v_base + 32 * kPitch, ntok - 32, P.scale_log2, tq,
                          tb - 32, lim0, lim1);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.empty[s]);
     }
 
+    if (kQReload) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.q_empty);   // the query tile was read for the last time
+    }
     // ---- end of the segment: row sums across the quad, then combine the slab's warps ---------
     if (paired && !peer_seen) {  // the peer's arrival at kernel start: long past by now
       cluster_wait();
