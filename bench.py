@@ -485,6 +485,8 @@ def main():
                     help="force one implementation of sparse_verify (default: the library picks by shape)")
     ap.add_argument("--long-context", action="store_true", help="only run the config-4 (ctx 131072) measurements")
     ap.add_argument("--no-long-context", action="store_true", help="skip the config-4 (ctx 131072) measurements")
+    ap.add_argument("--long-context-layers", type=int, default=8,
+                    help="target layers of config 4 held on the device (2.1 GB of K/V each)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of target layers (debug)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-select-workspace", action="store_true",
@@ -519,7 +521,8 @@ def main():
         return
 
     if args.long_context:
-        print(json.dumps({"long_context": long_context(dev, reps=min(10, max(2, args.steps)))}))
+        print(json.dumps({"long_context": long_context(dev, reps=min(10, max(2, args.steps)),
+                                                       n_layers=args.long_context_layers)}))
         return
 
     # every rank owns a batch of its own (batch sharding): same shapes, rank-specific seed
@@ -642,7 +645,7 @@ def main():
     if rank == 0 and not args.no_long_context:
         del step, pools
         torch.cuda.empty_cache()
-        line["extra"]["long_context"] = long_context(dev)
+        line["extra"]["long_context"] = long_context(dev, n_layers=args.long_context_layers)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

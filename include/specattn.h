@@ -111,7 +111,7 @@ extern "C" {
  * memory of one thread-block cluster (at most 8 CTAs per list, one launch).  With it, and for
  * the default selection (no variant) over rows of >= 2048 positions when the lists are so few
  * that one cluster each would leave SMs idle (lists x CTAs per cluster < 148), the call runs two
- * launches: every list's rows are summed by CTAs of 1024 positions each -- in the same order,
+ * launches: every list's rows are summed by CTAs of 512 positions each -- in the same order,
  * so a[] has the same bits -- into the workspace, and the search then reads a[] from there; the
  * lists are the same, the GPU is filled whatever the number of lists.  The workspace holds no
  * state between calls; two calls that may overlap on the GPU need separate workspaces.

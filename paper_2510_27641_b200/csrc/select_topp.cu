@@ -37,7 +37,7 @@
 // copied to shared memory at all but re-read from global memory (L2) by the later passes,
 // which shrinks a CTA to ~51 KB of shared memory so that four of them share an SM.
 // With a workspace and few lists the call becomes two launches: aggregate_rows_kernel sums the
-// rows with 1024 positions per CTA (the whole GPU streams, however few the lists) and the
+// rows with 512 positions per CTA (the whole GPU streams, however few the lists) and the
 // search runs in place over that sum.
 #include <cooperative_groups.h>
 #include <cuda_runtime.h>
@@ -965,14 +965,15 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   csync();  // nobody leaves while its shared memory may still be read remotely
 }
 
-// First launch of the two-launch form: a[i] = +0 + the contributing rows in order, for 1024
+// First launch of the two-launch form: a[i] = +0 + the contributing rows in order, for 512
 // positions per CTA, so that the number of CTAs streaming the rows from HBM does not depend on
 // the number of lists.  The adds are the ones of the cluster kernel (binary32, same order), so
 // the bits of a[] are the same.  A negative input, which a sum could hide, poisons its
 // position with NaN: the search then reports the list as invalid like the cluster kernel does.
-constexpr int kAggPositions = kThreads * 4;
-constexpr int kAggUnroll = 8;
-__global__ void __launch_bounds__(kThreads) aggregate_rows_kernel(const __grid_constant__ SelectParams P,
+constexpr int kAggThreads = 128;
+constexpr int kAggPositions = kAggThreads * 4;
+constexpr int kAggUnroll = 16;
+__global__ void __launch_bounds__(kAggThreads) aggregate_rows_kernel(const __grid_constant__ SelectParams P,
                                                                   float* __restrict__ out) {
   __shared__ long long row_off[SPECATTN_MAX_ROWS_PER_LIST];
   __shared__ int n_rows;
@@ -1237,7 +1238,7 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   if (two_launch) {
     const dim3 grid(static_cast<unsigned>((A.L_stride + specattn::kAggPositions - 1) / specattn::kAggPositions),
                     static_cast<unsigned>(n_lists), 1);
-    specattn::aggregate_rows_kernel<<<grid, specattn::kThreads, 0, cfg.stream>>>(P, static_cast<float*>(A.workspace));
+    specattn::aggregate_rows_kernel<<<grid, specattn::kAggThreads, 0, cfg.stream>>>(P, static_cast<float*>(A.workspace));
     if (cudaGetLastError() != cudaSuccess) return SPECATTN_ERR_CUDA;
     specattn::g_launch_count.fetch_add(1, std::memory_order_relaxed);
     // the search may be scheduled while the aggregation drains; it waits before reading a[]
