@@ -101,7 +101,7 @@ struct VShared {
   volatile int abort_flag;
   // cluster merge (two CTAs per unit): the odd CTA's records land here, in the even CTA
   unsigned long long peer_full;
-  float peer_rec[(MT <= 2) ? MT : 1][(MT <= 2) ? kRec : 1];
+  alignas(16) float peer_rec[(MT <= 2) ? MT : 1][(MT <= 2) ? kRec : 1];
 };
 
 __device__ __forceinline__ int unit_count(const VerifyParams& P, int u) {
@@ -882,34 +882,32 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
                               ((sh.part_start[u] & 1) == 0);
       if (pair_merge) {
         if (cluster_cta_rank() == 1) {
-          const uint32_t dst = map_to_cta(smem_u32(sh.peer_rec[mt]), 0) + lane * 4;
+          // 17 16-byte remote stores per lane (lane-major float4 records)
+          const uint32_t dst = map_to_cta(smem_u32(sh.peer_rec[mt]), 0) + lane * 16;
 #pragma unroll
-          for (int n = 0; n < 16; ++n)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) st_cluster_f32(dst + (n * 4 + i) * 128, acc[n][i]);
-          st_cluster_f32(dst + 64 * 128, m0);
-          st_cluster_f32(dst + 65 * 128, l0);
-          st_cluster_f32(dst + 66 * 128, m1);
-          st_cluster_f32(dst + 67 * 128, l1);
+          for (int n = 0; n < 16; ++n) st_cluster_v4(dst + n * 512, acc[n][0], acc[n][1], acc[n][2], acc[n][3]);
+          st_cluster_v4(dst + 16 * 512, m0, l0, m1, l1);
           __syncwarp();
           if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&sh.peer_full), 0));
         } else {
           if (!mbar_wait_cluster(&sh.peer_full, 0u, &sh.abort_flag)) { sh.abort_flag = 1; ok = false; break; }
-          const float* rec = sh.peer_rec[mt];
+          const float4* rec = reinterpret_cast<const float4*>(sh.peer_rec[mt]) + lane;
+          const float4 ml = rec[16 * 32];
           float mn, ao, ai;
-          merge_scales(m0, rec[64 * 32 + lane], mn, ao, ai);
-          l0 = l0 * ao + rec[65 * 32 + lane] * ai;
+          merge_scales(m0, ml.x, mn, ao, ai);
+          l0 = l0 * ao + ml.y * ai;
           m0 = mn;
           float mn1, ao1, ai1;
-          merge_scales(m1, rec[66 * 32 + lane], mn1, ao1, ai1);
-          l1 = l1 * ao1 + rec[67 * 32 + lane] * ai1;
+          merge_scales(m1, ml.z, mn1, ao1, ai1);
+          l1 = l1 * ao1 + ml.w * ai1;
           m1 = mn1;
 #pragma unroll
           for (int n = 0; n < 16; ++n) {
-            acc[n][0] = acc[n][0] * ao + rec[(n * 4 + 0) * 32 + lane] * ai;
-            acc[n][1] = acc[n][1] * ao + rec[(n * 4 + 1) * 32 + lane] * ai;
-            acc[n][2] = acc[n][2] * ao1 + rec[(n * 4 + 2) * 32 + lane] * ai1;
-            acc[n][3] = acc[n][3] * ao1 + rec[(n * 4 + 3) * 32 + lane] * ai1;
+            const float4 r = rec[n * 32];
+            acc[n][0] = acc[n][0] * ao + r.x * ai;
+            acc[n][1] = acc[n][1] * ao + r.y * ai;
+            acc[n][2] = acc[n][2] * ao1 + r.z * ai1;
+            acc[n][3] = acc[n][3] * ao1 + r.w * ai1;
           }
           finish = true;
         }
