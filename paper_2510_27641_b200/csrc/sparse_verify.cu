@@ -88,7 +88,7 @@ template <int MT, int WPM>
 struct VShared {
   alignas(128) unsigned char kv[kStages][2][kStageTok * kPitch];
   alignas(16) unsigned char q[MT * 16 * kPitch];
-  float scratch[MT][WPM / 2][kRec];
+  alignas(16) float scratch[MT][WPM / 2][kRec];
   alignas(8) unsigned long long full[kStages];
   unsigned long long empty[kStages];
   unsigned long long q_full, q_empty;
@@ -840,33 +840,31 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
 #pragma unroll
     for (int half = WPM / 2; half >= 1; half >>= 1) {
       if (wr >= half && wr < 2 * half) {
-        float* rec = sh.scratch[mt][wr - half];
+        // lane-major float4 records: 17 16-byte stores per lane
+        float4* rec = reinterpret_cast<float4*>(sh.scratch[mt][wr - half]) + lane;
 #pragma unroll
-        for (int n = 0; n < 16; ++n)
-#pragma unroll
-          for (int i = 0; i < 4; ++i) rec[(n * 4 + i) * 32 + lane] = acc[n][i];
-        rec[64 * 32 + lane] = m0;
-        rec[65 * 32 + lane] = l0;
-        rec[66 * 32 + lane] = m1;
-        rec[67 * 32 + lane] = l1;
+        for (int n = 0; n < 16; ++n) rec[n * 32] = make_float4(acc[n][0], acc[n][1], acc[n][2], acc[n][3]);
+        rec[16 * 32] = make_float4(m0, l0, m1, l1);
       }
       named_bar_sync(1 + mt, WPM * 32);
       if (wr < half) {
-        const float* rec = sh.scratch[mt][wr];
+        const float4* rec = reinterpret_cast<const float4*>(sh.scratch[mt][wr]) + lane;
+        const float4 ml = rec[16 * 32];
         float mn, ao, ai;
-        merge_scales(m0, rec[64 * 32 + lane], mn, ao, ai);
-        l0 = l0 * ao + rec[65 * 32 + lane] * ai;
+        merge_scales(m0, ml.x, mn, ao, ai);
+        l0 = l0 * ao + ml.y * ai;
         m0 = mn;
         float mn1, ao1, ai1;
-        merge_scales(m1, rec[66 * 32 + lane], mn1, ao1, ai1);
-        l1 = l1 * ao1 + rec[67 * 32 + lane] * ai1;
+        merge_scales(m1, ml.z, mn1, ao1, ai1);
+        l1 = l1 * ao1 + ml.w * ai1;
         m1 = mn1;
 #pragma unroll
         for (int n = 0; n < 16; ++n) {
-          acc[n][0] = acc[n][0] * ao + rec[(n * 4 + 0) * 32 + lane] * ai;
-          acc[n][1] = acc[n][1] * ao + rec[(n * 4 + 1) * 32 + lane] * ai;
-          acc[n][2] = acc[n][2] * ao1 + rec[(n * 4 + 2) * 32 + lane] * ai1;
-          acc[n][3] = acc[n][3] * ao1 + rec[(n * 4 + 3) * 32 + lane] * ai1;
+          const float4 r = rec[n * 32];
+          acc[n][0] = acc[n][0] * ao + r.x * ai;
+          acc[n][1] = acc[n][1] * ao + r.y * ai;
+          acc[n][2] = acc[n][2] * ao1 + r.z * ai1;
+          acc[n][3] = acc[n][3] * ao1 + r.w * ai1;
         }
       }
       named_bar_sync(1 + mt, WPM * 32);
