@@ -911,15 +911,12 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         }
       } else if (!whole) {
         // publish this CTA's share of the unit, then see whether it was the last to arrive
-        float* rec = P.partials + (static_cast<size_t>(2 * blockIdx.x + (a == a0 ? 0 : 1)) * MT + mt) * kRec;
+        // lane-major float4 records, as in shared memory
+        float4* rec = reinterpret_cast<float4*>(
+                          P.partials + (static_cast<size_t>(2 * blockIdx.x + (a == a0 ? 0 : 1)) * MT + mt) * kRec) + lane;
 #pragma unroll
-        for (int n = 0; n < 16; ++n)
-#pragma unroll
-          for (int i = 0; i < 4; ++i) __stcg(rec + (n * 4 + i) * 32 + lane, acc[n][i]);
-        __stcg(rec + 64 * 32 + lane, m0);
-        __stcg(rec + 65 * 32 + lane, l0);
-        __stcg(rec + 66 * 32 + lane, m1);
-        __stcg(rec + 67 * 32 + lane, l1);
+        for (int n = 0; n < 16; ++n) __stcg(rec + n * 32, make_float4(acc[n][0], acc[n][1], acc[n][2], acc[n][3]));
+        __stcg(rec + 16 * 32, make_float4(m0, l0, m1, l1));
         __threadfence();
         __syncwarp();
         const int i_lo = aligned ? sh.part_start[u] : cta_of_atom(us, N, NP);
@@ -935,28 +932,31 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           // common maxima, then one scaled accumulation pass with independent loads.
           m0 = m1 = -INFINITY;
           for (int i = i_lo; i <= i_hi; ++i) {
-            const float* r2 = P.partials +
-                (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * MT + mt) * kRec;
-            m0 = fmaxf(m0, __ldcg(r2 + 64 * 32 + lane));
-            m1 = fmaxf(m1, __ldcg(r2 + 66 * 32 + lane));
+            const float4* r2 = reinterpret_cast<const float4*>(P.partials +
+                (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * MT + mt) * kRec) + lane;
+            const float4 ml = __ldcg(r2 + 16 * 32);
+            m0 = fmaxf(m0, ml.x);
+            m1 = fmaxf(m1, ml.z);
           }
           const float base0 = (m0 == -INFINITY) ? 0.f : m0, base1 = (m1 == -INFINITY) ? 0.f : m1;
           l0 = l1 = 0.f;
 #pragma unroll
           for (int n = 0; n < 16; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
           for (int i = i_lo; i <= i_hi; ++i) {
-            const float* r2 = P.partials +
-                (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * MT + mt) * kRec;
-            const float w0 = ex2(__ldcg(r2 + 64 * 32 + lane) - base0);
-            const float w1 = ex2(__ldcg(r2 + 66 * 32 + lane) - base1);
-            l0 += __ldcg(r2 + 65 * 32 + lane) * w0;
-            l1 += __ldcg(r2 + 67 * 32 + lane) * w1;
+            const float4* r2 = reinterpret_cast<const float4*>(P.partials +
+                (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * MT + mt) * kRec) + lane;
+            const float4 ml = __ldcg(r2 + 16 * 32);
+            const float w0 = ex2(ml.x - base0);
+            const float w1 = ex2(ml.z - base1);
+            l0 += ml.y * w0;
+            l1 += ml.w * w1;
 #pragma unroll
             for (int n = 0; n < 16; ++n) {
-              acc[n][0] += __ldcg(r2 + (n * 4 + 0) * 32 + lane) * w0;
-              acc[n][1] += __ldcg(r2 + (n * 4 + 1) * 32 + lane) * w0;
-              acc[n][2] += __ldcg(r2 + (n * 4 + 2) * 32 + lane) * w1;
-              acc[n][3] += __ldcg(r2 + (n * 4 + 3) * 32 + lane) * w1;
+              const float4 r = __ldcg(r2 + n * 32);
+              acc[n][0] += r.x * w0;
+              acc[n][1] += r.y * w0;
+              acc[n][2] += r.z * w1;
+              acc[n][3] += r.w * w1;
             }
           }
           if (lane == 0) P.counters[u * kCountersPerUnit + mt] = 0u;  // ready for the next call
