@@ -611,7 +611,7 @@ def main():
                        "global_batch": cfg.batch * world, "ctx": cfg.ctx, "page_size": cfg.page_size,
                        "gamma": cfg.gamma, "p": cfg.p, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
                        "head_dim": cfg.head_dim, "parallelism": f"batch-sharded x{world}, no collective",
-                       "launch": f"CUDA graph of 1 select + {len(step.plans)} plan + {step.n_layers} verify launches",
+                       "launch": f"CUDA graph of 1 select + 1 plan launch ({len(step.plans)} plans) + {step.n_layers} verify launches",
                        "l2": "inputs exceed L2: 252 MB of draft rows and 1.3 GB of gathered K/V per step"},
             "e2e": {"value": round(us_e2e, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(n_step * args.steps),

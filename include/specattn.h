@@ -274,6 +274,11 @@ int specattn_sparse_verify(const specattn_verify_args* args, void* cuda_stream);
  * the mma.sync engine reads plans. */
 size_t specattn_verify_plan_bytes(const specattn_verify_args* args);
 int specattn_verify_plan(const specattn_verify_args* args, void* plan, size_t plan_bytes, void* cuda_stream);
+/* The same for n launches at once (HOST arrays of n argument structs, plan buffers and their
+ * sizes): one kernel launch per eight plans instead of one per plan -- a step whose target
+ * layers share the lists of four draft layers needs four plans. */
+int specattn_verify_plan_many(const specattn_verify_args* const* args, void* const* plans,
+                              const size_t* plan_bytes, int32_t n, void* cuda_stream);
 
 /* ========================================================================================
  * specattn_sparse_verify_static -- specattn_sparse_verify for callers that cannot allocate.

@@ -17,7 +17,7 @@ __all__ = ["select_topp", "sparse_verify", "sparse_verify_static", "verify_works
            "SelectArgs", "VerifyArgs", "StepHostArgs", "lib", "SpecAttnError",
            "ROW_OK", "ROW_INVALID_PROB", "ROW_OVERFLOW", "ROW_BAD_INDEX", "ROW_TIMEOUT",
            "VERIFY_LISTS_STABLE", "VERIFY_ENGINE_MMA_SYNC", "VERIFY_ENGINE_TCGEN05", "verify_plan",
-           "verify_plan_buffer"]
+           "verify_plan_buffer", "verify_plan_many"]
 
 ROW_OK, ROW_INVALID_PROB, ROW_OVERFLOW, ROW_BAD_INDEX, ROW_TIMEOUT = 0, 1, 2, 4, 8
 VERIFY_LISTS_STABLE = 1
@@ -93,6 +93,9 @@ def lib() -> C.CDLL:
         L.specattn_verify_plan_bytes.restype = C.c_size_t
         L.specattn_verify_plan.argtypes = [C.POINTER(VerifyArgs), C.c_void_p, C.c_size_t, C.c_void_p]
         L.specattn_verify_plan.restype = C.c_int
+        L.specattn_verify_plan_many.argtypes = [C.POINTER(C.POINTER(VerifyArgs)), C.POINTER(C.c_void_p),
+                                                C.POINTER(C.c_size_t), C.c_int32, C.c_void_p]
+        L.specattn_verify_plan_many.restype = C.c_int
         L.specattn_sparse_verify_static.argtypes = [C.POINTER(VerifyArgs), C.c_void_p]
         L.specattn_sparse_verify_static.restype = C.c_int
         L.specattn_verify_step_host.argtypes = [C.POINTER(StepHostArgs), C.c_void_p]
@@ -306,6 +309,18 @@ def verify_plan(args: VerifyArgs, plan: torch.Tensor, stream=None) -> None:
                                     _stream_ptr(stream))
     if rc != 0:
         raise SpecAttnError(rc, "specattn_verify_plan")
+
+
+def verify_plan_many(args: Sequence[VerifyArgs], plans: Sequence[torch.Tensor], stream=None) -> None:
+    """specattn_verify_plan_many: the plans of several launches in one kernel launch."""
+    n = len(args)
+    assert len(plans) == n
+    a = (C.POINTER(VerifyArgs) * n)(*[C.pointer(x) for x in args])
+    p = (C.c_void_p * n)(*[t.data_ptr() for t in plans])
+    b = (C.c_size_t * n)(*[t.numel() * t.element_size() for t in plans])
+    rc = lib().specattn_verify_plan_many(a, p, b, n, _stream_ptr(stream))
+    if rc != 0:
+        raise SpecAttnError(rc, "specattn_verify_plan_many")
 
 
 def sparse_verify_static(args: VerifyArgs, stream=None) -> None:

@@ -150,7 +150,7 @@ __host__ __device__ inline size_t plan_ints(int U, int grid) {
 }
 
 // One CTA computes what every CTA of a verify launch would compute for itself at start-up.
-__global__ void __launch_bounds__(256, 1) verify_plan_kernel(const __grid_constant__ VerifyParams P, int* plan, int G) {
+__device__ __forceinline__ void plan_body(const VerifyParams& P, int* plan, int G) {
   __shared__ int unit_start[kMaxUnits + 1];
   __shared__ int part_start[kAlignedMaxUnits + 1];
   __shared__ int cand_parts[kCandidates], cand_max[kCandidates];
@@ -281,6 +281,22 @@ __global__ void __launch_bounds__(256, 1) verify_plan_kernel(const __grid_consta
     plan[7] = P.dense;
     plan[0] = kPlanMagic;
   }
+}
+
+__global__ void __launch_bounds__(256, 1) verify_plan_kernel(const __grid_constant__ VerifyParams P, int* plan, int G) {
+  plan_body(P, plan, G);
+}
+
+// The plans of several launches (one per draft layer whose lists the step's layers share) in
+// one launch, one CTA each.
+constexpr int kPlanBatch = 8;
+struct PlanBatch {
+  VerifyParams p[kPlanBatch];
+  int* plan[kPlanBatch];
+  int G;
+};
+__global__ void __launch_bounds__(256, 1) verify_plan_many_kernel(const __grid_constant__ PlanBatch B) {
+  plan_body(B.p[blockIdx.x], B.plan[blockIdx.x], B.G);
 }
 
 // Online-softmax state of one warp: rows g and g+8 of its 16-row slab, 128 output columns.
@@ -1231,6 +1247,53 @@ extern "C" int specattn_verify_plan(const specattn_verify_args* args, void* plan
     return SPECATTN_ERR_CUDA;
   }
   specattn::g_launch_count.fetch_add(1, std::memory_order_relaxed);
+  return SPECATTN_OK;
+}
+
+extern "C" int specattn_verify_plan_many(const specattn_verify_args* const* args, void* const* plans,
+                                         const size_t* plan_bytes, int32_t n, void* cuda_stream) {
+  if (n < 0) return SPECATTN_ERR_RANGE;
+  if (n == 0) return SPECATTN_OK;
+  if (args == nullptr || plans == nullptr || plan_bytes == nullptr) return SPECATTN_ERR_NULL;
+  const int n_ctas = specattn::device_sm_count();
+  if (n_ctas <= 0) return SPECATTN_ERR_CUDA;
+  for (int i = 0; i < n; ++i) {  // everything is checked before anything is launched
+    const int v = specattn::validate(args[i]);
+    if (v != SPECATTN_OK) return v;
+    const specattn_verify_args& A = *args[i];
+    if (plans[i] == nullptr || !A.kv_len) return SPECATTN_ERR_NULL;
+    if (!A.dense && !A.counts) return SPECATTN_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(plans[i]) % 16 != 0) return SPECATTN_ERR_ALIGN;
+    if (plan_bytes[i] < specattn::plan_ints(A.batch * A.n_kv_heads, n_ctas) * sizeof(int)) return SPECATTN_ERR_WORKSPACE;
+  }
+  for (int i0 = 0; i0 < n; i0 += specattn::kPlanBatch) {
+    specattn::PlanBatch B;
+    memset(&B, 0, sizeof(B));
+    int m = 0;
+    for (int i = i0; i < n && i < i0 + specattn::kPlanBatch; ++i) {
+      if (args[i]->batch == 0) continue;
+      B.p[m] = specattn::make_params(*args[i]);
+      B.plan[m] = static_cast<int*>(plans[i]);
+      ++m;
+    }
+    if (m == 0) continue;
+    B.G = n_ctas;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(static_cast<unsigned>(m), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, specattn::verify_plan_many_kernel, B) != cudaSuccess) {
+      cudaGetLastError();
+      return SPECATTN_ERR_CUDA;
+    }
+    specattn::g_launch_count.fetch_add(1, std::memory_order_relaxed);
+  }
   return SPECATTN_OK;
 }
 

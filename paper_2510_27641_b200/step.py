@@ -11,7 +11,7 @@ from typing import Sequence
 import torch
 
 from . import (SelectArgs, VerifyArgs, SpecAttnError, VERIFY_LISTS_STABLE, lib, make_select_args, make_verify_args,
-               verify_plan, verify_plan_buffer,
+               verify_plan_buffer, verify_plan_many,
                verify_step_host, verify_workspace, _stream_ptr)
 
 __all__ = ["VerifyStep"]
@@ -90,9 +90,11 @@ class VerifyStep:
             raise SpecAttnError(rc, "specattn_select_topp")
 
     def run_plans(self, stream=None):
-        """One small launch per distinct list set: the work partition its verify launches share."""
-        for plan, j in self.plans.values():
-            verify_plan(self.verify_args[j], plan, stream)
+        """The work partitions that the verify launches of each distinct list set share: one
+        small launch for up to eight of them."""
+        if self.plans:
+            verify_plan_many([self.verify_args[j] for _, j in self.plans.values()],
+                             [plan for plan, _ in self.plans.values()], stream)
 
     def run_verify(self, j: int, stream=None):
         rc = lib().specattn_sparse_verify(C.byref(self.verify_args[j]), _stream_ptr(stream))
@@ -120,4 +122,4 @@ class VerifyStep:
         n_select = 0
         if self.select_args is not None:
             n_select = 2 if self.select_args.workspace else 1   # aggregation + search, or the cluster form
-        return n_select + len(self.plans) + self.n_layers
+        return n_select + (len(self.plans) + 7) // 8 + self.n_layers

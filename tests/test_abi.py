@@ -30,7 +30,7 @@ def test_library_exports_every_declared_symbol(sa):
     assert {"specattn_select_topp", "specattn_sparse_verify", "specattn_verify_workspace_bytes",
             "specattn_verify_workspace_init", "specattn_verify_step_host", "specattn_status_string",
             "specattn_kernel_launch_count", "specattn_verify_plan", "specattn_verify_plan_bytes",
-            "specattn_select_workspace_bytes"} <= set(names)
+            "specattn_select_workspace_bytes", "specattn_verify_plan_many"} <= set(names)
     L = sa.lib()
     for n in names:
         assert hasattr(L, n), f"{n} is declared in specattn.h but not exported"

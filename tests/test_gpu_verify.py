@@ -277,7 +277,27 @@ def test_precomputed_work_partition_gives_the_same_results_and_is_ignored_when_i
     assert sa.lib().specattn_sparse_verify(C.byref(at), None) == 0
     torch.cuda.synchronize()
     check_attention(o, l, *ref_t)
+    # several plans in one launch: the same bits as one launch each (here 11: two launches of <= 8)
+    variants = []
+    for k in range(11):
+        cnt_k = torch.clamp(cnt_d - 3 * k, min=0)
+        _, _, ak = run(None, cnt=cnt_k)
+        variants.append((ak, cnt_k))
+    singles = []
+    for ak, _ in variants:
+        pk = sa.verify_plan_buffer(ak)
+        sa.verify_plan(ak, pk)
+        singles.append(pk)
+    many = [sa.verify_plan_buffer(ak) for ak, _ in variants]
+    n0 = sa.kernel_launch_count()
+    sa.verify_plan_many([ak for ak, _ in variants], many)
+    torch.cuda.synchronize()
+    assert sa.kernel_launch_count() - n0 == 2
+    for pk, pm in zip(singles, many):
+        assert torch.equal(pk, pm)
     # argument errors
     small = torch.zeros(4, dtype=torch.int32, device=dev())
+    with pytest.raises(sa.SpecAttnError):
+        sa.verify_plan_many([a0], [small])
     assert sa.lib().specattn_verify_plan(C.byref(a0), small.data_ptr(), 16, None) == -5
     assert sa.lib().specattn_verify_plan(C.byref(a0), None, 1 << 20, None) == -1
