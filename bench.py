@@ -625,8 +625,16 @@ def main():
                       "kv_touched_fraction": round(kv_bytes_step / dense_kv_step, 5),
                       "sequences_per_s": round(cfg.batch * world / us_step * 1e6, 1)}}
 
+    # The sections below add context to the line; a failure in one of them (say, no memory left
+    # for the long-context pools on a shared GPU) is recorded and must not lose the step's numbers.
+    def extra(name, fn):
+        try:
+            line["extra"][name] = fn()
+        except Exception as e:  # noqa: BLE001
+            line["extra"][name] = {"error": f"{type(e).__name__}: {e}"[:300]}
+
     if rank == 0:
-        line["extra"]["select_variants"] = select_variants(step, cfg_r)
+        extra("select_variants", lambda: select_variants(step, cfg_r))
     if rank == 0 and not args.no_cpu_baseline:
         smp = OracleSample(cfg_r, si, n_attn_layers=8, pools=pools)
         us_cpu, sample = smp.step_us()
@@ -634,18 +642,19 @@ def main():
                                 "sample": sample}
     if rank == 0 and not args.no_topp_sweep:
         del g_step, g_verify, g_select
-        sweep = topp_sweep(dev)
-        line["extra"]["topp_sweep"] = sweep
-        # the second half of the metric: rows/s of the selection alone, per row length (geometric
-        # mean over the three families and three p of config 2)
-        by_n = {}
-        for k, v in sweep.items():
-            by_n.setdefault(k.split("/")[1], []).append(v["rows_per_s"])
-        line["extra"]["topp_rows_per_s"] = {n: round(float(np.exp(np.mean(np.log(v))))) for n, v in by_n.items()}
+        extra("topp_sweep", lambda: topp_sweep(dev))
+        sweep = line["extra"]["topp_sweep"]
+        if "error" not in sweep:
+            # the second half of the metric: rows/s of the selection alone, per row length
+            # (geometric mean over the three families and three p of config 2)
+            by_n = {}
+            for k, v in sweep.items():
+                by_n.setdefault(k.split("/")[1], []).append(v["rows_per_s"])
+            line["extra"]["topp_rows_per_s"] = {n: round(float(np.exp(np.mean(np.log(v))))) for n, v in by_n.items()}
     if rank == 0 and not args.no_long_context:
         del step, pools
         torch.cuda.empty_cache()
-        line["extra"]["long_context"] = long_context(dev, n_layers=args.long_context_layers)
+        extra("long_context", lambda: long_context(dev, n_layers=args.long_context_layers))
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
