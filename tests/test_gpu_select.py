@@ -368,3 +368,30 @@ def test_threshold_bin_population_around_the_short_cut_capacity(n, n_bin):
         p = (0.4 + frac * bin_mass) / total
         st, gd, od = _run_rows(rows, n, float(p))
         assert st["n"] == 3
+
+
+@pytest.mark.parametrize("n", [65536, 131072])
+@pytest.mark.parametrize("family", wl.TOPP_FAMILIES)
+def test_config2_full_size_in_the_benchmarks_launch_shape(family, n, form):
+    """Config 2 as the benchmark launches it: 256 rows per call (which decides how many CTAs a row
+    gets), at the two largest row lengths.  The GPU selects all 256 rows; the oracle checks a
+    sample of them row by row, and every count against the mass invariant M_>= >= target."""
+    if form == "cluster":
+        pytest.skip("single-row lists take the same path with and without a workspace")
+    import paper_2510_27641_b200 as sa
+    rows = wl.topp_rows(family, 256, n, seed=2)
+    d = to_dev(rows.reshape(256, 1, 1, n))
+    kv = np.full(256, n, np.int32)
+    p = 0.9
+    gi, gc, gs, gd = sa.select_topp([d], to_dev(kv), [0], p, want_diag=True)
+    torch.cuda.synchronize()
+    gc_h, gs_h, gd_h = gc.cpu().numpy().ravel(), gs.cpu().numpy().ravel(), gd.cpu().numpy().reshape(256, 4)
+    assert np.all(gs_h == 0)
+    assert np.all(gd_h[:, 3] >= gd_h[:, 1]) and np.all(gd_h[:, 2] < gd_h[:, 1])   # M_>= >= target > M_>
+    sample = np.random.default_rng(n).choice(256, size=12, replace=False)
+    sub = rows[sample]
+    oi, oc, os_, od = oracle.select_topp([sub.reshape(12, 1, 1, n)], np.zeros(1, np.int32), kv[:12], p)
+    gi_h = gi.cpu().numpy()[0, sample]
+    st = compare_lists(lambda i: sub[i], p, gi_h[None], gc_h[sample].reshape(1, 12, 1), gs_h[sample].reshape(1, 12, 1),
+                       oi, oc, os_, od)
+    assert st["n"] == 12
