@@ -110,6 +110,7 @@ struct Shared {
   float warp_max[kWarps];   // largest aggregated value seen by each warp (literal bisection only)
   float cta_max;            // read by the other CTAs of the cluster
   int local_kept;           // read by the other CTAs of the cluster
+  int bin_lo, bin_hi;       // first and last non-empty level-1 bin of this CTA (read by the cluster)
   int n_cand;               // keys this CTA found in the level-1 threshold bin (read by the cluster)
   unsigned int cand[kCandCap];
   unsigned int red_key[2 * kWarps];
@@ -212,7 +213,7 @@ __device__ __forceinline__ double shfl_down_f64(double v, int d) { return __shfl
 // of a cluster gets bit-identical results.  Results land in sh.found_bin, sh.mass_above,
 // sh.mass_ge, sh.total.  Called by all threads.  An empty bin has mass exactly 0.
 __device__ void scan_bins(Shared& sh, const double* mass, int nbins, double carry_mass, double target,
-                          bool target_is_fraction, float p) {
+                          bool target_is_fraction, float p, int grp_lo = 0, int grp_hi = 1 << 20) {
   const int groups = nbins / kGroup;
   const int tid = threadIdx.x;
   const int lane = tid & 31;
@@ -222,7 +223,7 @@ __device__ void scan_bins(Shared& sh, const double* mass, int nbins, double carr
   {
     const int grp = tid >> 2, part = tid & 3;
     double s = 0.0;
-    if (grp < groups) {
+    if (grp < groups && grp >= grp_lo && grp < grp_hi) {  // groups outside the range are empty and unwritten
       const double* m8 = mass + grp * kGroup + part * 8;
 #pragma unroll
       for (int b = 7; b >= 0; --b) s += m8[b];
@@ -422,6 +423,8 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     }
     sh.n_rows = n;
     sh.n_cand = 0;
+    sh.bin_lo = kL1Bins;
+    sh.bin_hi = -1;
   }
   for (int i = tid; i < kL1Bins; i += kThreads) sh.h_hi[i] = sh.h_lo[i] = 0u;
   __syncthreads();
@@ -589,21 +592,65 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   }
   // the ring is idle from here on: zero this CTA's level-2 and level-3 histograms
   for (int i = tid; i < 2 * 2 * kL23Bins; i += kThreads) lvl_base[i] = 0u;
+  {
+    // first and last non-empty bin of the level-1 histogram (complete since the barrier above):
+    // rows of attention probabilities fill a few hundred of the 2048 bins, and the cluster
+    // reduction and the scan below then touch only those
+    int bmin = kL1Bins, bmax = -1;
+    for (int bin = tid; bin < kL1Bins; bin += kThreads) {
+      if ((sh.h_lo[bin] | sh.h_hi[bin]) != 0u) {
+        bmin = min(bmin, bin);
+        bmax = max(bmax, bin);
+      }
+    }
+    bmin = __reduce_min_sync(kFull, bmin);
+    bmax = __reduce_max_sync(kFull, bmax);
+    if (lane == 0 && bmax >= 0) {
+      atomicMin(&sh.bin_lo, bmin);
+      atomicMax(&sh.bin_hi, bmax);
+    }
+  }
   __syncthreads();
 
   // ---- 3: threshold search --------------------------------------------------------------------
   csync();  // every CTA's level-1 histogram and invalid count are complete
-  int n_bad = 0;
-  for (int r = 0; r < cs; ++r) n_bad += *cluster.map_shared_rank(&sh.n_invalid, r);
+  int n_bad = 0, glo = kL1Bins, ghi = -1;
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    if (r < cs) {
+      n_bad += *cluster.map_shared_rank(&sh.n_invalid, r);
+      glo = min(glo, *cluster.map_shared_rank(&sh.bin_lo, r));
+      ghi = max(ghi, *cluster.map_shared_rank(&sh.bin_hi, r));
+    }
+  }
+  // whole scan groups; an empty histogram gives an empty range
+  glo = (ghi < 0) ? 0 : (glo & ~(kGroup - 1));
+  ghi = (ghi < 0) ? 0 : ((ghi | (kGroup - 1)) + 1);
+  // one or two CTAs: every CTA sums the bins over the ranks itself (one cluster barrier and the
+  // gather less).  Larger clusters: each CTA reduces its own share of the bins and all gather the
+  // result (all-to-all reads of every histogram by eight CTAs cost more than that barrier).
+  const bool narrow = cs <= 2;
 
   theta_key = 0u;
   invalid = n_bad != 0;  // the count only grows from step to step: the last one decides
   bool searching = !invalid;
-  if (searching) {
+  if (searching && narrow) {
+    for (int bin = glo + tid; bin < ghi; bin += kThreads) {
+      unsigned long long mh = 0, ml = 0;
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        if (r < cs) {
+          mh += *cluster.map_shared_rank(&sh.h_hi[bin], r);
+          ml += *cluster.map_shared_rank(&sh.h_lo[bin], r);
+        }
+      }
+      r_mass[bin] = static_cast<double>((mh << 16) + ml) * pow2_double(max(bin >> 3, 1) - 150);
+    }
+  } else if (searching) {
     // level 1: every CTA reduces its own range of bins over the cluster, then all gather
     const int per_bins = kL1Bins / cs;
-    const int blo = rank * per_bins;
-    for (int bin = blo + tid; bin < blo + per_bins; bin += kThreads) {
+    const int blo = max(rank * per_bins, glo), bhi = min((rank + 1) * per_bins, ghi);
+    for (int bin = blo + tid; bin < bhi; bin += kThreads) {
       unsigned long long mh = 0, ml = 0;
       for (int r = 0; r < cs; ++r) {
         mh += *cluster.map_shared_rank(&sh.h_hi[bin], r);
@@ -612,15 +659,17 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       r_mass[bin] = static_cast<double>((mh << 16) + ml) * pow2_double(max(bin >> 3, 1) - 150);
     }
   }
-  csync();  // every owner's range is reduced
+  if (!narrow) csync();  // every owner's range is reduced
   if (searching) {
-    const int per_bins = kL1Bins / cs;
-    for (int bin = tid; bin < kL1Bins; bin += kThreads) {
-      const int owner = bin / per_bins;
-      if (owner != rank) r_mass[bin] = *cluster.map_shared_rank(&r_mass[bin], owner);
+    if (!narrow) {
+      const int per_bins = kL1Bins / cs;
+      for (int bin = glo + tid; bin < ghi; bin += kThreads) {
+        const int owner = bin / per_bins;
+        if (owner != rank) r_mass[bin] = *cluster.map_shared_rank(&r_mass[bin], owner);
+      }
     }
     __syncthreads();
-    scan_bins(sh, r_mass, kL1Bins, 0.0, 0.0, true, P.p);
+    scan_bins(sh, r_mass, kL1Bins, 0.0, 0.0, true, P.p, glo / kGroup, ghi / kGroup);
     total = sh.total;
     target = static_cast<double>(P.p) * total;
     m_ge = total;
