@@ -349,10 +349,12 @@ def test_both_forms_give_the_same_bits_and_flag_hidden_negative_inputs(form):
 
 
 @pytest.mark.parametrize("n", [1024, 4096, 40000])
-@pytest.mark.parametrize("n_bin", [1, 37, 512, 513])
+@pytest.mark.parametrize("n_bin", [1, 37, 128, 129, 512, 513])
 def test_threshold_bin_population_around_the_short_cut_capacity(n, n_bin):
     """The search takes a short cut when the level-1 threshold bin can hold at most 512 values
-    (it gathers them instead of refining with two more histogram levels).  Rows whose threshold
+    (it gathers them instead of refining with two more histogram levels over the row; up to 128
+    gathered values are searched directly, more through two histogram levels over the gathered
+    values).  Rows whose threshold
     bin holds exactly n_bin distinct values just above 2^-10 (so the bin's mantissa sum >> 23
     equals n_bin), for populations on both sides of that capacity, in a shared-memory slice
     (n = 1024), a row read in place by one CTA and one read by a cluster."""
