@@ -114,6 +114,7 @@ struct Shared {
   int bin_lo, bin_hi;       // first and last non-empty level-1 bin of this CTA (read by the cluster)
   int n_cand;               // keys this CTA found in the level-1 threshold bin (read by the cluster)
   unsigned int cand[kCandCap];
+  int cand_pos[kCandCap];   // (rows read in place) their positions inside the slice
   unsigned int all_keys[kCandCap];  // the keys of the whole cluster in that bin (short cut)
   unsigned int red_key[2 * kWarps];
   unsigned long long red_sum[2 * kWarps];
@@ -194,7 +195,7 @@ __device__ __forceinline__ void hist_add4(const Hist& h, const bool (&take)[4], 
 
 // Appends the keys of the taking lanes to the CTA's candidate list (all 32 lanes call this
 // together); slots beyond the capacity are counted but not stored.
-__device__ __forceinline__ void cand_add(Shared& sh, bool take, unsigned int key) {
+__device__ __forceinline__ void cand_add(Shared& sh, bool take, unsigned int key, int pos) {
   const unsigned takers = __ballot_sync(kFull, take);
   if (takers == 0) return;
   const int lane = threadIdx.x & 31;
@@ -203,7 +204,10 @@ __device__ __forceinline__ void cand_add(Shared& sh, bool take, unsigned int key
   if (lane == leader) base = atomicAdd(&sh.n_cand, __popc(takers));
   base = __shfl_sync(kFull, base, leader);
   const int slot = base + __popc(takers & ((1u << lane) - 1u));
-  if (take && slot < kCandCap) sh.cand[slot] = key;
+  if (take && slot < kCandCap) {
+    sh.cand[slot] = key;
+    sh.cand_pos[slot] = pos;
+  }
 }
 
 __device__ __forceinline__ double shfl_down_f64(double v, int d) { return __shfl_down_sync(kFull, v, d); }
@@ -407,6 +411,11 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   double total = 0.0, target = 0.0, m_gt = 0.0, m_ge = 0.0;
   bool invalid = false;
   if (tid == 0) sh.n_invalid = 0;
+  bool short_cut = false;  // the threshold was found among the gathered keys of the level-1 bin
+  // (in place) the kept positions as ballot words, four per 128 positions, in the upper half of
+  // the scan array: by the time they are written the level-1 scan is over, the later levels use
+  // the lower half only, and no peer reads this array after the level-1 gather
+  unsigned int* const keep_words = reinterpret_cast<unsigned int*>(r_mass + kL23Bins);
   for (int step = 0; step < n_steps; ++step) {
   // contributing rows in the order that defines the aggregated value
   if (tid == 0) {
@@ -682,7 +691,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   unsigned int prefix = searching ? static_cast<unsigned int>(sh.found_bin) : 0u;
   const int e1 = max(static_cast<int>(prefix >> 3), 1) - 150;
   double carry_m = searching ? sh.mass_above : 0.0;
-  bool short_cut = false;  // the threshold was found among the gathered keys of the level-1 bin
+  short_cut = false;
   // Short cut: the threshold bin of level 1 usually holds few values (tens to hundreds for
   // attention rows).  Its mantissa sum S bounds their number (a normal mantissa is >= 2^23); when
   // at most kCandCap fit, every CTA collects its keys of that bin, fetches everybody's, and
@@ -703,16 +712,26 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
 #pragma unroll
         for (int uu = 0; uu < kIpUnroll; ++uu) {
           const int i4 = base + uu * kThreads + tid;
+          // values in a higher bin are kept whatever the threshold turns out to be: their
+          // ballot words go where the count pass would put them, and once the threshold is
+          // known the candidates that made it are added -- the row is not read a third time
+          unsigned int mine = 0u;
 #pragma unroll
-          for (int e = 0; e < 4; ++e)
-            cand_add(sh, act[uu] && (4 * i4 + e < n_loc) && (key[uu][e] >> 20) == prefix, key[uu][e]);
+          for (int e = 0; e < 4; ++e) {
+            const bool in_row = act[uu] && (4 * i4 + e < n_loc);
+            cand_add(sh, in_row && (key[uu][e] >> 20) == prefix, key[uu][e], 4 * i4 + e);
+            const unsigned int m = __ballot_sync(kFull, in_row && (key[uu][e] >> 20) > prefix);
+            if (lane == e) mine = m;
+          }
+          const int g4 = base + uu * kThreads + (tid & ~31);  // first float4 of this warp's 32
+          if (lane < 4 && g4 < n4) keep_words[(g4 >> 5) * 4 + lane] = mine;
         }
       }
     } else {
       for (int base = 0; base < n_srch; base += kThreads) {
         const int i = base + tid;
         const unsigned int key = (i < n_srch) ? key_at(i) : 0u;
-        cand_add(sh, i < n_srch && (key >> 20) == prefix, key);
+        cand_add(sh, i < n_srch && (key >> 20) == prefix, key, i);
       }
     }
     csync();  // every CTA's candidate list is complete
@@ -821,6 +840,18 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     m_gt = sh.mass_above;
     m_ge = sh.mass_ge;
     }
+    if (in_place && !kVariant) {
+      // this CTA's candidates that reach the threshold join the positions recorded above
+      const int n_own = min(sh.n_cand, kCandCap);
+      __syncthreads();  // the ballot words of the candidate pass are complete
+      for (int i = tid; i < n_own; i += kThreads) {
+        if (sh.cand[i] >= theta_key) {
+          const int pos = sh.cand_pos[i];
+          atomicOr(&keep_words[(pos >> 7) * 4 + (pos & 3)], 1u << ((pos >> 2) & 31));
+        }
+      }
+      __syncthreads();
+    }
   } else
   for (int level = 0; level < 2; ++level) {
     const int shift = (level == 0) ? 10 : 0;
@@ -928,11 +959,14 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   const int wchunk4 = (((n4 + kWarps - 1) / kWarps) + 31) & ~31;
   const int w4_lo = min(n4, warp * wchunk4);
   const int w4_hi = min(n4, w4_lo + wchunk4);
-  // (in place) the kept positions as ballot words, four per 128 positions; the scan array is
-  // idle by now and no peer reads it after the level-1 gather
-  unsigned int* const keep_words = reinterpret_cast<unsigned int*>(r_mass);
   int wc = 0;
-  if (!invalid && in_place) {
+  if (!invalid && in_place && !kVariant && short_cut) {
+    // the kept positions are already in the ballot words: count this warp's
+    // (a warp whose range is empty has w4_lo == w4_hi == n4, not a multiple of 32)
+    if (w4_lo < w4_hi)
+      for (int w = (w4_lo >> 5) * 4 + lane; w < ((w4_hi + 31) >> 5) * 4; w += 32) wc += __popc(keep_words[w]);
+    wc = __reduce_add_sync(kFull, wc);
+  } else if (!invalid && in_place) {
     for (int i0 = w4_lo; i0 < w4_hi; i0 += 32 * kIpUnroll) {
       unsigned int key[kIpUnroll][4];
       bool act[kIpUnroll];
