@@ -140,8 +140,12 @@ def build_step(cfg, dev, verify_flags=0, select_workspace=True):
     from paper_2510_27641_b200.step import VerifyStep
     from workloads import bf16
     si = wl.make_step_inputs(cfg)
-    pools = [wl.kv_pool(cfg.seed, j, si.n_pages, cfg.page_size, cfg.n_kv_heads, cfg.head_dim, device=dev)
-             for j in range(cfg.n_target_layers)]
+    # one allocation for all layers' pools (each layer's pool is a slice of it), so that the
+    # layer-batched upper bound below can address every layer through one block table
+    per_layer = si.n_pages * 2 * cfg.page_size * cfg.n_kv_heads * cfg.head_dim
+    big = torch.empty(cfg.n_target_layers * per_layer, dtype=torch.bfloat16, device=dev)
+    pools = [wl.kv_pool(cfg.seed, j, si.n_pages, cfg.page_size, cfg.n_kv_heads, cfg.head_dim, device=dev,
+                        out=big[j * per_layer:(j + 1) * per_layer]) for j in range(cfg.n_target_layers)]
     step = VerifyStep(layer_map=si.layer_map.tolist(), n_draft_layers=cfg.n_draft_layers, batch=cfg.batch,
                       n_draft_heads=cfg.n_draft_heads, gamma=cfg.gamma, L_stride=si.L_stride,
                       n_q_heads=cfg.n_q_heads, p=cfg.p, kv_pools=pools,
@@ -151,6 +155,7 @@ def build_step(cfg, dev, verify_flags=0, select_workspace=True):
     dp_host = [None if x is None else torch.from_numpy(x).pin_memory() for x in si.draft_probs]
     q_host = [bf16.bits_to_torch(q).pin_memory() for q in si.q]
     step.load_inputs(dp_host, q_host)
+    step.kv_big = big.view(cfg.n_target_layers * si.n_pages, 2, cfg.page_size, cfg.n_kv_heads, cfg.head_dim)
     torch.cuda.synchronize()
     return si, pools, step, dp_host, q_host
 
@@ -413,6 +418,45 @@ def verify_micro(dev, reps=10, flags=0):
     return out
 
 
+def layer_batched(step, cfg, si, reps=20):
+    """Secondary number, an upper bound and not something a model can do: the attention of ALL
+    target layers in ONE launch, as if the layers did not depend on one another (layer j's
+    queries exist only after layer j - 1 has run).  Every (layer, sequence) becomes a sequence of
+    a batch of layers x batch: its lists are copied from its draft layer's, its block table
+    points into its layer's slice of the pool allocation.  It shows what the per-launch start-up
+    and merge of the per-layer launches cost."""
+    import torch
+    import paper_2510_27641_b200 as sa
+    m, B = step.n_layers, cfg.batch
+    if si.block_table is None or m * B * cfg.n_kv_heads > 2048 or any(u < 0 for u in step.layer_map):
+        return {"skipped": "needs a paged cache, sparse layers only and layers x batch x kv heads <= 2048"}
+    dev = step.kv_big.device
+    bt = torch.from_numpy(si.block_table).to(dev)
+    bt_all = torch.cat([bt + j * si.n_pages for j in range(m)]).contiguous()
+    idx_all = torch.cat([step.idx[u] for u in step.layer_map]).contiguous()          # [m B, G, stride]
+    cnt_all = torch.cat([step.counts[u] for u in step.layer_map]).contiguous()
+    kv_len_all = step.kv_len.repeat(m).contiguous()
+    q_all = torch.cat(step.q).contiguous()
+    out = torch.empty((m * B,) + tuple(step.out[0].shape[1:]), dtype=torch.float32, device=dev)
+    lse = torch.empty((m * B,) + tuple(step.lse[0].shape[1:]), dtype=torch.float32, device=dev)
+    a = sa.make_verify_args(q_all, step.kv_big, kv_len_all, block_table=bt_all, idx=idx_all, counts=cnt_all,
+                            out=out, lse=lse)
+    ws = sa.verify_workspace(a)
+    f = lambda: sa.sparse_verify(q_all, step.kv_big, kv_len_all, block_table=bt_all, idx=idx_all, counts=cnt_all,
+                                 out=out, lse=lse, workspace=ws)
+    f()
+    torch.cuda.synchronize()
+    close = max(float((out[j * B:(j + 1) * B] - step.out[j]).abs().max()) for j in range(m))
+    g, _ = capture(f)
+    us = time_replays(g, reps, 5)
+    kept = int(cnt_all.clamp(min=0).sum())
+    kv_bytes = kept * cfg.n_kv_heads * cfg.head_dim * 4
+    return {"us_all_layers_one_launch": round(us, 1), "kv_gbs": round(kv_bytes / us / 1e3),
+            "frac_of_measured": round(kv_bytes / us / 1e3 / _measured_peaks()[0], 3),
+            "max_abs_diff_vs_per_layer_launches": close,
+            "note": "upper bound: layers treated as independent; the per-layer launches are the result"}
+
+
 def long_context(dev, reps=10, n_layers=8):
     """Config 4 (batch 4, ctx 131072, 64 q / 8 kv heads, gamma 4, 4 draft layers of 16 heads) on
     `n_layers` target layers of the 80 (each has its own 2.1 GB K/V pool, so nothing is served
@@ -635,6 +679,7 @@ def main():
 
     if rank == 0:
         extra("select_variants", lambda: select_variants(step, cfg_r))
+        extra("layer_batched_upper_bound", lambda: layer_batched(step, cfg_r, si))
     if rank == 0 and not args.no_cpu_baseline:
         smp = OracleSample(cfg_r, si, n_attn_layers=8, pools=pools)
         us_cpu, sample = smp.step_us()
