@@ -226,7 +226,9 @@ class OracleSample:
         self.strides = wl.kv_strides(cfg.page_size, cfg.n_kv_heads, cfg.head_dim)
         sp, sk, ss, sh = self.strides
         oi, oc, _, _ = oracle.select_topp(si.draft_probs, si.layer_map, si.kv_len, cfg.p)
-        self.layers = list(range(cfg.n_target_layers))[:max(1, n_attn_layers)]
+        # evenly spread, first and last target layer included
+        n_take = max(1, min(n_attn_layers, cfg.n_target_layers))
+        self.layers = sorted({int(round(x)) for x in np.linspace(0, cfg.n_target_layers - 1, n_take)})
         self.prepared = []
         for j in self.layers:
             u = int(si.layer_map[j])
@@ -267,7 +269,8 @@ class OracleSample:
         t_attn = time.perf_counter() - t0
         scale = cfg.n_target_layers / len(self.layers)
         sample = (f"select: all {int((oc >= 0).sum())} lists of the step ({t_sel:.3f} s); attention: "
-                  f"{len(self.layers)} of {cfg.n_target_layers} target layers, all sequences and heads "
+                  f"{len(self.layers)} of {cfg.n_target_layers} target layers (evenly spread, first and last "
+                  f"included), all sequences and heads "
                   f"({t_attn:.3f} s), scaled x{scale:g}")
         return (t_sel + t_attn * scale) * 1e6, sample
 
