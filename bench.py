@@ -2,19 +2,24 @@
 """Benchmark of the SpecAttn verification hot path on B200.
 
 A step = one pass of the whole hot path over one synthetic batch: one specattn_select_topp over
-the mapped draft layers followed by one specattn_sparse_verify per target layer (33 launches on
-the default workload).  Default workload: the Llama-3-8B-shaped configuration -- 32 target
+the mapped draft layers, one launch for the work partitions (plans) of the list sets, and one
+specattn_sparse_verify per target layer (34 launches on the default workload).  Default workload: the Llama-3-8B-shaped configuration -- 32 target
 layers, 4-layer 12-head draft, batch 8, context 32768, paged bf16 KV (page 16, shuffled block
 table), gamma = 5, p = 0.95.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--topp-sweep]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--no-topp-sweep] [--no-long-context] [--no-cpu-baseline]
 
 Prints ONE JSON line (rank 0).  `value` is microseconds per step with all inputs resident in
 HBM (CUDA-graph replay of the step, CUDA events, max over ranks); `e2e` is the same step issued
 through specattn_verify_step_host from pinned host buffers (draft probabilities and queries go
 host->device, outputs and LSE come back, inside the timed region); `roofline` describes the
 dominant kernel (sparse verify) against the measured HBM copy bandwidth; `cpu_baseline` is the
-CPU oracle timed on a bounded sample of the same workload and scaled to a step.
+CPU oracle timed on a bounded sample of the same workload and scaled to a step.  `extra` adds
+context measured in the same run: the selection variants of Alg. 2, the attention of all layers
+in one launch (an upper bound, labelled so), the selection micro-benchmark of config 2
+(256 rows x {1k, 8k, 64k, 128k} x 3 p x 3 families, rows/s) and config 4 (ctx 131072, 64 q / 8 kv
+heads: p in {0.8, 0.9, 0.95} against the same kernel at p = 1).
 With N > 1 every rank runs its own batch of 8 sequences (batch sharding, no collective).
 `--impl reference` times the CPU oracle alone (rank 0) and prints the same line.
 """
@@ -40,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per sparse_verify launch on this workload, from
 # the ncu capture summarised in profiles/sparse_verify_cfg1.md.
-NCU_VERIFY_TRAFFIC_BYTES = 40.85e6
+NCU_VERIFY_TRAFFIC_BYTES = 40.9e6
 
 
 # ----------------------------------------------------------------------------------------------
