@@ -378,9 +378,11 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     return in_place ? __float_as_uint(__ldg(A + i) + 0.f) : __float_as_uint(a[i]);
   };
   const int n4 = (n_loc + 3) >> 2;
-  // In-place passes read the row from global memory (L2) with eight independent 16-byte loads per
-  // thread in flight: with one dependent load per iteration a CTA moved ~4 GB/s (latency-bound).
-  constexpr int kIpUnroll = 8;
+  // In-place passes read the row from global memory (L2) with four independent 16-byte loads per
+  // thread in flight: with one dependent load per iteration a CTA moved ~4 GB/s (latency-bound);
+  // eight in flight were 3-4 % slower on 64k / 128k rows than four (twice the code per pass), two
+  // 3 % slower again.
+  constexpr int kIpUnroll = 4;
   auto load_keys4 = [&](int i4, unsigned int (&key)[4]) -> bool {  // keys of positions 4*i4 .. 4*i4+3
     const bool act = i4 < n4;
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
