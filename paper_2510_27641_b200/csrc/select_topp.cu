@@ -131,6 +131,10 @@ struct Shared {
 //   [16, 24 KB)  level-2 histogram of this CTA (low and high words)
 //   [24, 32 KB)  level-3 histogram of this CTA
 constexpr int kRingFloats = kDepth * kChunk;
+// a list read in place needs the fixed part and 32 KB of scan arrays: four such CTAs (plus 1 KB
+// each that the system reserves) must fit the 227 KB of an SM
+static_assert(4 * (((sizeof(Shared) + 127) / 128) * 128 + 32 * 1024 + 1024) <= 227 * 1024,
+              "four in-place CTAs per SM");
 static_assert(kRingFloats * 4 >= 32 * 1024, "the ring must hold the scan arrays");
 
 __device__ __forceinline__ double pow2_double(int k) {  // 2^k, k in the normal range
