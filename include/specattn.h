@@ -218,6 +218,13 @@ size_t specattn_select_workspace_bytes(const specattn_select_args* args);
 #define SPECATTN_VERIFY_LISTS_STABLE 1u
 #define SPECATTN_VERIFY_ENGINE_MMA_SYNC 2u
 #define SPECATTN_VERIFY_ENGINE_TCGEN05 4u
+/* TEST ONLY -- never set this in production.  Exercises the failure path of the kernels' bounded
+ * device-side waits without faulting anything: one producer warp of CTA 0 withholds the
+ * completion signal of its first tile, the waits on it give up after their poll limit (about
+ * half a second each), the CTA raises SPECATTN_ROW_TIMEOUT in status[0] and the kernel returns
+ * normally.  Outputs of that call are invalid and the workspace must be re-initialised with
+ * specattn_verify_workspace_init before its next use. */
+#define SPECATTN_VERIFY_TEST_LOSE_ARRIVAL 0x80000000u
 
 typedef struct specattn_verify_args {
   uint32_t struct_size;
@@ -271,7 +278,12 @@ int specattn_sparse_verify(const specattn_verify_args* args, void* cuda_stream);
  * 16-byte aligned, written by a small kernel on the stream (after whatever produces counts /
  * kv_len, e.g. specattn_select_topp) and valid until those change.  A kernel given a plan that
  * does not fit its launch (other batch, heads, tail_len, dense flag or GPU) ignores it.  Only
- * the mma.sync engine reads plans. */
+ * the mma.sync engine reads plans.
+ * Ordering: a plan must be at least as new as the lists it describes -- call this after every
+ * specattn_select_topp that rewrites counts -- and a verify call flagged
+ * SPECATTN_VERIFY_LISTS_STABLE must not be the first launch after the plan kernel (that flag's
+ * "two launches earlier" rule covers the plan like the lists): the plan kernel signals completion
+ * only when it has finished, and the first verify call after it waits for that. */
 size_t specattn_verify_plan_bytes(const specattn_verify_args* args);
 int specattn_verify_plan(const specattn_verify_args* args, void* plan, size_t plan_bytes, void* cuda_stream);
 /* The same for n launches at once (HOST arrays of n argument structs, plan buffers and their
@@ -306,7 +318,12 @@ int specattn_verify_plan_many(const specattn_verify_args* const* args, void* con
  *   - all calls on a device share the one array, which still holds what the previous call left
  *     there: the arrival counters are cleared on the stream at the start of every call, and
  *     two calls that may overlap on the GPU (different streams, or concurrent graph branches)
- *     race on it -- serialise them or use specattn_sparse_verify with separate workspaces.
+ *     race on it -- serialise them or use specattn_sparse_verify with separate workspaces;
+ *   - the clearing is a memset in front of the launch, so a call flagged
+ *     SPECATTN_VERIFY_LISTS_STABLE gains nothing here: the kernel cannot begin under its
+ *     predecessor as it does after specattn_sparse_verify, it starts when the memset is done;
+ *   - every argument check happens before the memset is enqueued: a negative return code means
+ *     that nothing at all was enqueued.
  * ======================================================================================== */
 #define SPECATTN_STATIC_SCRATCH_BYTES (6u << 20)
 

@@ -197,10 +197,15 @@ extern "C" int specattn_verify_step_host(const specattn_step_host_args* args, vo
   bool selected[SPECATTN_MAX_DRAFT_LAYERS] = {false};
   const void* planned[SPECATTN_MAX_DRAFT_LAYERS + 1];
   int n_planned = 0;
+  // A verify launch may skip its wait for the preceding kernel (SPECATTN_VERIFY_LISTS_STABLE)
+  // only when that kernel is another verify launch: the first one after a selection or a plan
+  // launch enqueued here reads what those kernels wrote, so the flag is dropped for it.
+  bool fresh = true;
   for (int j = 0; j < S.n_target_layers; ++j) {
     const int u = sel.layer_map[j];
     if (u >= 0 && !selected[u]) {
       selected[u] = true;
+      fresh = true;
       if (!ok(cudaStreamWaitEvent(stream, pipe.layer_in[u], 0))) return SPECATTN_ERR_CUDA;
       specattn_select_args one = sel;  // the lists of draft layer u only
       const int32_t only = u;
@@ -218,9 +223,13 @@ extern "C" int specattn_verify_step_host(const specattn_step_host_args* args, vo
         const int prc = specattn_verify_plan(&v, const_cast<void*>(v.plan), specattn_verify_plan_bytes(&v), cuda_stream);
         if (prc != SPECATTN_OK) return prc;
         if (n_planned < SPECATTN_MAX_DRAFT_LAYERS + 1) planned[n_planned++] = v.plan;
+        fresh = true;
       }
     }
-    const int rc = specattn_sparse_verify(&v, cuda_stream);
+    specattn_verify_args call = v;
+    if (fresh) call.flags &= ~SPECATTN_VERIFY_LISTS_STABLE;
+    fresh = false;
+    const int rc = specattn_sparse_verify(&call, cuda_stream);
     if (rc != SPECATTN_OK) return rc;
     // lane "out"
     const size_t rows = static_cast<size_t>(v.batch) * v.n_q * v.n_q_heads;

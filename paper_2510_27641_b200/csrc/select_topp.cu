@@ -685,6 +685,11 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
         if (owner != rank) r_mass[bin] = *cluster.map_shared_rank(&r_mass[bin], owner);
       }
     }
+  }
+  // (rows read in place) the ballot words of the kept positions overlay the upper half of this
+  // array from the candidate pass on: no CTA may get there while a peer still gathers from it
+  if (kInPlace && !narrow) csync();
+  if (searching) {
     __syncthreads();
     scan_bins(sh, r_mass, kL1Bins, 0.0, 0.0, true, P.p, glo / kGroup, ghi / kGroup);
     total = sh.total;
@@ -708,6 +713,8 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     const unsigned long long S = static_cast<unsigned long long>(r_mass[prefix] * pow2_double(-e1));
     short_cut = (S >> 23) <= static_cast<unsigned long long>(kCandCap);
   }
+  // every thread has read the bin's mass before a faster warp's ballot words can land on it
+  if (kInPlace) __syncthreads();
   if (short_cut) {
     if (in_place) {
       for (int base = 0; base < n4; base += kIpUnroll * kThreads) {

@@ -81,6 +81,7 @@ struct VerifyParams {
   int tail;          // in-flight tokens appended to every unit, attended causally
   int tail_off;      // tail - T: query t may see tail tokens j <= t + tail_off
   const int* plan;   // precomputed work partition (specattn_verify_plan) or nullptr
+  int test_lose;     // SPECATTN_VERIFY_TEST_LOSE_ARRIVAL: CTA 0 withholds one barrier arrival
 };
 
 // WPM = consumer warps per 16-row slab: 4 -> (stage parity, 32-key half), 2 -> (stage parity).
@@ -156,8 +157,10 @@ __device__ __forceinline__ void plan_body(const VerifyParams& P, int* plan, int 
   __shared__ int cand_parts[kCandidates], cand_max[kCandidates];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int U = P.B * P.Hkv;
-  pdl_wait();              // the lists are the previous kernel's output
-  pdl_launch_dependents();
+  // The lists are the previous kernel's output.  No early trigger for the next kernel either:
+  // a verify launch flagged SPECATTN_VERIFY_LISTS_STABLE reads the plan without waiting, so it
+  // must not be scheduled before this grid has completed (completion is the trigger).
+  pdl_wait();
   int* const p_us = plan + kPlanHeader;
   int* const p_cnt = p_us + (U + 1);
   int* const p_ps = p_cnt + U;
@@ -681,7 +684,10 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           const int k = t0 + jt;  // token index inside the unit: the list first, then the tail
           int pos = (k >= c_list) ? (kvlen_b + (k - c_list)) : (P.dense ? k : __ldg(list + k));
           if (pos < 0 || pos >= kvlen_b + P.tail) { bad = true; pos = 0; }
-          const int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
+          int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
+          // a position beyond the sequence's row of the block table (kv_len larger than the
+          // table covers) is a bad index like any other: it reads position 0 instead
+          if (lp >= P.bt_stride) { bad = true; pos = 0; lp = 0; }
           const int slot = pos - lp * P.page_size;
           long long page = P.bt ? static_cast<long long>(__ldg(P.bt + b * P.bt_stride + lp))
                                 : (b * P.bt_stride + lp);
@@ -729,7 +735,8 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
             }
           }
         }
-        cp_async_mbar_arrive_noinc(&sh.full[s]);
+        // (test hook: the first tile of CTA 0 never completes, so the bounded waits run out)
+        if (!(P.test_lose && blockIdx.x == 0 && it == 0)) cp_async_mbar_arrive_noinc(&sh.full[s]);
         if (q_pending) {
           q_pending = false;
           if (!load_q()) { sh.abort_flag = 1; dead = true; break; }
@@ -1107,6 +1114,19 @@ using specattn::VerifyParams;
 
 namespace specattn {
 namespace {
+// Pointer, alignment and stride rules of a call that will launch (everything except the
+// workspace); shared by the entry points so that each of them checks before it enqueues anything.
+int check_buffers(const specattn_verify_args& A) {
+  if (!A.q || !A.kv_pages || !A.kv_len || !A.out || !A.lse) return SPECATTN_ERR_NULL;
+  if (!A.dense && (!A.idx || !A.counts)) return SPECATTN_ERR_NULL;
+  if (!A.dense && A.idx_stride < 0) return SPECATTN_ERR_RANGE;
+  if (A.block_table_stride < 0 || A.n_pages < 0) return SPECATTN_ERR_RANGE;
+  auto mis = [](const void* p, uintptr_t a) { return reinterpret_cast<uintptr_t>(p) % a != 0; };
+  if (mis(A.q, 16) || mis(A.kv_pages, 16) || mis(A.out, 16)) return SPECATTN_ERR_ALIGN;
+  if (A.stride_page % 8 || A.stride_kv % 8 || A.stride_slot % 8 || A.stride_head % 8) return SPECATTN_ERR_ALIGN;
+  return SPECATTN_OK;
+}
+
 // The kernel-side view of the arguments (everything except the workspace).
 VerifyParams make_params(const specattn_verify_args& A) {
   VerifyParams P;
@@ -1146,6 +1166,7 @@ VerifyParams make_params(const specattn_verify_args& A) {
   P.tail_off = A.tail_len - A.n_q;
 
   P.plan = static_cast<const int*>(A.plan);
+  P.test_lose = (A.flags & SPECATTN_VERIFY_TEST_LOSE_ARRIVAL) ? 1 : 0;
   return P;
 }
 }  // namespace
@@ -1175,13 +1196,10 @@ extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cu
   if (v != SPECATTN_OK) return v;
   const specattn_verify_args& A = *args;
   if (A.batch == 0) return SPECATTN_OK;
-  if (!A.q || !A.kv_pages || !A.kv_len || !A.out || !A.lse || !A.workspace) return SPECATTN_ERR_NULL;
-  if (!A.dense && (!A.idx || !A.counts)) return SPECATTN_ERR_NULL;
-  if (!A.dense && A.idx_stride < 0) return SPECATTN_ERR_RANGE;
-  if (A.block_table_stride < 0 || A.n_pages < 0) return SPECATTN_ERR_RANGE;
-  auto mis = [](const void* p, uintptr_t a) { return reinterpret_cast<uintptr_t>(p) % a != 0; };
-  if (mis(A.q, 16) || mis(A.kv_pages, 16) || mis(A.out, 16) || mis(A.workspace, 256)) return SPECATTN_ERR_ALIGN;
-  if (A.stride_page % 8 || A.stride_kv % 8 || A.stride_slot % 8 || A.stride_head % 8) return SPECATTN_ERR_ALIGN;
+  const int pc = specattn::check_buffers(A);
+  if (pc != SPECATTN_OK) return pc;
+  if (!A.workspace) return SPECATTN_ERR_NULL;
+  if (reinterpret_cast<uintptr_t>(A.workspace) % 256 != 0) return SPECATTN_ERR_ALIGN;
   const int n_ctas = specattn::device_sm_count();
   if (n_ctas <= 0) return SPECATTN_ERR_CUDA;
   if (A.workspace_bytes < specattn::workspace_bytes_for(A, n_ctas)) return SPECATTN_ERR_WORKSPACE;
@@ -1310,30 +1328,33 @@ extern "C" int specattn_sparse_verify_static(const specattn_verify_args* args, v
   const int v = specattn::validate(args);
   if (v != SPECATTN_OK) return v;
   if (args->batch == 0) return SPECATTN_OK;
+  // every argument check comes before the first thing that is enqueued
+  const int pc = specattn::check_buffers(*args);
+  if (pc != SPECATTN_OK) return pc;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
     cudaGetLastError();
     return SPECATTN_ERR_CUDA;
   }
+  const int n_ctas = specattn::device_sm_count();
+  if (n_ctas <= 0) return SPECATTN_ERR_CUDA;
+  if (specattn::workspace_bytes_for(*args, n_ctas) > SPECATTN_STATIC_SCRATCH_BYTES)
+    return SPECATTN_ERR_STATIC_SCRATCH;
   // In host code the array's name is only a handle; the kernel needs its device address,
-  // looked up once per device with that device current.
-  static void* device_addr[64] = {nullptr};
-  static std::atomic<unsigned long long> looked_up{0};
-  if (!((looked_up.load(std::memory_order_acquire) >> dev) & 1ull)) {
+  // looked up once per device with that device current (racing first callers store the same
+  // value).
+  static std::atomic<void*> device_addr[64];
+  void* scratch = device_addr[dev].load(std::memory_order_acquire);
+  if (scratch == nullptr) {
     void* p = nullptr;
     const cudaError_t e = cudaGetSymbolAddress(&p, specattn::g_static_scratch);
     if (e != cudaSuccess || p == nullptr) {
       cudaGetLastError();
       return SPECATTN_ERR_CUDA;
     }
-    device_addr[dev] = p;
-    looked_up.fetch_or(1ull << dev, std::memory_order_release);
+    device_addr[dev].store(p, std::memory_order_release);
+    scratch = p;
   }
-  void* scratch = device_addr[dev];
-  const int n_ctas = specattn::device_sm_count();
-  if (n_ctas <= 0) return SPECATTN_ERR_CUDA;
-  if (specattn::workspace_bytes_for(*args, n_ctas) > SPECATTN_STATIC_SCRATCH_BYTES)
-    return SPECATTN_ERR_STATIC_SCRATCH;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   // the array keeps the previous call's contents: the arrival counters must start at zero
   if (cudaMemsetAsync(scratch, 0, specattn::kCounterBytes, stream) != cudaSuccess) {

@@ -424,7 +424,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           const int k = h0 + jt;  // token index inside the unit: the list first, then the tail
           int pos = (k >= c_list) ? (kvlen_b + (k - c_list)) : (P.dense ? k : __ldg(list + k));
           if (pos < 0 || pos >= kvlen_b + P.tail) { bad = true; pos = 0; }
-          const int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
+          int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
+          // a position beyond the sequence's row of the block table (kv_len larger than the
+          // table covers) is a bad index like any other: it reads position 0 instead
+          if (lp >= P.bt_stride) { bad = true; pos = 0; lp = 0; }
           const int slot = pos - lp * P.page_size;
           long long page = P.bt ? static_cast<long long>(__ldg(P.bt + b * P.bt_stride + lp))
                                 : (b * P.bt_stride + lp);
@@ -475,7 +478,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         asm volatile("cp.async.wait_all;" ::: "memory");
         fence_proxy_async();  // generic-proxy writes -> visible to the tensor core's reads
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.full[s]);
+        // (test hook: the first tile of CTA 0 never completes, so the bounded waits run out)
+        if (lane == 0 && !(P.test_lose && blockIdx.x == 0 && it == 0 && half == 0)) mbar_arrive(&sh.full[s]);
         if (bad && P.status) atomicOr(P.status + b, SPECATTN_ROW_BAD_INDEX);
         if (q_pending) {
           q_pending = false;

@@ -372,28 +372,98 @@ def test_threshold_bin_population_around_the_short_cut_capacity(n, n_bin):
         assert st["n"] == 3
 
 
-@pytest.mark.parametrize("n", [65536, 131072])
+@pytest.mark.parametrize("n", wl.TOPP_SIZES)
 @pytest.mark.parametrize("family", wl.TOPP_FAMILIES)
 def test_config2_full_size_in_the_benchmarks_launch_shape(family, n, form):
     """Config 2 as the benchmark launches it: 256 rows per call (which decides how many CTAs a row
-    gets), at the two largest row lengths.  The GPU selects all 256 rows; the oracle checks a
-    sample of them row by row, and every count against the mass invariant M_>= >= target."""
+    gets), every row length and every p of the configuration.  The GPU selects all 256 rows; the
+    oracle checks a sample of them row by row, and every row against the mass invariant
+    M_> < target <= M_>=."""
     if form == "cluster":
         pytest.skip("single-row lists take the same path with and without a workspace")
     import paper_2510_27641_b200 as sa
     rows = wl.topp_rows(family, 256, n, seed=2)
     d = to_dev(rows.reshape(256, 1, 1, n))
     kv = np.full(256, n, np.int32)
-    p = 0.9
-    gi, gc, gs, gd = sa.select_topp([d], to_dev(kv), [0], p, want_diag=True)
-    torch.cuda.synchronize()
-    gc_h, gs_h, gd_h = gc.cpu().numpy().ravel(), gs.cpu().numpy().ravel(), gd.cpu().numpy().reshape(256, 4)
-    assert np.all(gs_h == 0)
-    assert np.all(gd_h[:, 3] >= gd_h[:, 1]) and np.all(gd_h[:, 2] < gd_h[:, 1])   # M_>= >= target > M_>
     sample = np.random.default_rng(n).choice(256, size=12, replace=False)
     sub = rows[sample]
-    oi, oc, os_, od = oracle.select_topp([sub.reshape(12, 1, 1, n)], np.zeros(1, np.int32), kv[:12], p)
-    gi_h = gi.cpu().numpy()[0, sample]
-    st = compare_lists(lambda i: sub[i], p, gi_h[None], gc_h[sample].reshape(1, 12, 1), gs_h[sample].reshape(1, 12, 1),
-                       oi, oc, os_, od)
-    assert st["n"] == 12
+    for p in wl.TOPP_PS:
+        gi, gc, gs, gd = sa.select_topp.func([d], to_dev(kv), [0], p, want_diag=True)
+        torch.cuda.synchronize()
+        gc_h, gs_h, gd_h = gc.cpu().numpy().ravel(), gs.cpu().numpy().ravel(), gd.cpu().numpy().reshape(256, 4)
+        assert np.all(gs_h == 0)
+        assert np.all(gd_h[:, 3] >= gd_h[:, 1]) and np.all(gd_h[:, 2] < gd_h[:, 1])   # M_>= >= target > M_>
+        oi, oc, os_, od = oracle.select_topp([sub.reshape(12, 1, 1, n)], np.zeros(1, np.int32), kv[:12], p)
+        gi_h = gi.cpu().numpy()[0, sample]
+        st = compare_lists(lambda i: sub[i], p, gi_h[None], gc_h[sample].reshape(1, 12, 1),
+                           gs_h[sample].reshape(1, 12, 1), oi, oc, os_, od)
+        assert st["n"] == 12
+
+
+FMAX = float(np.finfo(np.float32).max)
+
+
+@pytest.mark.parametrize("variant", ["exact", "per_step", "chunk"])
+def test_sum_overflow_voids_the_list_like_the_oracle(variant):
+    """Finite inputs whose binary32 sum leaves the format: the list is invalid, as in the oracle;
+    a sum that lands exactly on the largest finite value is valid.  Multi-row lists (both forms
+    of the call through the fixture), and the same rule for chunk scores."""
+    import paper_2510_27641_b200 as sa
+    B, H, gamma, Ls = 4, 2, 2, 4096
+    rng = np.random.default_rng(5)
+    probs = (rng.random((B, H, gamma, Ls), dtype=np.float32) * 1e-3).astype(np.float32)
+    probs[0, :, :, 100] = [[3e38, 0.0], [3e38, 0.0]]        # heads sum to +inf (also per query)
+    probs[1, :, :, 200] = [[FMAX, 0.0], [0.0, 0.0]]         # exactly FLT_MAX: valid
+    probs[2, :, :, 300] = [[3e38, 3e38], [0.0, 0.0]]        # overflows across queries only
+    probs[3, :, :, 64:68] = 1e38 * 0.6                      # each position finite, a 4-chunk of them not
+    kv = np.array([Ls, Ls, 3000, Ls], np.int32)
+    kw = dict(per_step=variant == "per_step", chunk=4 if variant == "chunk" else 1)
+    gi, gc, gs, _ = sa.select_topp([to_dev(probs)], to_dev(kv), [0], 0.9, **kw)
+    torch.cuda.synchronize()
+    if variant == "exact":
+        oi, oc, os_, od = oracle.select_topp([probs], [0], kv, 0.9)
+    else:
+        oi, oc, os_, od = oracle.select_variant([probs], [0], kv, 0.9, **kw)
+    assert gs.cpu().numpy().ravel().tolist() == os_.ravel().tolist()
+    assert gc.cpu().numpy().ravel().tolist() == oc.ravel().tolist()
+    bad, ok = sa.ROW_INVALID_PROB, 0
+    expect = {"exact": [bad, ok, bad, ok], "per_step": [bad, ok, ok, ok], "chunk": [bad, ok, bad, bad]}[variant]
+    assert os_.ravel().tolist() == expect
+    for b in range(B):
+        c = int(oc[0, b, 0])
+        assert np.array_equal(gi.cpu().numpy()[0, b, 0, :c], oi[0, b, 0, :c])
+
+
+def test_single_rows_at_the_edge_of_binary32():
+    """R = 1 (a row read in place from 2048 positions on, and the shared-memory path below that):
+    FLT_MAX is a valid value, +inf is not."""
+    for n in (1024, 4096):
+        rows = np.full((3, n), 1e-3, np.float32)
+        rows[0, 17] = FMAX
+        rows[1, 17] = np.inf
+        rows[2, 17] = FMAX
+        rows[2, 18] = FMAX          # the row total exceeds binary32 but not the binary64 masses
+        st, gd, od = _run_rows(rows, n, 0.9)
+        assert st["n"] == 3
+
+
+def test_few_lists_wide_clusters_thresholds_above_two():
+    """The two-launch form on very few lists (the search then runs eight CTAs per list) with
+    aggregated values of 2.0 and more around the threshold -- level-1 bins in the upper half of
+    the histogram -- for bins that take the short cut (few values per bin) and bins that do not."""
+    import paper_2510_27641_b200 as sa
+    B, H, gamma, Ls = 2, 16, 4, 32768
+    rng = np.random.default_rng(9)
+    kv = np.array([Ls, 30001], np.int32)
+    flat = rng.random((B, H, gamma, Ls), dtype=np.float32)                       # sums ~ 32
+    spread = np.exp(3.0 * rng.standard_normal((B, H, gamma, Ls))).astype(np.float32)  # sums spread over octaves
+    for probs in (flat, spread):
+        for p in (0.3, 0.9):
+            gi, gc, gs, gd = sa.select_topp([to_dev(probs)], to_dev(kv), [0], p, want_diag=True)
+            torch.cuda.synchronize()
+            oi, oc, os_, od = oracle.select_topp([probs], [0], kv, p)
+            theta = od[0, :, 0, 5]
+            assert np.all(theta >= 2.0)
+            st = compare_lists(lambda i: oracle.aggregate(probs[i], L=int(kv[i]))[0], p, gi.cpu().numpy(),
+                               gc.cpu().numpy(), gs.cpu().numpy(), oi, oc, os_, od)
+            assert st["n"] == B

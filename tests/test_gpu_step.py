@@ -12,9 +12,17 @@ from workloads import bf16
 pytestmark = pytest.mark.gpu
 
 
-def _build(cfg, n_groups=1, head_group=None, dense_first=0):
+def _build(cfg, n_groups=1, head_group=None, dense_first=0, layer_map=None):
     from paper_2510_27641_b200.step import VerifyStep
     si = wl.make_step_inputs(cfg)
+    if layer_map is not None:
+        # a chosen map (e.g. one target layer per draft layer): the draft rows of a layer depend
+        # only on (seed, draft layer), so they are the full configuration's
+        si.layer_map = np.asarray(layer_map, np.int32)
+        sink, slope = (8.0, 0.002)
+        assert not cfg.ragged
+        si.draft_probs = [wl.draft_probs(cfg.seed, u, si.kv_len, cfg.n_draft_heads, cfg.gamma, si.L_stride, sink, slope)
+                          if u in set(si.layer_map.tolist()) else None for u in range(cfg.n_draft_layers)]
     if dense_first:
         si.layer_map[:dense_first] = -1
     pools = [wl.kv_pool(cfg.seed, j, si.n_pages, cfg.page_size, cfg.n_kv_heads, cfg.head_dim, device=dev())
@@ -166,18 +174,57 @@ def test_host_buffer_step_matches_device_resident_step():
         assert torch.equal(out_host[j], ref_out[j].cpu()) and torch.equal(lse_host[j], ref_lse[j].cpu())
 
 
-@pytest.mark.parametrize("which", ["cfg1", "cfg3", "cfg4"])
+def test_host_buffer_steps_with_changing_inputs_match_the_oracle():
+    """Two steps from host buffers whose draft rows differ (so the lists, their lengths and the
+    work partitions change between the steps): each step must match the oracle on its own
+    inputs -- a launch that read the previous step's partition or lists would not."""
+    cfg = wl.config1().scaled(n_target_layers=6, n_draft_layers=3, batch=3, ctx=5000)
+    si, pools, step = _build(cfg, layer_map=[0, 0, 1, 1, 2, 2])
+    sp = wl.kv_strides(cfg.page_size, cfg.n_kv_heads, cfg.head_dim)
+    q_host = [bf16.bits_to_torch(q).pin_memory() for q in si.q]
+    out_host = [torch.zeros(o.shape, dtype=torch.float32).pin_memory() for o in step.out]
+    lse_host = [torch.zeros(l.shape, dtype=torch.float32).pin_memory() for l in step.lse]
+    kv_bits = [bf16.torch_to_bits(pl.cpu()) for pl in pools]
+    prev_counts = None
+    for k, (p_sink, p_slope) in enumerate([(8.0, 0.002), (2.0, 0.0004), (8.0, 0.002)]):
+        probs = [wl.draft_probs(cfg.seed + 17 * k, u, si.kv_len, cfg.n_draft_heads, cfg.gamma, si.L_stride,
+                                p_sink, p_slope) for u in range(3)]
+        dp_host = [torch.from_numpy(x).pin_memory() for x in probs]
+        step.run_host(dp_host, q_host, out_host, lse_host)
+        torch.cuda.synchronize()
+        oi, oc, os_, od = oracle.select_topp(probs, si.layer_map, si.kv_len, cfg.p)
+        st = compare_lists(lambda i: oracle.aggregate(probs[i // 3][i % 3], L=int(si.kv_len[i % 3]))[0], cfg.p,
+                           step.idx.cpu().numpy(), step.counts.cpu().numpy(), step.row_status.cpu().numpy(),
+                           oi, oc, os_, od)
+        assert st["n"] == 9
+        if prev_counts is not None:
+            assert not np.array_equal(prev_counts, oc)     # the partitions really changed
+        prev_counts = oc.copy()
+        for j in range(6):
+            u = int(si.layer_map[j])
+            ro, rl = oracle.sparse_verify(si.q[j], kv_bits[j], sp, si.block_table, si.kv_len,
+                                          step.idx[u].cpu().numpy(), step.counts[u].cpu().numpy(),
+                                          n_kv_heads=cfg.n_kv_heads, page_size=cfg.page_size, n_groups=1, dense=False,
+                                          pages_per_seq=si.pages_per_seq)
+            check_attention(out_host[j], lse_host[j], ro, rl)
+        assert int(step.status.abs().sum()) == 0
+
+
+@pytest.mark.parametrize("which", ["cfg1", "cfg3", "cfg4_p0.8", "cfg4_p0.9", "cfg4_p0.95"])
 def test_full_size_sampled_outputs(which):
-    """Full batch / context of configs 1, 3 and 4 (two target layers for 1 and 4): every list is
-    compared; attention is checked on sampled (layer, sequence, kv head) units whose K/V rows
-    are regenerated on the CPU from the hashed pool definition."""
+    """Full batch / context of configs 1, 3 and 4: every list is compared (config 1: the lists
+    of all four draft layers, one target layer mapped to each; config 4: two target layers at
+    each p of the configuration); attention is checked on sampled (layer, sequence, kv head)
+    units whose K/V rows are regenerated on the CPU from the hashed pool definition."""
+    lmap = None
     if which == "cfg1":
-        cfg = wl.config1().scaled(n_target_layers=2)
+        cfg = wl.config1().scaled(n_target_layers=4)
+        lmap = [0, 1, 2, 3]
     elif which == "cfg3":
         cfg = wl.config3()
     else:
-        cfg = wl.config4(n_target_layers=2, p=0.9)   # 70B-shaped: 64 q / 8 kv heads, ctx 131072
-    si, pools, step = _build(cfg)
+        cfg = wl.config4(n_target_layers=2, p=float(which.split("_p")[1]))   # 70B-shaped, ctx 131072
+    si, pools, step = _build(cfg, layer_map=lmap)
     step.run()
     torch.cuda.synchronize()
     oi, oc, os_, od = oracle.select_topp(si.draft_probs, si.layer_map, si.kv_len, cfg.p)

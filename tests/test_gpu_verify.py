@@ -301,3 +301,67 @@ def test_precomputed_work_partition_gives_the_same_results_and_is_ignored_when_i
         sa.verify_plan_many([a0], [small])
     assert sa.lib().specattn_verify_plan(C.byref(a0), small.data_ptr(), 16, None) == -5
     assert sa.lib().specattn_verify_plan(C.byref(a0), None, 1 << 20, None) == -1
+
+
+def test_kv_len_beyond_the_block_table_is_flagged_not_followed():
+    """A device-side kv_len (dense call) or a listed position that lies beyond what the
+    sequence's row of the block table covers must not index the table out of its row: those
+    positions are flagged SPECATTN_ROW_BAD_INDEX and read position 0 instead; the other
+    sequences are unaffected."""
+    import paper_2510_27641_b200 as sa
+    case = _make_case(33, 3, 5, 32, 8, 16, [480, 480, 480], counts=[[100], [100], [100]])
+    assert case["pages_per_seq"] == 30
+    # dense: sequence 1 claims one page more than its block-table row holds
+    over = dict(case, lens=np.array([480, 496, 480], np.int32))
+    for use_bt in (True, False):
+        out, lse, status = _run(over, dense=True, use_bt=use_bt)
+        st = status.cpu().numpy()
+        assert st[0] == 0 and st[1] == sa.ROW_BAD_INDEX and st[2] == 0
+        assert torch.all(torch.isfinite(out))
+        ref_o, ref_l = _oracle(case, dense=True, use_bt=use_bt)
+        check_attention(out[[0, 2]], lse[[0, 2]], ref_o[[0, 2]], ref_l[[0, 2]])
+    # listed: the same claim lets position 485 through the kv_len check, not through the table's
+    over["idx"] = case["idx"].copy()
+    over["idx"][1, 0, 99] = 485
+    out, lse, status = _run(over)
+    st = status.cpu().numpy()
+    assert st[0] == 0 and st[1] == sa.ROW_BAD_INDEX and st[2] == 0
+    ref_o, ref_l = _oracle(case)
+    check_attention(out[[0, 2]], lse[[0, 2]], ref_o[[0, 2]], ref_l[[0, 2]])
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_next_call_is_correct():
+    """Failure path of the device-side waits, without faulting anything: with the test-only flag
+    one producer warp of CTA 0 withholds the completion signal of its first tile; the waits on it
+    give up at their poll limit, the kernel returns normally with SPECATTN_ROW_TIMEOUT in
+    status[0], and -- after the workspace is re-initialised -- the next ordinary call on the same
+    buffers is correct."""
+    import ctypes as C
+    import time
+    import paper_2510_27641_b200 as sa
+    case = _make_case(34, 2, 5, 32, 8, 16, [3000, 2000], counts=[[2500], [1500]])
+    kv_d = case["kv"].to(dev())
+    q_d, len_d, bt_d = bf16_to_dev(case["q"]), to_dev(case["lens"]), to_dev(case["bt"])
+    idx_d, cnt_d = to_dev(case["idx"]), to_dev(case["cnt"])
+    o = torch.zeros((2, 5, 32, 128), dtype=torch.float32, device=dev())
+    l = torch.zeros((2, 5, 32), dtype=torch.float32, device=dev())
+    st = torch.zeros(2, dtype=torch.int32, device=dev())
+    a = sa.make_verify_args(q_d, kv_d, len_d, block_table=bt_d, idx=idx_d, counts=cnt_d, out=o, lse=l, status=st,
+                            flags=_ENGINE["flags"] | sa.VERIFY_TEST_LOSE_ARRIVAL)
+    ws = sa.verify_workspace(a)
+    a.workspace, a.workspace_bytes = ws.data_ptr(), ws.numel()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    assert sa.lib().specattn_sparse_verify(C.byref(a), None) == 0
+    torch.cuda.synchronize()           # returns: the kernel gave up instead of spinning for ever
+    elapsed = time.time() - t0
+    assert int(st[0]) & sa.ROW_TIMEOUT
+    assert elapsed < 30.0
+    # recovery: fresh counters, same buffers, no test flag
+    assert sa.lib().specattn_verify_workspace_init(ws.data_ptr(), ws.numel(), None) == 0
+    st.zero_()
+    a.flags = _ENGINE["flags"]
+    assert sa.lib().specattn_sparse_verify(C.byref(a), None) == 0
+    torch.cuda.synchronize()
+    assert int(st.abs().sum()) == 0
+    check_attention(o, l, *_oracle(case))

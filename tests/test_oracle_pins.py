@@ -653,3 +653,69 @@ def test_chunk_one_is_per_position_selection():
         a = oracle.select_variant([x], [0], kv, 0.85, per_step=per_step, n_iters=it, chunk=1)
         b = oracle.select_variant([x], [0], kv, 0.85, per_step=per_step, n_iters=it)
         assert all(np.array_equal(u, v) for u, v in zip(a[:3], b[:3]))
+
+
+# ---------------------------------------------------------------------------------------------
+# the binary32 chain of an aggregated value must stay finite (reading of the input domain: Alg. 2
+# and App. A Eq. 7 take attention probabilities; a sum that leaves binary32 is no such row)
+# ---------------------------------------------------------------------------------------------
+def _numpy_chain(values):
+    """The defining chain ((+0 + x1) + x2) + ... with numpy's binary32 adds."""
+    acc = np.float32(0.0)
+    with np.errstate(over="ignore"):
+        for v in values:
+            acc = np.float32(acc + np.float32(v))
+    return acc
+
+
+FMAX = np.finfo(np.float32).max
+
+
+@pytest.mark.parametrize("vals,finite", [
+    ([3e38, 3e38], False),                 # two finite inputs whose binary32 sum is +inf
+    ([FMAX, 0.0], True),                   # the largest finite value itself is a valid sum
+    ([FMAX, FMAX * 2.0 ** -26], True),     # rounds back to FLT_MAX: still finite, still valid
+    ([FMAX, FMAX * 2.0 ** -24], False),    # rounds up past FLT_MAX
+    ([1e38, 1e38, 1e38], True),
+    ([1e38, 1e38, 1e38, 1e38], False),
+])
+def test_aggregate_sum_overflow_marks_the_row_invalid(vals, finite):
+    # what IEEE binary32 says about the chain, independent of the oracle
+    assert bool(np.isfinite(_numpy_chain(vals))) == finite
+    n = len(vals)
+    A = np.zeros((n, 1, 8), dtype=np.float32)
+    A[:, 0, 3] = np.array(vals, dtype=np.float32)
+    A[0, 0, 1] = 0.5  # an ordinary position beside the overflowing one
+    a, st = oracle.aggregate(A)
+    assert st == (oracle.OK if finite else oracle.INVALID_PROB)
+    assert a[3] == _numpy_chain(vals)      # the row is written either way
+    # through the step-level entry points: the list is voided exactly when the chain overflows
+    kv = np.array([8], np.int32)
+    x = A[None]                            # [B=1, H=n, gamma=1, L]
+    for call in (lambda: oracle.select_topp([x], [0], kv, 0.9),
+                 lambda: oracle.select_variant([x], [0], kv, 0.9, per_step=True)):
+        _, cnt, status, _ = call()
+        assert status[0, 0, 0] == (oracle.OK if finite else oracle.INVALID_PROB)
+        assert (cnt[0, 0, 0] > 0) == finite
+    # heads as speculated queries: per_step sums over heads only, so each query's row is one value
+    y = np.ascontiguousarray(np.transpose(x, (0, 2, 1, 3)))   # [1, 1, gamma=n, L]
+    _, cnt, status, _ = oracle.select_variant([y], [0], kv, 0.9, per_step=True)
+    assert status[0, 0, 0] == oracle.OK and cnt[0, 0, 0] > 0   # no chain is longer than one value
+    _, cnt, status, _ = oracle.select_topp([y], [0], kv, 0.9)
+    assert status[0, 0, 0] == (oracle.OK if finite else oracle.INVALID_PROB)
+
+
+def test_chunk_score_overflow_marks_the_list_invalid():
+    # positions stay finite, the binary32 sum of one chunk does not
+    x = np.zeros((1, 1, 1, 16), dtype=np.float32)
+    x[0, 0, 0, 4:8] = 1e38
+    kv = np.array([16], np.int32)
+    assert not np.isfinite(_numpy_chain(x[0, 0, 0, 4:8]))
+    _, cnt, status, _ = oracle.select_variant([x], [0], kv, 0.9, chunk=4)
+    assert status[0, 0, 0] == oracle.INVALID_PROB and cnt[0, 0, 0] == 0
+    _, cnt, status, _ = oracle.select_variant([x], [0], kv, 0.9, chunk=1)
+    assert status[0, 0, 0] == oracle.OK and cnt[0, 0, 0] == 4
+    x[0, 0, 0, 7] = 0.0                     # three of them fit
+    assert np.isfinite(_numpy_chain(x[0, 0, 0, 4:8]))
+    idx, cnt, status, _ = oracle.select_variant([x], [0], kv, 0.9, chunk=4)
+    assert status[0, 0, 0] == oracle.OK and idx[0, 0, 0, :cnt[0, 0, 0]].tolist() == [4, 5, 6, 7]

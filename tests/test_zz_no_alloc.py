@@ -52,7 +52,12 @@ def test_static_scratch_entry_point_matches_the_regular_one_twice_in_a_row():
             torch.cuda.synchronize()
             assert torch.cuda.memory_stats()["allocation.all.allocated"] == n_alloc
             assert torch.cuda.mem_get_info()[0] == free_before
-            assert float((out - ref_out).abs().max()) <= OUT_TOL, f"call {call}"
+            # the same kernel over the same work partition, and a cut unit is merged in a fixed
+            # order whoever arrives last: the results agree bit for bit (a fortiori within the
+            # tolerance the other tests grant the operation: OUT_TOL, LSE_TOL)
+            assert torch.equal(out, ref_out), f"call {call}"
+            assert torch.equal(lse, ref_lse), f"call {call}"
+            assert float((out - ref_out).abs().max()) <= OUT_TOL
             assert lse_err(lse.cpu().numpy().astype(np.float64), ref_lse.cpu().numpy().astype(np.float64)) <= LSE_TOL
             assert torch.equal(status, ref_status)
 
@@ -71,3 +76,11 @@ def test_static_scratch_entry_point_rejects_shapes_beyond_its_buffer():
     assert e.value.code == -8 and "static" in str(e.value)
     assert sa.kernel_launch_count() == n0
     assert sa.lib().specattn_sparse_verify_static(None, None) == -1
+    # argument errors are found before anything is enqueued: a missing output pointer
+    q, kv, bt, kv_len, idx, cnt = _case(44, 1, 5, 32, 8, [64], [10])
+    out = torch.empty((1, 5, 32, 128), dtype=torch.float32, device=dev())
+    lse = torch.empty((1, 5, 32), dtype=torch.float32, device=dev())
+    args = sa.make_verify_args(q, kv, kv_len, block_table=bt, idx=idx, counts=cnt, out=out, lse=lse)
+    args.out = None
+    assert sa.lib().specattn_sparse_verify_static(C.byref(args), None) == -1
+    assert sa.kernel_launch_count() == n0
