@@ -175,23 +175,33 @@ def capture(fn):
     return g, sa.kernel_launch_count() - n0
 
 
-def time_replays(g, steps, warmup, barrier=None):
-    """Microseconds per replay, CUDA events on the replaying (current) stream."""
+def time_replays(g, steps, warmup, barrier=None, stats=None):
+    """Microseconds per replay, CUDA events on the replaying (current) stream.  The `steps`
+    replays run back to back inside one bracket (barrier + synchronize on both sides); events
+    recorded between them, without any synchronisation, cut the bracket into up to ten batches
+    whose per-replay times give a median and a minimum (returned through `stats`)."""
     import torch
     for _ in range(warmup):
         g.replay()
     torch.cuda.synchronize()
     if barrier is not None:
         barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        g.replay()
-    e1.record()
+    nb = max(1, min(10, steps))
+    edges = [round(k * steps / nb) for k in range(nb + 1)]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(nb + 1)]
+    ev[0].record()
+    for k in range(nb):
+        for _ in range(edges[k + 1] - edges[k]):
+            g.replay()
+        ev[k + 1].record()
     torch.cuda.synchronize()
     if barrier is not None:
         barrier()
-    return e0.elapsed_time(e1) * 1e3 / steps
+    if stats is not None:
+        per = [ev[k].elapsed_time(ev[k + 1]) * 1e3 / (edges[k + 1] - edges[k]) for k in range(nb)]
+        stats.update(batches=nb, median=round(float(np.median(per)), 3), min=round(float(np.min(per)), 3),
+                     max=round(float(np.max(per)), 3))
+    return ev[0].elapsed_time(ev[nb]) * 1e3 / steps
 
 
 def verify_bytes(cfg, si, counts_layer):
@@ -310,25 +320,27 @@ def run_reference(args, cfg):
 
 
 # ----------------------------------------------------------------------------------------------
-def topp_sweep(dev, reps=5):
+def topp_sweep(dev, reps=5, families=None, sizes=None, ps=None, n_rows=256):
     """Selection micro-benchmark: 256 rows x n x p x family, rows/s per cell (R = 1).
     Each cell is timed as a CUDA graph of launches over rotating copies of the rows (at least
-    256 MB in total, so every launch reads cold data), replayed `reps` times."""
+    256 MB in total, so every launch reads cold data), replayed `reps` times.  Bytes are the
+    algorithmic ones: every row read once plus the index list written."""
     import ctypes as C
     import torch
     import paper_2510_27641_b200 as sa
     import workloads as wl
     out = {}
-    for fam in wl.TOPP_FAMILIES:
-        for n in wl.TOPP_SIZES:
-            base = torch.from_numpy(wl.topp_rows(fam, 256, n, seed=2)).to(dev).view(256, 1, 1, n)
-            copies = max(2, min(64, (256 << 20) // (256 * n * 4)))
+    R = n_rows
+    for fam in (families or wl.TOPP_FAMILIES):
+        for n in (sizes or wl.TOPP_SIZES):
+            base = torch.from_numpy(wl.topp_rows(fam, R, n, seed=2)).to(dev).view(R, 1, 1, n)
+            copies = max(2, min(64, (256 << 20) // (R * n * 4)))
             rows = [base.clone() for _ in range(copies)]
-            kv = torch.full((256,), n, dtype=torch.int32, device=dev)
-            idx = torch.empty((1, 256, 1, n), dtype=torch.int32, device=dev)
-            cnt = torch.empty((1, 256, 1), dtype=torch.int32, device=dev)
-            st = torch.empty((1, 256, 1), dtype=torch.int32, device=dev)
-            for p in wl.TOPP_PS:
+            kv = torch.full((R,), n, dtype=torch.int32, device=dev)
+            idx = torch.empty((1, R, 1, n), dtype=torch.int32, device=dev)
+            cnt = torch.empty((1, R, 1), dtype=torch.int32, device=dev)
+            st = torch.empty((1, R, 1), dtype=torch.int32, device=dev)
+            for p in (ps or wl.TOPP_PS):
                 args = [sa.make_select_args([r], kv, [0], p, idx=idx, counts=cnt, row_status=st) for r in rows]
 
                 def launch_all():
@@ -340,9 +352,13 @@ def topp_sweep(dev, reps=5):
                 torch.cuda.synchronize()
                 g, _ = capture(launch_all)
                 us = time_replays(g, reps, 2) / copies
-                out[f"{fam}/n={n}/p={p}"] = {"us": round(us, 2), "rows_per_s": round(256 / us * 1e6),
-                                             "gbs": round(256 * n * 4 / us / 1e3, 1),
-                                             "kept_mean": float(cnt.float().mean().item())}
+                assert int(st.abs().sum()) == 0, f"row_status not clean in cell {fam}/n={n}/p={p}"
+                kept = float(cnt.float().mean().item())
+                byts = R * (n * 4 + kept * 4)
+                out[f"{fam}/n={n}/p={p}"] = {"us": round(us, 2), "rows_per_s": round(R / us * 1e6),
+                                             "gbs": round(byts / us / 1e3, 1),
+                                             "frac_of_measured": round(byts / us / 1e3 / _measured_peaks()[0], 3),
+                                             "kept_mean": kept}
                 del g
             del rows, idx, base
     return out
@@ -465,6 +481,62 @@ def layer_batched(step, cfg, si, reps=20):
             "note": "upper bound: layers treated as independent; the per-layer launches are the result"}
 
 
+def config_section(cfg, dev, copies, reps=20):
+    """One whole step (select + plans + verify per target layer) of a small configuration, timed
+    as a CUDA graph over `copies` independent copies of ALL its inputs (draft rows, K/V pools,
+    queries), one step per copy in turn, so that every step reads data that is not in L2
+    (config 0's footprint is far below L2; one copy suffices where a step reads more than L2
+    holds).  Bytes are the algorithmic ones of select and verify."""
+    import torch
+    peak = _measured_peaks()[0]
+    built = [build_step(cfg, dev) for _ in range(copies)]
+    si, _, step0, _, _ = built[0]
+    steps = [b[2] for b in built]
+    for st in steps:
+        st.run()
+    torch.cuda.synchronize()
+    assert all(int(st.status.abs().sum()) == 0 and int((st.row_status > 0).sum()) == 0 for st in steps)
+    counts = step0.counts.cpu().numpy()
+    g_step, n_launch = capture(lambda: [st.run() for st in steps])
+    g_sel, _ = capture(lambda: [st.run_select() for st in steps])
+    g_ver, _ = capture(lambda: [st.run_verify(j) for st in steps for j in range(st.n_layers)])
+    stats = {}
+    us = time_replays(g_step, reps, 5, stats=stats) / copies
+    us_sel = time_replays(g_sel, reps, 5) / copies
+    us_ver = time_replays(g_ver, reps, 5) / copies
+    per_layer = [verify_bytes(cfg, si, counts[int(u)]) for u in si.layer_map]
+    v_bytes = sum(b for b, _ in per_layer)
+    kv_bytes = sum(k for _, k in per_layer)
+    dense_kv = int(si.kv_len.astype(np.int64).sum()) * cfg.n_kv_heads * cfg.head_dim * 4 * cfg.n_target_layers
+    s_bytes = select_bytes(cfg, si, len(step0.used), counts)
+    kept = counts[counts >= 0]
+    return {"workload": cfg.name, "us_per_step": round(us, 2),
+            "us_per_step_median": round(stats["median"] / copies, 2), "us_per_step_min": round(stats["min"] / copies, 2),
+            "us_select": round(us_sel, 2), "us_verify": round(us_ver, 2),
+            "launches_per_step": n_launch // copies, "rotating_copies": copies,
+            "algorithmic_bytes": int(s_bytes + v_bytes), "gbs": round((s_bytes + v_bytes) / us / 1e3, 1),
+            "frac_of_measured": round((s_bytes + v_bytes) / us / 1e3 / peak, 4),
+            "select_bytes": int(s_bytes), "select_gbs": round(s_bytes / us_sel / 1e3, 1),
+            "verify_bytes": int(v_bytes), "verify_gbs": round(v_bytes / us_ver / 1e3, 1),
+            "kv_bytes_touched": int(kv_bytes), "kv_bytes_dense": int(dense_kv),
+            "kv_touched_fraction": round(kv_bytes / dense_kv, 4),
+            "kept_min_mean_max": [int(kept.min()), round(float(kept.mean()), 1), int(kept.max())],
+            "ctx_min_max": [int(si.kv_len.min()), int(si.kv_len.max())]}
+
+
+def long_context_layers(dev, want=80, reserve_gb=6.0):
+    """Target layers of config 4 that fit the free HBM: every layer holds its own 2.147 GB K/V
+    pool (batch 4 x 131072 positions x 8 heads x 128 x K and V in bf16)."""
+    import torch
+    import workloads as wl
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info(dev)
+    cfg = wl.config4(n_target_layers=1)
+    per_layer = cfg.batch * cfg.ctx * cfg.n_kv_heads * cfg.head_dim * 2 * 2
+    draft = cfg.n_draft_layers * cfg.batch * cfg.n_draft_heads * cfg.gamma * cfg.ctx * 4 * 2   # rows + sums
+    return int(max(1, min(want, (free - reserve_gb * 1e9 - draft) // per_layer)))
+
+
 def long_context(dev, reps=10, n_layers=8):
     """Config 4 (batch 4, ctx 131072, 64 q / 8 kv heads, gamma 4, 4 draft layers of 16 heads) on
     `n_layers` target layers of the 80 (each has its own 2.1 GB K/V pool, so nothing is served
@@ -537,8 +609,12 @@ def main():
                     help="force one implementation of sparse_verify (default: the library picks by shape)")
     ap.add_argument("--long-context", action="store_true", help="only run the config-4 (ctx 131072) measurements")
     ap.add_argument("--no-long-context", action="store_true", help="skip the config-4 (ctx 131072) measurements")
-    ap.add_argument("--long-context-layers", type=int, default=8,
-                    help="target layers of config 4 held on the device (2.1 GB of K/V each)")
+    ap.add_argument("--long-context-layers", type=int, default=0,
+                    help="target layers of config 4 held on the device (2.1 GB of K/V each); "
+                         "0 = as many of the 80 as the free HBM holds")
+    ap.add_argument("--no-small-configs", action="store_true", help="skip configs 0 and 3")
+    ap.add_argument("--topp-case", default="",
+                    help="only run one cell of the selection micro-benchmark: family,n,p,rows (e.g. zipf,131072,0.9,32)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of target layers (debug)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-select-workspace", action="store_true",
@@ -573,8 +649,14 @@ def main():
         return
 
     if args.long_context:
-        print(json.dumps({"long_context": long_context(dev, reps=min(10, max(2, args.steps)),
-                                                       n_layers=args.long_context_layers)}))
+        nl = args.long_context_layers or long_context_layers(dev)
+        print(json.dumps({"long_context": long_context(dev, reps=min(10, max(2, args.steps)), n_layers=nl)}))
+        return
+
+    if args.topp_case:
+        fam, n, p, rows = args.topp_case.split(",")
+        print(json.dumps({"topp_case": topp_sweep(dev, reps=min(5, max(1, args.steps)), families=[fam], sizes=[int(n)],
+                                                   ps=[float(p)], n_rows=int(rows))}))
         return
 
     # every rank owns a batch of its own (batch sharding): same shapes, rank-specific seed
@@ -596,7 +678,8 @@ def main():
         uuid = None
     sampler = ClockSampler(local_rank, uuid)
     with sampler:
-        us_step = time_replays(g_step, args.steps, args.warmup, barrier)
+        step_stats = {}
+        us_step = time_replays(g_step, args.steps, args.warmup, barrier, stats=step_stats)
         us_verify_all = time_replays(g_verify, args.steps, args.warmup)
         us_select = time_replays(g_select, args.steps, args.warmup)
     clocks = sampler.summary()
@@ -668,7 +751,7 @@ def main():
             "e2e": {"value": round(us_e2e, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(n_step * args.steps),
             "clocks": clocks, "roofline": roofline,
-            "extra": {"us_verify_per_step": round(us_verify_all, 3), "us_select_per_step": round(us_select, 3),
+            "extra": {"us_step_batches": step_stats, "us_verify_per_step": round(us_verify_all, 3), "us_select_per_step": round(us_select, 3),
                       "us_step_eager_launches": round(us_eager, 3),
                       "topp_lists_per_s": round(n_used * cfg.batch / us_select * 1e6),
                       "topp_prob_rows_per_s": round(n_used * cfg.batch * cfg.n_draft_heads * cfg.gamma / us_select * 1e6),
@@ -693,8 +776,14 @@ def main():
         us_cpu, sample = smp.step_us()
         line["cpu_baseline"] = {"value": round(us_cpu, 1), "unit": UNIT, "cores": smp.cores, "kind": "oracle",
                                 "sample": sample}
+    # the step's own buffers (34 GB of K/V pools) make room for the other configurations
+    del g_step, g_verify, g_select, step, pools
+    if "smp" in locals():
+        del smp
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
     if rank == 0 and not args.no_topp_sweep:
-        del g_step, g_verify, g_select
         extra("topp_sweep", lambda: topp_sweep(dev))
         sweep = line["extra"]["topp_sweep"]
         if "error" not in sweep:
@@ -704,10 +793,15 @@ def main():
             for k, v in sweep.items():
                 by_n.setdefault(k.split("/")[1], []).append(v["rows_per_s"])
             line["extra"]["topp_rows_per_s"] = {n: round(float(np.exp(np.mean(np.log(v))))) for n, v in by_n.items()}
-    if rank == 0 and not args.no_long_context:
-        del step, pools
+    if rank == 0 and not args.no_small_configs:
+        # config 0 is latency-bound (0.8 MB of draft rows, 3 MB of K/V): 64 rotating copies of
+        # all inputs keep every step's reads out of L2; config 3 reads more than L2 per step
+        extra("config0", lambda: config_section(wl.config0(), dev, copies=64))
         torch.cuda.empty_cache()
-        extra("long_context", lambda: long_context(dev, n_layers=args.long_context_layers))
+        extra("config3", lambda: config_section(wl.config3(), dev, copies=1))
+        torch.cuda.empty_cache()
+    if rank == 0 and not args.no_long_context:
+        extra("long_context", lambda: long_context(dev, n_layers=args.long_context_layers or long_context_layers(dev)))
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
