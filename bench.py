@@ -405,7 +405,13 @@ def verify_micro(dev, reps=10, flags=0):
              ("dense_b4_ctx131072_q5x64_kv8", 4, 131072, 5, 64, 8, None),
              ("sparse1245_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, 1245),
              ("sparse12450_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, 12450),
-             ("sparse1000_b4_ctx131072_q5x64_kv8", 4, 131072, 5, 64, 8, 1000)]
+             ("sparse1000_b4_ctx131072_q5x64_kv8", 4, 131072, 5, 64, 8, 1000),
+             # the same number of positions as scattered tokens and as whole 16-position chunks
+             # (the second with SPECATTN_VERIFY_PAGE_LISTS: page-wise K/V reads)
+             ("tokens1536_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, 1536),
+             ("chunks96x16_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, -96),
+             ("tokens12288_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, 12288),
+             ("chunks768x16_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, -768)]
     for name, B, L, T, Hq, Hkv, count in cases:
         page = 16
         pps = (L + page - 1) // page
@@ -415,8 +421,17 @@ def verify_micro(dev, reps=10, flags=0):
         kv_len = torch.full((B,), L, dtype=torch.int32, device=dev)
         o = torch.empty((B, T, Hq, 128), dtype=torch.float32, device=dev)
         l = torch.empty((B, T, Hq), dtype=torch.float32, device=dev)
+        case_flags = flags
         if count is None:
             kw, c = dict(dense=True), L
+        elif count < 0:
+            nch = -count
+            ch = torch.stack([torch.sort(torch.randperm(L // 16, device=dev)[:nch])[0] for _ in range(B)])
+            idx = (ch[:, :, None] * 16 + torch.arange(16, device=dev)[None, None, :]).reshape(B, 1, nch * 16)
+            kw = dict(idx=idx.to(torch.int32).contiguous(),
+                      counts=torch.full((B, 1), nch * 16, dtype=torch.int32, device=dev))
+            c = nch * 16
+            case_flags = flags | sa.VERIFY_PAGE_LISTS
         else:
             idx = torch.stack([torch.sort(torch.randperm(L, device=dev)[:count])[0] for _ in range(B)])
             kw = dict(idx=idx.to(torch.int32).view(B, 1, count).contiguous(),
@@ -425,7 +440,7 @@ def verify_micro(dev, reps=10, flags=0):
         a = sa.make_verify_args(q, kv, kv_len, block_table=bt, out=o, lse=l, idx=kw.get("idx"),
                                 counts=kw.get("counts"), dense=kw.get("dense", False))
         ws = sa.verify_workspace(a)
-        f = lambda: sa.sparse_verify(q, kv, kv_len, block_table=bt, out=o, lse=l, workspace=ws, flags=flags, **kw)
+        f = lambda: sa.sparse_verify(q, kv, kv_len, block_table=bt, out=o, lse=l, workspace=ws, flags=case_flags, **kw)
         for _ in range(3):
             f()
         torch.cuda.synchronize()

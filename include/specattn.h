@@ -209,15 +209,27 @@ size_t specattn_select_workspace_bytes(const specattn_select_args* args);
  * SPECATTN_VERIFY_ENGINE_MMA_SYNC / SPECATTN_VERIFY_ENGINE_TCGEN05: force one of the two
  * implementations of the same operation (warp-level mma.sync with register accumulators, or
  * tcgen05.mma with accumulators in tensor memory).  With neither bit the library picks by
- * what the host can see: tcgen05 for dense calls with more than 32 query rows per KV head
- * (n_q * n_q_heads / n_kv_heads) over caches of at least 8192 positions per sequence
- * (block_table_stride * page_size), mma.sync otherwise -- list lengths live on the device, so a
+ * what the host can see: tcgen05 for dense calls over caches of at least 8192 positions per
+ * sequence (block_table_stride * page_size) that either have more than 32 query rows per KV head
+ * (n_q * n_q_heads / n_kv_heads) or can be read page-wise (page_size a multiple of 16, n_pages
+ * given), mma.sync otherwise -- list lengths live on the device, so a
  * caller that knows its lists are long (thousands of positions per sequence) and has more than
  * 32 query rows should set SPECATTN_VERIFY_ENGINE_TCGEN05 itself.  Results agree within the
  * tolerance of the operation either way.  Setting both bits is SPECATTN_ERR_RANGE. */
 #define SPECATTN_VERIFY_LISTS_STABLE 1u
 #define SPECATTN_VERIFY_ENGINE_MMA_SYNC 2u
 #define SPECATTN_VERIFY_ENGINE_TCGEN05 4u
+/* SPECATTN_VERIFY_PAGE_LISTS: the caller promises that every list consists of whole aligned
+ * 16-position chunks -- entries 16 a ... 16 a + 15 are 16 consecutive positions starting at a
+ * multiple of 16, for every a; only the last chunk of a list may be shorter (cut at kv_len or at
+ * idx_stride).  Lists written by specattn_select_topp with chunk = 16, 32 or 64 have this form
+ * (Sec. 4: chunk size 16).  Where the cache's page size is a multiple of 16 and n_pages is given,
+ * the kernel then reads K/V page-wise -- one list entry, one block-table entry and four tiled
+ * bulk tensor copies (16 slots x 128 bytes each) per 16 tokens instead of 16 entries and 512
+ * 16-byte copies -- and so does every dense call.  A list that breaks the promise gives wrong
+ * results for its sequence (entries that are not multiples of 16 raise SPECATTN_ROW_BAD_INDEX),
+ * never a fault.  Results are the same as without the flag. */
+#define SPECATTN_VERIFY_PAGE_LISTS 8u
 /* TEST ONLY -- never set this in production.  Exercises the failure path of the kernels' bounded
  * device-side waits without faulting anything: one producer warp of CTA 0 withholds the
  * completion signal of its first tile, the waits on it give up after their poll limit (about

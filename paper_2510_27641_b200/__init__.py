@@ -17,13 +17,14 @@ __all__ = ["select_topp", "sparse_verify", "sparse_verify_static", "verify_works
            "SelectArgs", "VerifyArgs", "StepHostArgs", "lib", "SpecAttnError",
            "ROW_OK", "ROW_INVALID_PROB", "ROW_OVERFLOW", "ROW_BAD_INDEX", "ROW_TIMEOUT",
            "VERIFY_LISTS_STABLE", "VERIFY_ENGINE_MMA_SYNC", "VERIFY_ENGINE_TCGEN05",
-           "VERIFY_TEST_LOSE_ARRIVAL", "verify_plan",
+           "VERIFY_TEST_LOSE_ARRIVAL", "VERIFY_PAGE_LISTS", "verify_plan",
            "verify_plan_buffer", "verify_plan_many"]
 
 ROW_OK, ROW_INVALID_PROB, ROW_OVERFLOW, ROW_BAD_INDEX, ROW_TIMEOUT = 0, 1, 2, 4, 8
 VERIFY_LISTS_STABLE = 1
 VERIFY_ENGINE_MMA_SYNC = 2
 VERIFY_ENGINE_TCGEN05 = 4
+VERIFY_PAGE_LISTS = 8
 VERIFY_TEST_LOSE_ARRIVAL = 0x80000000   # test only: see include/specattn.h
 
 _LIB_PATH = Path(__file__).resolve().parent / "libspecattn.so"

@@ -25,6 +25,7 @@
 //     cut between CTAs is finished by whichever CTA arrives last at the unit's counter, which
 //     merges all partial (O, m, l) records in a fixed order -- nobody ever waits on a peer.
 // Every mbarrier wait is bounded; on expiry the CTA flags SPECATTN_ROW_TIMEOUT and leaves.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <math.h>
@@ -1092,12 +1093,56 @@ int row_blocks(const specattn_verify_args& A) { return (m_tiles(A) + 1) / 2; }
 // 3.6-3.9 TB/s; up to 32 rows, and on short lists at any size (one-shot set-up and merge cost),
 // mma.sync is ahead.  List lengths live on the device, so only dense calls whose cache holds at
 // least 8192 positions per sequence are switched.
+bool page_granular(const specattn_verify_args& A);
 bool use_tcgen05(const specattn_verify_args& A) {
   if (A.flags & SPECATTN_VERIFY_ENGINE_TCGEN05) return true;
   if (A.flags & SPECATTN_VERIFY_ENGINE_MMA_SYNC) return false;
   const long long rows = static_cast<long long>(A.n_q) * (A.n_q_heads / A.n_kv_heads);
   const long long capacity = static_cast<long long>(A.block_table_stride) * A.page_size;
-  return A.dense && rows > 32 && capacity >= 8192;
+  // (with page-wise K/V reads the tcgen05 engine is ahead on long dense caches at any number of
+  // query rows: 24 rows over 4 x 131072 positions 5.5 TB/s against 5.3)
+  return A.dense && capacity >= 8192 && (rows > 32 || page_granular(A));
+}
+
+// Page-granular K/V reads (tiled bulk tensor copies of 16-slot boxes) apply to dense calls and to
+// lists the caller declares to be made of whole aligned 16-position chunks, when a page holds a
+// multiple of 16 slots and the pool's extent is known.
+bool page_granular(const specattn_verify_args& A) {
+  return (A.dense || (A.flags & SPECATTN_VERIFY_PAGE_LISTS)) && A.page_size % 16 == 0 && A.n_pages > 0 &&
+         A.n_pages < (1ll << 31) && A.n_kv_heads <= 256 && A.page_size <= 4096;
+}
+
+// The K/V pool as a 5-D tensor (element, head, slot, k/v, page) with a box of [64 elements x 1
+// head x 16 slots], 128-byte swizzle: one box is one 128-byte half of 16 consecutive rows in the
+// tcgen05 operand layout.  The driver's encoder is looked up through the runtime (no link-time
+// dependency on the driver library).  Returns false if it is unavailable or refuses the strides.
+bool make_kv_map(const specattn_verify_args& A, CUtensorMap* map) {
+  typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static std::atomic<encode_fn> cached{nullptr};
+  encode_fn fn = cached.load(std::memory_order_acquire);
+  if (fn == nullptr) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess || sym == nullptr) {
+      cudaGetLastError();
+      return false;
+    }
+    fn = reinterpret_cast<encode_fn>(sym);
+    cached.store(fn, std::memory_order_release);
+  }
+  const cuuint64_t dims[5] = {static_cast<cuuint64_t>(kD), static_cast<cuuint64_t>(A.n_kv_heads),
+                              static_cast<cuuint64_t>(A.page_size), 2ull, static_cast<cuuint64_t>(A.n_pages)};
+  const cuuint64_t strides[4] = {static_cast<cuuint64_t>(A.stride_head) * 2, static_cast<cuuint64_t>(A.stride_slot) * 2,
+                                 static_cast<cuuint64_t>(A.stride_kv) * 2, static_cast<cuuint64_t>(A.stride_page) * 2};
+  const cuuint32_t box[5] = {64u, 1u, 16u, 1u, 1u};
+  const cuuint32_t elem[5] = {1u, 1u, 1u, 1u, 1u};
+  if (A.stride_head <= 0 || A.stride_slot <= 0 || A.stride_kv <= 0 || A.stride_page <= 0) return false;
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(A.kv_pages), dims, strides, box, elem,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Sized for either engine, so that the choice never depends on the workspace at hand.
@@ -1211,11 +1256,22 @@ extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cu
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t err;
   if (specattn::use_tcgen05(A)) {
-    switch (specattn::m_tiles(A)) {
-      case 1: err = specattn::launch_tc<1>(P, n_ctas, stream); break;
-      case 2: err = specattn::launch_tc<2>(P, n_ctas, stream); break;
-      case 3: err = specattn::launch_tc<3>(P, n_ctas, stream); break;
-      default: err = specattn::launch_tc<4>(P, n_ctas, stream); break;
+    alignas(64) CUtensorMap kv_map;
+    memset(&kv_map, 0, sizeof(kv_map));
+    if (specattn::page_granular(A) && specattn::make_kv_map(A, &kv_map)) {
+      switch (specattn::m_tiles(A)) {
+        case 1: err = specattn::launch_tc<1, true>(P, kv_map, n_ctas, stream); break;
+        case 2: err = specattn::launch_tc<2, true>(P, kv_map, n_ctas, stream); break;
+        case 3: err = specattn::launch_tc<3, true>(P, kv_map, n_ctas, stream); break;
+        default: err = specattn::launch_tc<4, true>(P, kv_map, n_ctas, stream); break;
+      }
+    } else {
+      switch (specattn::m_tiles(A)) {
+        case 1: err = specattn::launch_tc<1, false>(P, kv_map, n_ctas, stream); break;
+        case 2: err = specattn::launch_tc<2, false>(P, kv_map, n_ctas, stream); break;
+        case 3: err = specattn::launch_tc<3, false>(P, kv_map, n_ctas, stream); break;
+        default: err = specattn::launch_tc<4, false>(P, kv_map, n_ctas, stream); break;
+      }
     }
   } else {
     switch (specattn::m_tiles(A)) {

@@ -22,6 +22,15 @@
 // rescale of the O^T columns in tensor memory).  Whether a tile takes it is agreed per tile
 // through one named barrier of the softmax warps.
 //
+// Page-granular calls (kPaged: dense calls, and lists made of whole aligned 16-position chunks, on
+// caches whose page size is a multiple of 16): a 16-token atom of a unit is 16 consecutive slots
+// of one page, i.e. a regular [16 slots x 64 elements] box of the K/V pool for each 128-byte half
+// of the head dimension.  Those tiles are fetched with tiled bulk tensor copies (TMA, 128-byte
+// swizzle: exactly the operand layout above, completion counted in bytes on the stage's barrier)
+// -- four requests per atom instead of 512 16-byte copies, no per-thread addresses, no proxy
+// fence.  Half tiles that hold in-flight tokens behind a list, or a list's cut last chunk, take
+// the per-row path.
+//
 // Warps: 0-7 softmax (TMEM lane quadrant = warp % 4, half of the query rows = warp / 4, so every
 // SM sub-partition runs two of them), 8 = MMA issue (one thread), 9-12 = producers: two warps per tile, 64 keys each, 16-byte cp.async straight into the
 // 128-byte-swizzled operand layout, then fence.proxy.async before the arrival.
@@ -66,6 +75,23 @@ __device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a, uint64_t 
 // arrival on an mbarrier once every tcgen05 operation issued so far by this thread has completed
 __device__ __forceinline__ void tc_commit(unsigned long long* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// One box of a 5-D tiled tensor map (element, head, slot, k/v, page) into shared memory; bytes are
+// counted on `bar`.  No multicast; x (c0) is 0 or 64 elements, i.e. a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_5d(uint32_t dst_smem, const CUtensorMap* map, unsigned long long* bar, int c0,
+                                            int c1, int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::
+          "r"(dst_smem),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+// The same box, only as far as L2 (no destination, no completion to wait for).
+__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4) {
+  asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global.tile [%0, {%1, %2, %3, %4, %5}];" ::"l"(
+                   reinterpret_cast<uint64_t>(map)),
+               "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
                : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -183,8 +209,9 @@ struct TcShared {
 };
 
 // NT = N / 16, N = query rows rounded up to a multiple of 16
-template <int NT>
-__global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const __grid_constant__ VerifyParams P) {
+template <int NT, bool kPaged>
+__global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const __grid_constant__ VerifyParams P,
+                                                                       const __grid_constant__ CUtensorMap kv_map) {
   constexpr int N = NT * 16;
   constexpr int NS = kTcStages;
   constexpr int NTH = kTcThreads;
@@ -436,6 +463,29 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         }
         return bad;
       };
+      // (page-granular) lane j < 4 resolves atom j of this warp's half tile to (page, first slot),
+      // packed as page * 4096 + slot; one list entry and one block-table entry per 16 tokens
+      const int c_list16 = c_list & ~15;
+      auto tma_half = [&](int h0) -> bool {
+        return kPaged && (P.dense || min(h0 + 64, tok_hi) <= c_list16);
+      };
+      auto resolve_atom = [&](int h0, long long& where) -> bool {
+        bool bad = false;
+        where = 0;
+        const int k = h0 + 16 * lane;
+        if (lane < 4 && k < tok_hi) {
+          int pos = P.dense ? k : __ldg(list + k);
+          if (pos < 0 || pos >= kvlen_b + P.tail || (pos & 15)) { bad = true; pos = 0; }
+          int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
+          if (lp >= P.bt_stride) { bad = true; pos = 0; lp = 0; }
+          const int slot = pos - lp * P.page_size;
+          long long page = P.bt ? static_cast<long long>(__ldg(P.bt + b * P.bt_stride + lp))
+                                : (b * P.bt_stride + lp);
+          if (page < 0 || page >= P.n_pages) { bad = true; page = 0; }
+          where = page * 4096 + slot;
+        }
+        return bad;
+      };
       long long off_next[2] = {0, 0};
       bool bad_next = false;
       int t0_next = -1;
@@ -444,6 +494,56 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         const int s = it % NS;
         const unsigned ph = (it / NS) & 1u;
         const int h0 = t0 + half * 64;
+        if (tma_half(h0)) {
+          long long where;
+          bool bad;
+          if (t0_next == t0) {
+            where = off_next[0];
+            bad = bad_next;
+          } else {
+            bad = resolve_atom(h0, where);
+          }
+          t0_next = t0 + 2 * kTcTile;
+          if (t0_next < tok_hi && tma_half(t0_next + half * 64)) {
+            // this warp's next half tile: resolved now, and its boxes asked into L2 at once -- two
+            // tiles ahead of the ring, so that the copies into shared memory find them there
+            bad_next = resolve_atom(t0_next + half * 64, off_next[0]);
+            const int hn = t0_next + half * 64;
+            if (lane < 4 && hn + 16 * lane < tok_hi) {
+              const int page = static_cast<int>(off_next[0] >> 12), slot = static_cast<int>(off_next[0] & 4095);
+              tma_prefetch_5d(&kv_map, 0, kvh, slot, 0, page);
+              tma_prefetch_5d(&kv_map, 64, kvh, slot, 0, page);
+              tma_prefetch_5d(&kv_map, 0, kvh, slot, 1, page);
+              tma_prefetch_5d(&kv_map, 64, kvh, slot, 1, page);
+            }
+          } else {
+            t0_next = -1;
+          }
+          if (!mbar_wait(&sh.empty[s], ph ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
+          const int ntok = max(0, min(64, tok_hi - h0));
+          const int natoms = (ntok + 15) >> 4;
+          if (lane == 0) {
+            // 4 boxes of 2 KB per atom: K and V, two 128-byte halves of the head dimension each
+            if (natoms > 0) mbar_arrive_expect_tx(&sh.full[s], static_cast<uint32_t>(natoms) * 4u * 2048u);
+            else mbar_arrive(&sh.full[s]);
+          }
+          __syncwarp();
+          if (lane < natoms) {
+            const int page = static_cast<int>(where >> 12), slot = static_cast<int>(where & 4095);
+            const uint32_t k_dst = smem_u32(sh.kv[s]) + (half * 64 + 16 * lane) * 128;
+            const uint32_t v_dst = k_dst + kTcTileBytes;
+            tma_load_5d(k_dst, &kv_map, &sh.full[s], 0, kvh, slot, 0, page);
+            tma_load_5d(k_dst + kTcTile * 128, &kv_map, &sh.full[s], 64, kvh, slot, 0, page);
+            tma_load_5d(v_dst, &kv_map, &sh.full[s], 0, kvh, slot, 1, page);
+            tma_load_5d(v_dst + kTcTile * 128, &kv_map, &sh.full[s], 64, kvh, slot, 1, page);
+          }
+          if (__any_sync(0xffffffffu, bad) && P.status && lane == 0) atomicOr(P.status + b, SPECATTN_ROW_BAD_INDEX);
+          if (q_pending) {
+            q_pending = false;
+            if (!load_q()) { sh.abort_flag = 1; dead = true; break; }
+          }
+          continue;
+        }
         long long off[2] = {0, 0};
         bool bad;
         if (t0_next == t0) {
@@ -454,7 +554,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           bad = resolve(h0, off);
         }
         t0_next = t0 + 2 * kTcTile;
-        if (t0_next < tok_hi) bad_next = resolve(t0_next + half * 64, off_next); else t0_next = -1;
+        if (t0_next < tok_hi && !tma_half(t0_next + half * 64)) bad_next = resolve(t0_next + half * 64, off_next);
+        else t0_next = -1;
         if (!mbar_wait(&sh.empty[s], ph ^ 1u, &sh.abort_flag)) { sh.abort_flag = 1; dead = true; break; }
         const int ntok = max(0, min(64, tok_hi - h0));
         const int npad = (ntok + 15) & ~15;  // the P V product runs over whole 16-key steps
@@ -749,6 +850,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
             st_shared_v4(pb + (ch_hi >> 3) * 16384 + (((ch_hi & 7) ^ (key_lane & 7)) << 4), hi[0], hi[1], hi[2], hi[3]);
             st_shared_v4(pb + (ch_lo >> 3) * 16384 + (((ch_lo & 7) ^ (key_lane & 7)) << 4), lo[0], lo[1], lo[2], lo[3]);
           }
+          if (kPaged && warp < 4 && !kvalid && key_lane < ((ntok + 15) & ~15)) {
+            // a box copy brought 16 whole slots: those beyond the unit's last token hold whatever
+            // the pool holds there (possibly non-finite) and meet P = 0 in the product -- clear them
+            const uint32_t vb = smem_u32(sh.kv[s]) + kTcTileBytes;
+#pragma unroll
+            for (int c = 0; c < 16; ++c) st_shared_v4(vb + tc_sw(key_lane, c, kTcTile), 0u, 0u, 0u, 0u);
+          }
           fence_proxy_async();  // P^T is read by the tensor core through the async proxy
           __syncwarp();
           if (lane == 0) mbar_arrive(&sh.p_full[sb]);
@@ -890,8 +998,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   }
 }
 
-template <int NT>
-cudaError_t launch_tc(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
+template <int NT, bool kPaged>
+cudaError_t launch_tc(const VerifyParams& P, const CUtensorMap& kv_map, int n_ctas, cudaStream_t stream) {
   const size_t smem = sizeof(TcShared) + 1024;
   static std::atomic<unsigned long long> done_mask{0};
   int dev = 0;
@@ -899,7 +1007,7 @@ cudaError_t launch_tc(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
   if (err != cudaSuccess) return err;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   if (!((done_mask.load(std::memory_order_acquire) >> dev) & 1ull)) {
-    err = cudaFuncSetAttribute(sparse_verify_tc_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    err = cudaFuncSetAttribute(sparse_verify_tc_kernel<NT, kPaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                static_cast<int>(smem));
     if (err != cudaSuccess) return err;
     done_mask.fetch_or(1ull << dev, std::memory_order_release);
@@ -915,7 +1023,7 @@ cudaError_t launch_tc(const VerifyParams& P, int n_ctas, cudaStream_t stream) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  err = cudaLaunchKernelEx(&cfg, sparse_verify_tc_kernel<NT>, P);
+  err = cudaLaunchKernelEx(&cfg, sparse_verify_tc_kernel<NT, kPaged>, P, kv_map);
   if (err != cudaSuccess) cudaGetLastError();
   return err;
 }

@@ -365,3 +365,92 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_next_call_is_correct()
     torch.cuda.synchronize()
     assert int(st.abs().sum()) == 0
     check_attention(o, l, *_oracle(case))
+
+
+def _chunk_lists(case, rng, chunk=16, frac=0.4):
+    """Replaces the case's lists by lists of whole aligned chunks (the form specattn_select_topp
+    emits with chunk = 16, 32 or 64): a random subset of each sequence's chunks, always including
+    the last one (cut at kv_len) for half of the lists."""
+    B, G = case["cnt"].shape
+    for b in range(B):
+        L = int(case["lens"][b])
+        n_chunks = (L + chunk - 1) // chunk
+        for g in range(G):
+            take = rng.random(n_chunks) < frac
+            if n_chunks and (b + g) % 2 == 0:
+                take[-1] = True
+            pos = np.concatenate([np.arange(j * chunk, min(L, (j + 1) * chunk)) for j in np.flatnonzero(take)]
+                                 or [np.zeros(0, np.int64)])
+            case["idx"][b, g, :len(pos)] = pos
+            case["idx"][b, g, len(pos):] = 0
+            case["cnt"][b, g] = len(pos)
+
+
+@pytest.mark.parametrize("page,chunk", [(16, 16), (32, 16), (16, 64), (64, 32)])
+def test_page_granular_lists_and_dense_calls(page, chunk):
+    """Lists of whole aligned chunks flagged SPECATTN_VERIFY_PAGE_LISTS, and dense calls, read K/V
+    page-wise (tiled bulk tensor copies in the tcgen05 engine): page sizes 16 to 64, partial last
+    pages and chunks, shuffled block table, per-kv-head lists, lists cut between CTAs.  The slots
+    of a last page beyond kv_len are poisoned with NaN: they must not reach the result."""
+    import paper_2510_27641_b200 as sa
+    rng = np.random.default_rng(page * 100 + chunk)
+    lens = [5000, 777, 16, 1, 4096, 3333]
+    case = _make_case(80 + page, 6, 5, 32, 8, page, lens, G=1)
+    _chunk_lists(case, rng, chunk)
+    kv = case["kv"].clone()
+    for b, L in enumerate(lens):                       # poison what lies beyond kv_len in the last page
+        if L % page:
+            pg = int(case["bt"][b, L // page])
+            kv[pg, :, L % page:] = float("nan")
+    poisoned = dict(case, kv=kv)
+    flags0 = _ENGINE["flags"]
+    try:
+        _ENGINE["flags"] = flags0 | sa.VERIFY_PAGE_LISTS
+        out, lse, status = _run(poisoned)
+        assert int(status.abs().sum()) == 0
+        check_attention(out, lse, *_oracle(case))
+        o_d, l_d, status = _run(poisoned, dense=True)
+        assert int(status.abs().sum()) == 0
+        check_attention(o_d, l_d, *_oracle(case, dense=True))
+        # the flag changes how rows are fetched, not the results
+        _ENGINE["flags"] = flags0
+        out0, lse0, _ = _run(case)
+        assert float((out - out0).abs().max()) <= 2e-5
+        assert float(torch.nan_to_num(lse - lse0, nan=0.0).abs().max()) <= 2e-5    # (-inf) - (-inf): empty lists
+    finally:
+        _ENGINE["flags"] = flags0
+
+
+def test_page_granular_per_head_lists_tails_and_contiguous_cache():
+    import paper_2510_27641_b200 as sa
+    rng = np.random.default_rng(7)
+    flags0 = _ENGINE["flags"]
+    try:
+        _ENGINE["flags"] = flags0 | sa.VERIFY_PAGE_LISTS
+        # per-kv-head lists; in-flight tokens behind the lists (they start in the middle of a page)
+        case = _make_case(90, 3, 5, 16, 4, 16, [2000, 1000, 37], G=4, tail=5)
+        _chunk_lists(case, rng, 16)
+        out, lse, status = _run(case)
+        assert int(status.abs().sum()) == 0
+        check_attention(out, lse, *_oracle(case))
+        # dense + tail: ordinary causal decode attention of the verified tokens, page-wise
+        o_d, l_d, _ = _run(case, dense=True)
+        check_attention(o_d, l_d, *_oracle(case, dense=True))
+        # contiguous cache (no block table), one long sequence cut among all CTAs
+        case = _make_case(91, 1, 6, 8, 2, 32, [40000], shuffle=False)
+        _chunk_lists(case, rng, 32, frac=0.8)
+        out, lse, _ = _run(case, use_bt=False)
+        check_attention(out, lse, *_oracle(case, use_bt=False))
+        o_d, l_d, _ = _run(case, dense=True, use_bt=False)
+        check_attention(o_d, l_d, *_oracle(case, dense=True, use_bt=False))
+        # a list that breaks the promise is flagged, and nothing faults
+        case = _make_case(92, 2, 5, 32, 8, 16, [3000, 3000])
+        _chunk_lists(case, rng, 16)
+        case["idx"][1, 0, 16 * 3] += 5
+        out, lse, status = _run(case)
+        st = status.cpu().numpy()
+        assert st[0] == 0 and torch.all(torch.isfinite(out))
+        if flags0 == sa.VERIFY_ENGINE_TCGEN05:
+            assert st[1] == sa.ROW_BAD_INDEX
+    finally:
+        _ENGINE["flags"] = flags0
