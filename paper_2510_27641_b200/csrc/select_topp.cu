@@ -112,6 +112,8 @@ struct Shared {
   float cta_max;            // read by the other CTAs of the cluster
   int local_kept;           // read by the other CTAs of the cluster
   int bin_lo, bin_hi;       // first and last non-empty level-1 bin of this CTA (read by the cluster)
+  unsigned int bin_kmin, bin_kmax;  // (rows read in place) smallest / largest key of this CTA inside the
+                                    // level-1 threshold bin (read by the cluster)
   int n_cand;               // keys this CTA found in the level-1 threshold bin (read by the cluster)
   unsigned int cand[kCandCap];
   int cand_pos[kCandCap];   // (rows read in place) their positions inside the slice
@@ -385,7 +387,11 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   // In-place passes read the row from global memory (L2) with four independent 16-byte loads per
   // thread in flight: with one dependent load per iteration a CTA moved ~4 GB/s (latency-bound);
   // eight in flight were 3-4 % slower on 64k / 128k rows than four (twice the code per pass), two
-  // 3 % slower again.
+  // 3 % slower again.  Asking for the pieces ahead into L2 (bulk prefetch, 64 KB ahead per CTA)
+  // changed nothing: the passes are not waiting for HBM.  Two copies of the level-1 histogram for
+  // even and odd lanes (rows of probabilities only use the lower half of the bins) made the pass
+  // 30 % slower, with the copies in the same banks or in different ones: lanes that hit the same
+  // bin in one instruction are not what the pass waits for.
   constexpr int kIpUnroll = 4;
   auto load_keys4 = [&](int i4, unsigned int (&key)[4]) -> bool {  // keys of positions 4*i4 .. 4*i4+3
     const bool act = i4 < n4;
@@ -418,6 +424,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   bool invalid = false;
   if (tid == 0) sh.n_invalid = 0;
   bool short_cut = false;  // the threshold was found among the gathered keys of the level-1 bin
+  bool tie_done = false;   // (rows read in place) the threshold bin held one distinct value: the threshold
   // (in place) the kept positions as ballot words, four per 128 positions, in the upper half of
   // the scan array: by the time they are written the level-1 scan is over, the later levels use
   // the lower half only, and no peer reads this array after the level-1 gather
@@ -467,12 +474,13 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
         unsigned int mant[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const float x = __uint_as_float(key[uu][e]);
-          bad |= act[uu] && !(x >= 0.f && x <= FLT_MAX);  // negative, NaN or infinite
-          if (kVariant && !chunked) vmax = fmaxf(vmax, x);
-          take[e] = act[uu] && (4 * i4 + e < n_loc) && key[uu][e] != 0u && !(key[uu][e] >> 31) && !chunked;
-          bin[e] = static_cast<int>(key[uu][e] >> 20);
-          mant[e] = mantissa_of(key[uu][e]);
+          const unsigned int k = key[uu][e];
+          // negative, NaN or infinite: sign bit set, or an all-ones exponent
+          bad |= act[uu] && k > 0x7f7fffffu;
+          if (kVariant && !chunked) vmax = fmaxf(vmax, __uint_as_float(k));
+          take[e] = act[uu] && (4 * i4 + e < n_loc) && k != 0u && !(k >> 31) && !chunked;
+          bin[e] = static_cast<int>(k >> 20);
+          mant[e] = mantissa_of(k);
         }
         hist_add4(h1, take, bin, mant);
       }
@@ -715,10 +723,119 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   }
   // every thread has read the bin's mass before a faster warp's ballot words can land on it
   if (kInPlace) __syncthreads();
+  // What the candidates are: the keys whose bits above `csh` equal `cpre` -- the level-1 bin
+  // (11 bits), or, after the merged pass below, a level-2 bin inside it (21 bits).
+  int csh = 20, lvl0 = 0;
+  unsigned int cpre = prefix;
+  tie_done = false;
+  bool level2_done = false;  // the merged pass ran but its bin is too full for the short cut
+  const double m_ge_l1 = searching ? sh.mass_ge : 0.0;
+  if (kInPlace && !kVariant && searching && !short_cut) {
+    // Rows read in place whose threshold bin is well filled (flat or tie-heavy rows).  Every pass
+    // over such a row costs as much as the level-1 pass, so the second one does three things at
+    // once: it notes the positions inside or above the threshold bin as ballot words, builds the
+    // level-2 histogram of the bin, and tracks the smallest and largest key inside the bin.  If
+    // those are equal (ties) the search is over and the ballot words are the kept set; otherwise
+    // the level-2 bin found is normally sparse enough for the short cut, whose candidate pass
+    // then is the third and last pass over the row (five before: two more histogram levels, a
+    // count pass and the write pass's own read).
+    unsigned int* const lb2 = lvl_base;                                  // level-2 histogram
+    const Hist hr = {lb2, lb2 + kL23Bins};
+    unsigned int kmin = 0xffffffffu, kmax = 0u;
+    for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
+      unsigned int key[kIpUnroll][4];
+      bool act[kIpUnroll];
+#pragma unroll
+      for (int uu = 0; uu < kIpUnroll; ++uu) act[uu] = load_keys4(base + uu * kThreads + tid, key[uu]);
+#pragma unroll
+      for (int uu = 0; uu < kIpUnroll; ++uu) {
+        const int i4 = base + uu * kThreads + tid;
+        unsigned int mine = 0u;
+        bool take[4];
+        int bin[4];
+        unsigned int mant[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const unsigned int k = key[uu][e];
+          const bool in_row = act[uu] && (4 * i4 + e < n_loc);
+          const bool inb = in_row && (k >> 20) == prefix;
+          take[e] = inb;
+          bin[e] = static_cast<int>((k >> 10) & 1023u);
+          mant[e] = mantissa_of(k);
+          kmin = inb ? min(kmin, k) : kmin;
+          kmax = inb ? max(kmax, k) : kmax;
+          // in the bin or above it: exactly the kept set if the bin turns out to hold one value
+          const unsigned int m = __ballot_sync(kFull, in_row && (k >> 20) >= prefix);
+          if (lane == e) mine = m;
+        }
+        hist_add4(hr, take, bin, mant);
+        const int g4 = base + uu * kThreads + (tid & ~31);  // first float4 of this warp's 32
+        if (lane < 4 && g4 < n4) keep_words[(g4 >> 5) * 4 + lane] = mine;
+      }
+    }
+    kmin = __reduce_min_sync(kFull, kmin);
+    kmax = __reduce_max_sync(kFull, kmax);
+    if (lane == 0) {
+      sh.red_key[warp] = kmin;
+      sh.red_key[kWarps + warp] = kmax;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      unsigned int a0 = 0xffffffffu, a1 = 0u;
+      for (int w = 0; w < kWarps; ++w) {
+        a0 = min(a0, sh.red_key[w]);
+        a1 = max(a1, sh.red_key[kWarps + w]);
+      }
+      sh.bin_kmin = a0;
+      sh.bin_kmax = a1;
+    }
+    csync();  // every CTA's level-2 histogram and key range are complete
+    kmin = 0xffffffffu;
+    kmax = 0u;
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      if (r < cs) {
+        kmin = min(kmin, *cluster.map_shared_rank(&sh.bin_kmin, r));
+        kmax = max(kmax, *cluster.map_shared_rank(&sh.bin_kmax, r));
+      }
+    }
+    if (kmin == kmax) {
+      // one distinct value in the bin: it is the threshold, and all its positions are kept
+      theta_key = kmin;
+      m_gt = carry_m;
+      m_ge = m_ge_l1;
+      tie_done = true;
+    } else {
+      const double scale = pow2_double(e1);
+      for (int bin = tid; bin < kL23Bins; bin += kThreads) {
+        unsigned long long ml = 0, mh = 0;
+        for (int r = 0; r < cs; ++r) {
+          const unsigned int* src = cluster.map_shared_rank(lb2, r);
+          ml += src[bin];
+          mh += src[kL23Bins + bin];
+        }
+        r_mass[bin] = static_cast<double>((mh << 16) + ml) * scale;
+      }
+      __syncthreads();
+      scan_bins(sh, r_mass, kL23Bins, carry_m, target, false, P.p);
+      const unsigned long long S2 =
+          static_cast<unsigned long long>(r_mass[sh.found_bin] * pow2_double(-e1));
+      prefix = (prefix << 10) | static_cast<unsigned int>(sh.found_bin);
+      carry_m = sh.mass_above;
+      level2_done = true;
+      if ((S2 >> 23) <= static_cast<unsigned long long>(kCandCap)) {
+        short_cut = true;
+        csh = 10;
+        lvl0 = 1;
+        cpre = prefix;
+      }
+      __syncthreads();  // everybody has read r_mass / the scan results before they are reused
+    }
+  }
   if (short_cut) {
     if (in_place) {
-      for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
-        unsigned int key[kIpUnroll][4];
+        for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
+          unsigned int key[kIpUnroll][4];
         bool act[kIpUnroll];
 #pragma unroll
         for (int uu = 0; uu < kIpUnroll; ++uu) act[uu] = load_keys4(base + uu * kThreads + tid, key[uu]);
@@ -732,8 +849,8 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const bool in_row = act[uu] && (4 * i4 + e < n_loc);
-            cand_add(sh, in_row && (key[uu][e] >> 20) == prefix, key[uu][e], 4 * i4 + e);
-            const unsigned int m = __ballot_sync(kFull, in_row && (key[uu][e] >> 20) > prefix);
+            cand_add(sh, in_row && (key[uu][e] >> csh) == cpre, key[uu][e], 4 * i4 + e);
+            const unsigned int m = __ballot_sync(kFull, in_row && (key[uu][e] >> csh) > cpre);
             if (lane == e) mine = m;
           }
           const int g4 = base + uu * kThreads + (tid & ~31);  // first float4 of this warp's 32
@@ -744,7 +861,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       for (int base = 0; base < n_srch; base += kThreads) {
         const int i = base + tid;
         const unsigned int key = (i < n_srch) ? key_at(i) : 0u;
-        cand_add(sh, i < n_srch && (key >> 20) == prefix, key, i);
+        cand_add(sh, i < n_srch && (key >> csh) == cpre, key, i);
       }
     }
     csync();  // every CTA's candidate list is complete
@@ -827,10 +944,10 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       m_gt = carry_m + static_cast<double>(s_gt) * scale;
       m_ge = carry_m + static_cast<double>(s_ge) * scale;
     } else {
-    unsigned int pre = prefix;
+    unsigned int pre = cpre;
     double carry = carry_m;
 #pragma unroll 1
-    for (int level = 0; level < 2; ++level) {
+    for (int level = lvl0; level < 2; ++level) {
       const int shift = (level == 0) ? 10 : 0;
       unsigned int* lb = lvl_base + level * 2 * kL23Bins;  // zeroed above; the cluster does not use it on this path
       const Hist hr = {lb, lb + kL23Bins};
@@ -865,16 +982,16 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       }
       __syncthreads();
     }
-  } else
-  for (int level = 0; level < 2; ++level) {
+  } else if (!tie_done) {
+  for (int level = level2_done ? 1 : 0; level < 2; ++level) {
     const int shift = (level == 0) ? 10 : 0;
     unsigned int* lb = lvl_base + level * 2 * kL23Bins;
     if (searching) {
       // only the elements inside the threshold bin take part
       const Hist hr = {lb, lb + kL23Bins};
       if (in_place) {
-        for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
-          unsigned int key[kIpUnroll][4];
+            for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
+              unsigned int key[kIpUnroll][4];
           bool act[kIpUnroll];
 #pragma unroll
           for (int uu = 0; uu < kIpUnroll; ++uu) act[uu] = load_keys4(base + uu * kThreads + tid, key[uu]);
@@ -918,7 +1035,8 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
       carry_m = sh.mass_above;
     }
   }
-  if (searching && !short_cut) {
+  }
+  if (searching && !short_cut && !tie_done) {
     theta_key = prefix;
     m_gt = sh.mass_above;
     m_ge = sh.mass_ge;
@@ -973,7 +1091,7 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   const int w4_lo = min(n4, warp * wchunk4);
   const int w4_hi = min(n4, w4_lo + wchunk4);
   int wc = 0;
-  if (!invalid && in_place && !kVariant && short_cut) {
+  if (!invalid && in_place && !kVariant && (short_cut || tie_done)) {
     // the kept positions are already in the ballot words: count this warp's
     // (a warp whose range is empty has w4_lo == w4_hi == n4, not a multiple of 32)
     if (w4_lo < w4_hi)
