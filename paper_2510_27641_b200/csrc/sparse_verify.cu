@@ -437,6 +437,8 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   const int lane = tid & 31;
   const int warp = tid >> 5;
   const int U = P.B * P.Hkv;
+  constexpr bool kQReload = (WPM == 2);   // query fragments re-read from shared memory per block
+  constexpr bool kDirectQ = !kQReload;    // consumers fetch the CTA's first query block themselves
 
   // Unless the caller vouched for the lists, nothing is read before the previous kernel is
   // done.  Only then may the next kernel of the stream be scheduled: a successor that starts
@@ -659,6 +661,14 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       // K/V prefetch is already in flight while the warp waits for the previous kernel.
       auto load_q = [&]() -> bool {
         if (seg == 0 && P.lists_stable) pdl_wait();
+        if (kDirectQ && seg == 0) {
+          // The consumers fetch the first query block themselves (see there); only the barrier's
+          // phase is completed here, so that later segments find the parity they expect.  (No wait
+          // on q_empty: nobody reads an older block, and the consumers may already have released
+          // this one -- the "previous phase" a fresh barrier grants would then be one they hold.)
+          if (lane == 0) mbar_arrive(&sh.q_full);
+          return true;
+        }
         if (!mbar_wait(&sh.q_empty, (seg & 1u) ^ 1u, &sh.abort_flag)) return false;
         if (lane == 0) mbar_arrive_expect_tx(&sh.q_full, static_cast<uint32_t>(P.M) * kRowBytes);
         __syncwarp();
@@ -803,9 +813,27 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     // re-read from shared memory for every block instead of being held in 32 registers: the
     // compiler spends those on fragment prefetch (dense, 40 rows: 3.11 -> 3.37 TB/s); with
     // four warps per slab the same change loses 3 %.
-    constexpr bool kQReload = (WPM == 2);
     uint32_t qf[8][4];
-    ok = mbar_wait(&sh.q_full, seg & 1u, &sh.abort_flag);
+    if (kDirectQ && seg == 0) {
+      // First query block of the CTA: every consumer warp copies the 16 rows of its own slab
+      // itself (the four warps of a slab write the same bytes), straight after its wait for
+      // the previous kernel -- the queries are the one input that kernel may have produced.
+      // Going through the producer warp (which first issues its K/V tile, then waits, then
+      // starts a bulk copy) put ~2.5 us between the previous launch's end and the first product.
+      for (int i = lane; i < 16 * 16; i += 32) {
+        const int r = mt * 16 + (i >> 4), c = i & 15;
+        if (r < P.M) {
+          const int t = r / P.grp, h = kvh * P.grp + r % P.grp;
+          cp_async16(smem_u32(sh.q) + r * kPitch + c * 16,
+                     P.q + ((static_cast<long long>(b) * P.T + t) * P.Hq + h) * kD + c * 8);
+        }
+      }
+      asm volatile("cp.async.wait_all;" ::: "memory");
+      __syncwarp();
+      ok = true;
+    } else {
+      ok = mbar_wait(&sh.q_full, seg & 1u, &sh.abort_flag);
+    }
     if (!ok) sh.abort_flag = 1;
     if (!kQReload) {
 #pragma unroll
