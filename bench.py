@@ -394,7 +394,7 @@ def select_variants(step, cfg, reps=5):
     return out
 
 
-def verify_micro(dev, reps=10, flags=0):
+def verify_micro(dev, reps=10, flags=0, only=""):
     """sparse_verify alone on synthetic shapes: dense long context and sparse lists of several
     lengths (shuffled block table, page 16).  Returns {case: {us, gbs}}; bytes = K/V rows read."""
     import torch
@@ -413,6 +413,8 @@ def verify_micro(dev, reps=10, flags=0):
              ("tokens12288_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, 12288),
              ("chunks768x16_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, -768)]
     for name, B, L, T, Hq, Hkv, count in cases:
+        if only and name != only:
+            continue
         page = 16
         pps = (L + page - 1) // page
         kv = wl.kv_pool(9, 0, B * pps, page, Hkv, 128, device=dev)
@@ -620,6 +622,7 @@ def main():
     ap.add_argument("--topp-sweep", action="store_true", help="(default on) the 256-row selection micro-benchmark of config 2")
     ap.add_argument("--no-topp-sweep", action="store_true", help="skip the selection micro-benchmark")
     ap.add_argument("--verify-micro", action="store_true", help="only run the sparse_verify micro-benchmark")
+    ap.add_argument("--verify-case", default="", help="with --verify-micro: run only the case of this name")
     ap.add_argument("--verify-engine", default="auto", choices=["auto", "mma_sync", "tcgen05"],
                     help="force one implementation of sparse_verify (default: the library picks by shape)")
     ap.add_argument("--long-context", action="store_true", help="only run the config-4 (ctx 131072) measurements")
@@ -659,7 +662,8 @@ def main():
 
     vflags = {"auto": 0, "mma_sync": sa.VERIFY_ENGINE_MMA_SYNC, "tcgen05": sa.VERIFY_ENGINE_TCGEN05}[args.verify_engine]
     if args.verify_micro:
-        print(json.dumps({"verify_micro": verify_micro(dev, reps=min(10, max(2, args.steps)), flags=vflags),
+        print(json.dumps({"verify_micro": verify_micro(dev, reps=min(10, max(2, args.steps)), flags=vflags,
+                                                       only=args.verify_case),
                           "engine": args.verify_engine}))
         return
 
