@@ -438,7 +438,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   const int warp = tid >> 5;
   const int U = P.B * P.Hkv;
   constexpr bool kQReload = (WPM == 2);   // query fragments re-read from shared memory per block
-  constexpr bool kDirectQ = !kQReload;    // consumers fetch the CTA's first query block themselves
+  constexpr bool kDirectQ = true;         // consumers fetch the CTA's first query block themselves
 
   // Unless the caller vouched for the lists, nothing is read before the previous kernel is
   // done.  Only then may the next kernel of the stream be scheduled: a successor that starts
@@ -816,7 +816,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     uint32_t qf[8][4];
     if (kDirectQ && seg == 0) {
       // First query block of the CTA: every consumer warp copies the 16 rows of its own slab
-      // itself (the four warps of a slab write the same bytes), straight after its wait for
+      // itself (the warps of a slab write the same bytes), straight after its wait for
       // the previous kernel -- the queries are the one input that kernel may have produced.
       // Going through the producer warp (which first issues its K/V tile, then waits, then
       // starts a bulk copy) put ~2.5 us between the previous launch's end and the first product.
