@@ -1443,7 +1443,9 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   // (a single-row list keeps nothing but the 32 KB of scan arrays behind the fixed part)
   const size_t smem = fixed + slice_bytes +
                       (P.single_row ? static_cast<size_t>(32 * 1024) : static_cast<size_t>(specattn::kRingFloats) * sizeof(float)) +
-                      (P.per_step ? static_cast<size_t>(specattn::kSliceCap / 8) : 0);  // the union's bit mask
+                      // the union's bit mask: one bit per position of the slice (sized to the slice, not
+                      // to the largest one: with 3 KB for it two CTAs no longer fitted an SM on 32k rows)
+                      (P.per_step ? static_cast<size_t>((slice + 127) / 128 * 16) : 0);
   if (smem > 224 * 1024) return SPECATTN_ERR_UNSUPPORTED;
   // Opt in to large dynamic shared memory once per device, so that later calls issue nothing
   // but the launch.
