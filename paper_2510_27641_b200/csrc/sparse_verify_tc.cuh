@@ -334,9 +334,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
 
   const bool is_softmax = warp < 8;
   const bool is_mma = (warp == kTcMmaWarp);
-  if (is_softmax) {
-    // the only warps that write global memory: the previous kernel is complete from here on
-    if (P.lists_stable) pdl_wait();
+  // The softmax warps are the only ones that write global memory; with SPECATTN_VERIFY_LISTS_STABLE
+  // they wait for the previous kernel here.  (For a CTA that gets work this comes after the
+  // tensor-memory allocation and the barrier behind it: the producers must not be held up by
+  // that wait -- their copies are what may run under the previous kernel.)
+  auto wait_and_clear_empty_units = [&]() {
+    if (P.lists_stable) pdl_wait();  // (otherwise the whole kernel has waited at its start)
     // units with an empty list: out = 0, lse = -inf
     for (int u = blockIdx.x; u < U; u += gridDim.x) {
       if (unit_count(P, u) != 0) continue;
@@ -347,8 +350,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         if (e % kD == 0) P.lse[(static_cast<long long>(b) * P.T + t) * P.Hq + h] = -INFINITY;
       }
     }
+  };
+  if (is_softmax && !P.lists_stable) wait_and_clear_empty_units();  // nothing to wait for: do it now
+  if (static_cast<long long>(blockIdx.x) >= NP) {
+    if (is_softmax && P.lists_stable) wait_and_clear_empty_units();
+    return;
   }
-  if (static_cast<long long>(blockIdx.x) >= NP) return;
   int a0, a1;
   if (aligned) {
     int lo = 0, hi = U - 1;
@@ -388,6 +395,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
   tc_fence_after();
   const uint32_t tmem = sh.tmem_base;
   const uint32_t col_o = tmem + 2u * N;  // 2 N columns: the P_hi part, then the P_lo part
+  if (is_softmax && P.lists_stable) wait_and_clear_empty_units();
 
   auto next_unit = [&](int& a, int& u, int seg_hi, int ue) {
     a = seg_hi;
