@@ -139,7 +139,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------
-def build_step(cfg, dev, verify_flags=0, select_workspace=True):
+def build_step(cfg, dev, verify_flags=0, select_workspace=True, select_form=0):
     import torch
     import workloads as wl
     from paper_2510_27641_b200.step import VerifyStep
@@ -156,7 +156,8 @@ def build_step(cfg, dev, verify_flags=0, select_workspace=True):
                       n_q_heads=cfg.n_q_heads, p=cfg.p, kv_pools=pools,
                       kv_len=torch.from_numpy(si.kv_len).to(dev),
                       block_table=None if si.block_table is None else torch.from_numpy(si.block_table).to(dev),
-                      pages_per_seq=si.pages_per_seq, verify_flags=verify_flags, select_workspace=select_workspace)
+                      pages_per_seq=si.pages_per_seq, verify_flags=verify_flags, select_workspace=select_workspace,
+                      select_form=select_form)
     dp_host = [None if x is None else torch.from_numpy(x).pin_memory() for x in si.draft_probs]
     q_host = [bf16.bits_to_torch(q).pin_memory() for q in si.q]
     step.load_inputs(dp_host, q_host)
@@ -498,7 +499,7 @@ def layer_batched(step, cfg, si, reps=20):
             "note": "upper bound: layers treated as independent; the per-layer launches are the result"}
 
 
-def config_section(cfg, dev, copies, reps=20):
+def config_section(cfg, dev, copies, reps=20, select_form=0):
     """One whole step (select + plans + verify per target layer) of a small configuration, timed
     as a CUDA graph over `copies` independent copies of ALL its inputs (draft rows, K/V pools,
     queries), one step per copy in turn, so that every step reads data that is not in L2
@@ -506,7 +507,7 @@ def config_section(cfg, dev, copies, reps=20):
     holds).  Bytes are the algorithmic ones of select and verify."""
     import torch
     peak = _measured_peaks()[0]
-    built = [build_step(cfg, dev) for _ in range(copies)]
+    built = [build_step(cfg, dev, select_form=select_form) for _ in range(copies)]
     si, _, step0, _, _ = built[0]
     steps = [b[2] for b in built]
     for st in steps:
@@ -817,7 +818,9 @@ def main():
         # all inputs keep every step's reads out of L2; config 3 reads more than L2 per step
         extra("config0", lambda: config_section(wl.config0(), dev, copies=64))
         torch.cuda.empty_cache()
-        extra("config3", lambda: config_section(wl.config3(), dev, copies=1))
+        # (a ragged batch: the caller knows it and asks for the selection's two-launch form)
+        extra("config3", lambda: config_section(wl.config3(), dev, copies=1,
+                                                 select_form=sa.SELECT_FORM_TWO_LAUNCH))
         torch.cuda.empty_cache()
     if rank == 0 and not args.no_long_context:
         extra("long_context", lambda: long_context(dev, n_layers=args.long_context_layers or long_context_layers(dev)))

@@ -115,7 +115,20 @@ extern "C" {
  * so a[] has the same bits -- into the workspace, and the search then reads a[] from there; the
  * lists are the same, the GPU is filled whatever the number of lists.  The workspace holds no
  * state between calls; two calls that may overlap on the GPU need separate workspaces.
+ *
+ * form: which of the two the call takes when both apply (a workspace is given, default selection,
+ * multi-row lists of >= 2048 positions).  SPECATTN_SELECT_FORM_AUTO decides by what the host
+ * can see (the number of lists).  What it cannot see is kv_len: in a ragged batch one cluster per
+ * list means the longest list sets the time while most of the GPU is done, and the two-launch
+ * form, whose first launch spends CTAs in proportion to each list's length, is the better one --
+ * a caller that knows its batch is ragged says SPECATTN_SELECT_FORM_TWO_LAUNCH
+ * (specattn_select_workspace_bytes then answers for that form).  SPECATTN_SELECT_FORM_CLUSTER
+ * keeps one launch.  The lists are the same bits in every form.
  * ======================================================================================== */
+#define SPECATTN_SELECT_FORM_AUTO 0
+#define SPECATTN_SELECT_FORM_CLUSTER 1
+#define SPECATTN_SELECT_FORM_TWO_LAUNCH 2
+
 typedef struct specattn_select_args {
   uint32_t struct_size;
   int32_t n_draft_layers;
@@ -141,7 +154,7 @@ typedef struct specattn_select_args {
   int32_t per_step;     /* 0 | 1 */
   int32_t bisect_iters; /* 0 = exact threshold, else 1..64 */
   int32_t chunk;        /* 0 | 1 = per position, else 4, 8, 16, 32 or 64 */
-  int32_t reserved;     /* 0 */
+  int32_t form;         /* SPECATTN_SELECT_FORM_*: 0 = the library picks */
   void* workspace;          /* device, or NULL */
   uint64_t workspace_bytes; /* size of *workspace */
 } specattn_select_args;

@@ -17,7 +17,8 @@ __all__ = ["select_topp", "sparse_verify", "sparse_verify_static", "verify_works
            "SelectArgs", "VerifyArgs", "StepHostArgs", "lib", "SpecAttnError",
            "ROW_OK", "ROW_INVALID_PROB", "ROW_OVERFLOW", "ROW_BAD_INDEX", "ROW_TIMEOUT",
            "VERIFY_LISTS_STABLE", "VERIFY_ENGINE_MMA_SYNC", "VERIFY_ENGINE_TCGEN05",
-           "VERIFY_TEST_LOSE_ARRIVAL", "VERIFY_PAGE_LISTS", "verify_plan",
+           "VERIFY_TEST_LOSE_ARRIVAL", "VERIFY_PAGE_LISTS", "SELECT_FORM_AUTO", "SELECT_FORM_CLUSTER",
+           "SELECT_FORM_TWO_LAUNCH", "verify_plan",
            "verify_plan_buffer", "verify_plan_many"]
 
 ROW_OK, ROW_INVALID_PROB, ROW_OVERFLOW, ROW_BAD_INDEX, ROW_TIMEOUT = 0, 1, 2, 4, 8
@@ -25,6 +26,7 @@ VERIFY_LISTS_STABLE = 1
 VERIFY_ENGINE_MMA_SYNC = 2
 VERIFY_ENGINE_TCGEN05 = 4
 VERIFY_PAGE_LISTS = 8
+SELECT_FORM_AUTO, SELECT_FORM_CLUSTER, SELECT_FORM_TWO_LAUNCH = 0, 1, 2
 VERIFY_TEST_LOSE_ARRIVAL = 0x80000000   # test only: see include/specattn.h
 
 _LIB_PATH = Path(__file__).resolve().parent / "libspecattn.so"
@@ -46,7 +48,7 @@ class SelectArgs(C.Structure):
                 ("p", C.c_float), ("idx", C.c_void_p), ("idx_stride", C.c_int64),
                 ("counts", C.c_void_p), ("row_status", C.c_void_p), ("diag", C.c_void_p),
                 ("per_step", C.c_int32), ("bisect_iters", C.c_int32), ("chunk", C.c_int32),
-                ("reserved", C.c_int32), ("workspace", C.c_void_p), ("workspace_bytes", C.c_uint64)]
+                ("form", C.c_int32), ("workspace", C.c_void_p), ("workspace_bytes", C.c_uint64)]
 
 
 class VerifyArgs(C.Structure):
@@ -134,7 +136,7 @@ def make_select_args(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.T
                      head_group: Sequence[int] | None = None, idx: torch.Tensor,
                      counts: torch.Tensor, row_status: torch.Tensor,
                      diag: torch.Tensor | None = None, per_step: bool = False, bisect_iters: int = 0,
-                     chunk: int = 1, workspace: torch.Tensor | bool | None = True):
+                     chunk: int = 1, workspace: torch.Tensor | bool | None = True, form: int = 0):
     """Fills a SelectArgs.  Returns (args, keepalive) -- keepalive holds the host arrays the
     struct points at and must outlive the call.  workspace: a uint8 CUDA tensor, True (allocate
     what specattn_select_workspace_bytes asks for, if anything) or None / False (none: the
@@ -163,6 +165,7 @@ def make_select_args(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.T
     a.counts, a.row_status = counts.data_ptr(), row_status.data_ptr()
     a.diag = None if diag is None else diag.data_ptr()
     a.per_step, a.bisect_iters, a.chunk = int(bool(per_step)), int(bisect_iters), int(chunk)
+    a.form = int(form)
     if workspace is True:
         need = int(lib().specattn_select_workspace_bytes(C.byref(a)))
         workspace = torch.empty((need,), dtype=torch.uint8, device=ref.device) if need > 0 else None
@@ -180,7 +183,7 @@ def select_topp(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.Tensor
                 idx: torch.Tensor | None = None, counts: torch.Tensor | None = None,
                 row_status: torch.Tensor | None = None, diag: torch.Tensor | None = None,
                 want_diag: bool = False, per_step: bool = False, bisect_iters: int = 0, chunk: int = 1,
-                workspace: torch.Tensor | bool | None = True, stream=None):
+                workspace: torch.Tensor | bool | None = True, form: int = 0, stream=None):
     """specattn_select_topp.  draft_probs: per draft layer a float32 CUDA tensor
     [B, H_d, gamma, L_stride] (None for layers no target layer maps to).  Returns
     (idx [n_d,B,G,idx_stride] int32, counts [n_d,B,G], row_status [n_d,B,G], diag or None)."""
@@ -200,7 +203,7 @@ def select_topp(draft_probs: Sequence[torch.Tensor | None], kv_len: torch.Tensor
     args, keep = make_select_args(draft_probs, kv_len, layer_map, p, n_groups=n_groups,
                                   head_group=head_group, idx=idx, counts=counts,
                                   row_status=row_status, diag=diag, per_step=per_step,
-                                  bisect_iters=bisect_iters, chunk=chunk, workspace=workspace)
+                                  bisect_iters=bisect_iters, chunk=chunk, workspace=workspace, form=form)
     rc = lib().specattn_select_topp(C.byref(args), _stream_ptr(stream))
     if rc != 0:
         raise SpecAttnError(rc, "specattn_select_topp")

@@ -1325,7 +1325,9 @@ bool two_launch_shape(const specattn_select_args& A) {
   if (variant || static_cast<long long>(A.n_draft_heads) * A.gamma <= 1 || A.L_stride < 2048 || A.L_stride % 4 != 0)
     return false;
   const long long n_lists = count_lists(A);
-  return n_lists > 0 && n_lists * pick_cluster(A.L_stride, n_lists) < 148;
+  if (n_lists <= 0 || A.form == SPECATTN_SELECT_FORM_CLUSTER) return false;
+  if (A.form == SPECATTN_SELECT_FORM_TWO_LAUNCH) return true;  // the caller knows its batch (ragged lengths)
+  return n_lists * pick_cluster(A.L_stride, n_lists) < 148;
 }
 
 }  // namespace
@@ -1351,6 +1353,7 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
   if (A.L_stride < 0 || A.idx_stride < 0) return SPECATTN_ERR_RANGE;
   if (!(A.p > 0.0f)) return SPECATTN_ERR_RANGE;  // also rejects NaN
   if (A.bisect_iters < 0 || A.bisect_iters > 64 || (A.per_step != 0 && A.per_step != 1)) return SPECATTN_ERR_RANGE;
+  if (A.form < 0 || A.form > SPECATTN_SELECT_FORM_TWO_LAUNCH) return SPECATTN_ERR_RANGE;
   if (A.chunk < 0 || A.chunk > 64 || (A.chunk > 1 && (A.chunk < 4 || (A.chunk & (A.chunk - 1)) != 0)))
     return SPECATTN_ERR_RANGE;  // 0 / 1 = per position, else a power of two in [4, 64]
   if (A.L_stride % 4 != 0) return SPECATTN_ERR_ALIGN;

@@ -24,7 +24,7 @@ class VerifyStep:
                  block_table: torch.Tensor | None, pages_per_seq: int | None = None,
                  n_groups: int = 1, head_group: Sequence[int] | None = None,
                  idx_stride: int | None = None, sm_scale: float = 0.0, verify_flags: int = 0,
-                 use_plans: bool = True, select_workspace: bool = True, device=None):
+                 use_plans: bool = True, select_workspace: bool = True, select_form: int = 0, device=None):
         dev = device or kv_pools[0].device
         self.layer_map = [int(x) for x in layer_map]
         self.n_layers = len(self.layer_map)
@@ -50,7 +50,7 @@ class VerifyStep:
             self.select_args, self._keep = make_select_args(
                 self.draft_probs, kv_len, self.layer_map, p, n_groups=n_groups, head_group=head_group,
                 idx=self.idx, counts=self.counts, row_status=self.row_status, diag=self.diag,
-                workspace=select_workspace)
+                workspace=select_workspace, form=select_form)
         self.verify_args: list[VerifyArgs] = []
         self.workspace = None
         self.plans: dict[int, tuple[torch.Tensor, int]] = {}   # draft layer (-1: dense) -> (plan, a layer using it)

@@ -112,6 +112,10 @@ def test_select_workspace_query_follows_the_documented_rule(sa):
     assert need(1, 4, 1, 1, 131072) == 0                           # single-row lists are read in place
     assert need(1, 4, 16, 4, 1024) == 0                            # short rows
     assert need(1, 4, 16, 4, 131072, per_step=1) == 0              # variants keep the cluster form
+    # the caller's choice of form: two launches whatever the number of lists, or never
+    assert need(32, 8, 12, 5, 32768, form=2) == 32 * 32768 * 4
+    assert need(1, 4, 16, 4, 131072, form=1) == 0
+    assert need(1, 4, 1, 1, 131072, form=2) == 0                   # single-row lists have nothing to sum
     assert need(1, 4, 16, 4, 131072, chunk=16) == 0
     assert need(1, 4, 16, 4, 131072, bisect_iters=10) == 0
     assert L.specattn_select_workspace_bytes(None) == 0
