@@ -66,8 +66,10 @@ class VerifyStep:
             if self.workspace is None:
                 self.workspace = verify_workspace(a, dev)
             a.workspace, a.workspace_bytes = self.workspace.data_ptr(), self.workspace.numel()
-            # target layers that share a draft layer's lists (or are dense) share a work partition
-            if use_plans:
+            # target layers that share a draft layer's lists (or are dense) share a work partition;
+            # a list set that a single layer uses is cheaper partitioned by that layer's own launch
+            # than by a plan launch in front of it
+            if use_plans and self.layer_map.count(u) > 1:
                 if u not in self.plans:
                     self.plans[u] = (verify_plan_buffer(a, dev), j)
                 a.plan = self.plans[u][0].data_ptr()
