@@ -1432,7 +1432,7 @@ extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda
     cs = 1;
     while (cs < 8 && (A.L_stride + cs - 1) / cs > 65536) cs *= 2;
     while (cs < 8 && n_lists * cs < 296 && (A.L_stride + cs - 1) / cs > 16384) cs *= 2;
-    while (cs < 8 && n_lists * cs < 148) cs *= 2;
+    while (cs < 8 && n_lists * cs < 148 && (A.L_stride + cs - 1) / cs > 2048) cs *= 2;  // (short rows: fewer cluster barriers beat more CTAs)
   }
   const long long s_align = (P.chunk > 4) ? P.chunk : 4;
   const long long slice = P.single_row ? 0 : (((A.L_stride + cs - 1) / cs) + s_align - 1) / s_align * s_align;

@@ -56,6 +56,10 @@ constexpr int kRec = 68 * 32;  // floats of one warp's (acc[64], m0, l0, m1, l1)
 constexpr int kCountersPerUnit = 4;
 constexpr int kAlignedMaxUnits = 256;  // the unit-aligned partition is tried up to this many units
 constexpr int kCandidates = 8;         // candidate target shares tried for it
+// A unit is not cut into parts of fewer than this many atoms (two 64-token tiles) even when
+// there are CTAs to spare: every part costs a record, an arrival and a share of the merge, which
+// on a small call (one short sequence) outweighs the streaming time saved.
+constexpr int kMinPartAtoms = 8;
 constexpr size_t kCounterBytes = static_cast<size_t>(kMaxUnits) * kCountersPerUnit * sizeof(unsigned int);
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -200,6 +204,7 @@ __device__ __forceinline__ void plan_body(const VerifyParams& P, int* plan, int 
         int k = static_cast<int>((2u * num + den) / (2u * den));
         if (k < 1) k = 1;
         if (k > atoms) k = atoms;
+        if (k * kMinPartAtoms > atoms) k = max(1, atoms / kMinPartAtoms);  // no part shorter than that
         atomicAdd(&cand_parts[c], k);
         atomicMax(&cand_max[c], (atoms + k - 1) / k);
       }
@@ -226,6 +231,7 @@ __device__ __forceinline__ void plan_body(const VerifyParams& P, int* plan, int 
           k = static_cast<int>((2u * num + den) / (2u * den));
           if (k < 1) k = 1;
           if (k > atoms) k = atoms;
+        if (k * kMinPartAtoms > atoms) k = max(1, atoms / kMinPartAtoms);  // no part shorter than that
         }
       }
       int v = k;
@@ -545,6 +551,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         int k = static_cast<int>((2u * num + den) / (2u * den));  // round to nearest
         if (k < 1) k = 1;
         if (k > atoms) k = atoms;
+        if (k * kMinPartAtoms > atoms) k = max(1, atoms / kMinPartAtoms);  // no part shorter than that
         atomicAdd(&sh.cand_parts[c], k);
         atomicMax(&sh.cand_max[c], (atoms + k - 1) / k);
       }
@@ -573,6 +580,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           k = static_cast<int>((2u * num + den) / (2u * den));
           if (k < 1) k = 1;
           if (k > atoms) k = atoms;
+        if (k * kMinPartAtoms > atoms) k = max(1, atoms / kMinPartAtoms);  // no part shorter than that
         }
       }
       int v = k;

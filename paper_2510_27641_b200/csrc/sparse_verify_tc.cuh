@@ -290,6 +290,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
         int k = static_cast<int>((2 * num + den) / (2 * den));
         if (k < 1) k = 1;
         if (k > atoms) k = atoms;
+        if (k * kMinPartAtoms > atoms) k = max(1, atoms / kMinPartAtoms);  // no part shorter than that
         atomicAdd(&sh.cand_parts[c], k);
         atomicMax(&sh.cand_max[c], (atoms + k - 1) / k);
       }
@@ -316,6 +317,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) sparse_verify_tc_kernel(const _
           k = static_cast<int>((2 * num + den) / (2 * den));
           if (k < 1) k = 1;
           if (k > atoms) k = atoms;
+        if (k * kMinPartAtoms > atoms) k = max(1, atoms / kMinPartAtoms);  // no part shorter than that
         }
       }
       int v = k;
