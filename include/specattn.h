@@ -21,6 +21,9 @@
  *     code never traps.
  *   - `struct_size` must be sizeof() of the struct the caller was compiled against.
  *   - Strides are in ELEMENTS of the array they index.
+ *   - Tracing: specattn_select_topp, specattn_sparse_verify, specattn_verify_plan(_many) and
+ *     specattn_verify_step_host each open an NVTX range of their own name around their host-side
+ *     work (visible in a profiler's timeline; a null-pointer test when no tool is attached).
  */
 #ifndef SPECATTN_H_
 #define SPECATTN_H_

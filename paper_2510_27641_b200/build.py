@@ -20,7 +20,7 @@ FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std
 
 
 def _headers() -> list[Path]:
-    return list(CSRC.glob("*.cuh")) + list(INCLUDE.glob("*.h"))
+    return list(CSRC.glob("*.cuh")) + list(CSRC.glob("*.h")) + list(INCLUDE.glob("*.h"))
 
 
 def _stale(target: Path, deps: list[Path]) -> bool:
@@ -46,7 +46,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     with ThreadPoolExecutor(len(SOURCES)) as pool:
         objs = list(pool.map(compile_one, SOURCES))
     subprocess.run(["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-Xcompiler", "-fPIC",
-                    *[str(o) for o in objs], "-o", str(LIB)], check=True)
+                    *[str(o) for o in objs], "-ldl", "-o", str(LIB)], check=True)
     return LIB
 
 

@@ -10,6 +10,7 @@
 #include <new>
 
 #include "specattn.h"
+#include "nvtx_range.h"
 
 namespace specattn {
 
@@ -125,6 +126,7 @@ bool prepare_pipe(HostPipe& pipe, int n_target_layers) {
 // call returns with everything enqueued; the caller's stream has been made to wait for the last
 // download, so stream order is what it would be had everything run on that stream.
 extern "C" int specattn_verify_step_host(const specattn_step_host_args* args, void* cuda_stream) {
+  specattn::NvtxRange nvtx_range("specattn_verify_step_host");
   if (args == nullptr) return SPECATTN_ERR_NULL;
   if (args->struct_size != sizeof(specattn_step_host_args)) return SPECATTN_ERR_STRUCT_SIZE;
   const specattn_step_host_args& S = *args;

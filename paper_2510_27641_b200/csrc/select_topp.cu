@@ -48,6 +48,7 @@
 #include <atomic>
 
 #include "ptx.cuh"
+#include "nvtx_range.h"
 #include "specattn.h"
 
 namespace cg = cooperative_groups;
@@ -1342,6 +1343,7 @@ extern "C" size_t specattn_select_workspace_bytes(const specattn_select_args* ar
 }
 
 extern "C" int specattn_select_topp(const specattn_select_args* args, void* cuda_stream) {
+  specattn::NvtxRange nvtx_range("specattn_select_topp");
   if (args == nullptr) return SPECATTN_ERR_NULL;
   if (args->struct_size != sizeof(specattn_select_args)) return SPECATTN_ERR_STRUCT_SIZE;
   const specattn_select_args& A = *args;

@@ -35,6 +35,7 @@
 #include <atomic>
 
 #include "ptx.cuh"
+#include "nvtx_range.h"
 #include "specattn.h"
 
 namespace specattn {
@@ -1273,6 +1274,7 @@ extern "C" int specattn_verify_workspace_init(void* workspace, size_t workspace_
 }
 
 extern "C" int specattn_sparse_verify(const specattn_verify_args* args, void* cuda_stream) {
+  specattn::NvtxRange nvtx_range("specattn_sparse_verify");
   const int v = specattn::validate(args);
   if (v != SPECATTN_OK) return v;
   const specattn_verify_args& A = *args;
@@ -1331,6 +1333,7 @@ extern "C" size_t specattn_verify_plan_bytes(const specattn_verify_args* args) {
 
 extern "C" int specattn_verify_plan(const specattn_verify_args* args, void* plan, size_t plan_bytes,
                                     void* cuda_stream) {
+  specattn::NvtxRange nvtx_range("specattn_verify_plan");
   const int v = specattn::validate(args);
   if (v != SPECATTN_OK) return v;
   const specattn_verify_args& A = *args;
@@ -1362,6 +1365,7 @@ extern "C" int specattn_verify_plan(const specattn_verify_args* args, void* plan
 
 extern "C" int specattn_verify_plan_many(const specattn_verify_args* const* args, void* const* plans,
                                          const size_t* plan_bytes, int32_t n, void* cuda_stream) {
+  specattn::NvtxRange nvtx_range("specattn_verify_plan_many");
   if (n < 0) return SPECATTN_ERR_RANGE;
   if (n == 0) return SPECATTN_OK;
   if (args == nullptr || plans == nullptr || plan_bytes == nullptr) return SPECATTN_ERR_NULL;
