@@ -291,6 +291,16 @@ class OracleSample:
         return (t_sel + t_attn * scale) * 1e6, sample
 
 
+def config_dict(cfg, world: int):
+    """The `config` object of the JSON line: the same for both arms (--impl ours / reference)."""
+    return {"workload": cfg.name, "n_target_layers": cfg.n_target_layers,
+            "n_draft_layers": cfg.n_draft_layers, "batch_per_gpu": cfg.batch,
+            "global_batch": cfg.batch * world, "ctx": cfg.ctx, "page_size": cfg.page_size,
+            "gamma": cfg.gamma, "p": cfg.p, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
+            "head_dim": cfg.head_dim, "parallelism": f"batch-sharded x{world}, no collective",
+            "l2": "inputs exceed L2: 252 MB of draft rows and 1.3 GB of gathered K/V per step"}
+
+
 def run_reference(args, cfg):
     import workloads as wl
     rank, _, world = _rank_env()
@@ -308,11 +318,7 @@ def run_reference(args, cfg):
     line = {"impl": "reference", "metric": METRIC, "value": round(v, 1), "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(v / 1e3, 3), "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "n_target_layers": cfg.n_target_layers,
-                       "n_draft_layers": cfg.n_draft_layers, "batch_per_gpu": cfg.batch,
-                       "global_batch": cfg.batch, "ctx": cfg.ctx, "page_size": cfg.page_size,
-                       "gamma": cfg.gamma, "p": cfg.p, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
-                       "head_dim": cfg.head_dim},
+            "config": config_dict(cfg, max(1, args.gpus)),
             "cpu_baseline": {"value": round(v, 1), "unit": UNIT, "cores": smp.cores, "kind": "oracle",
                              "sample": sample + f"; wall {time.perf_counter() - t_start:.1f} s for all steps"},
             "e2e": {"value": round(v, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -761,17 +767,12 @@ def main():
     line = {"metric": METRIC, "value": round(us_step, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(us_step / 1e3, 6), "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": cfg.name, "n_target_layers": cfg.n_target_layers,
-                       "n_draft_layers": cfg.n_draft_layers, "batch_per_gpu": cfg.batch,
-                       "global_batch": cfg.batch * world, "ctx": cfg.ctx, "page_size": cfg.page_size,
-                       "gamma": cfg.gamma, "p": cfg.p, "q_heads": cfg.n_q_heads, "kv_heads": cfg.n_kv_heads,
-                       "head_dim": cfg.head_dim, "parallelism": f"batch-sharded x{world}, no collective",
-                       "launch": f"CUDA graph of 1 select + 1 plan launch ({len(step.plans)} plans) + {step.n_layers} verify launches",
-                       "l2": "inputs exceed L2: 252 MB of draft rows and 1.3 GB of gathered K/V per step"},
+            "config": config_dict(cfg, world),
             "e2e": {"value": round(us_e2e, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(n_step * args.steps),
             "clocks": clocks, "roofline": roofline,
-            "extra": {"us_step_batches": step_stats, "us_verify_per_step": round(us_verify_all, 3), "us_select_per_step": round(us_select, 3),
+            "extra": {"launch": f"CUDA graph of 1 select + 1 plan launch ({len(step.plans)} plans) + {step.n_layers} verify launches",
+                      "us_step_batches": step_stats, "us_verify_per_step": round(us_verify_all, 3), "us_select_per_step": round(us_select, 3),
                       "us_step_eager_launches": round(us_eager, 3),
                       "topp_lists_per_s": round(n_used * cfg.batch / us_select * 1e6),
                       "topp_prob_rows_per_s": round(n_used * cfg.batch * cfg.n_draft_heads * cfg.gamma / us_select * 1e6),
