@@ -385,6 +385,9 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     return in_place ? __float_as_uint(__ldg(A + i) + 0.f) : __float_as_uint(a[i]);
   };
   const int n4 = (n_loc + 3) >> 2;
+  // (rows read in place) float4s in whole iterations of the CTA whose values all lie inside the
+  // slice: the lean bodies of the passes cover [0, n4_main), the general ones the rest
+  const int n4_main = ((n_loc >> 2) / (4 * kThreads)) * (4 * kThreads);
   // In-place passes read the row from global memory (L2) with four independent 16-byte loads per
   // thread in flight: with one dependent load per iteration a CTA moved ~4 GB/s (latency-bound);
   // eight in flight were 3-4 % slower on 64k / 128k rows than four (twice the code per pass), two
@@ -461,8 +464,63 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   // ---- 1+2: aggregate the slice and build the level-1 histogram ------------------------------
   bool bad = false;
   if (in_place) {
-    // single contributing row: one pass over the slice for validity and the level-1 histogram
-    for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
+    // single contributing row: one pass over the slice for validity and the level-1 histogram.
+    // The pass is bound by instruction issue, so whole iterations (every float4 of the CTA inside
+    // the slice and complete: all but the last one or two) run a lean body: validity through a
+    // running maximum of the bit patterns (a negative, NaN or infinite value is a pattern above
+    // 0x7f7fffff), no bounds tests, and the test "does the whole warp hit one bin" (ties) once
+    // per 16 values of a thread instead of once per 4.
+    int ip_main = 0;
+    if (!kVariant) {
+      unsigned int kbits = 0u;
+      for (; ip_main < n4_main; ip_main += kIpUnroll * kThreads) {
+        float4 v[kIpUnroll];
+#pragma unroll
+        for (int uu = 0; uu < kIpUnroll; ++uu)
+          v[uu] = __ldg(reinterpret_cast<const float4*>(A) + ip_main + uu * kThreads + tid);
+        unsigned int k[kIpUnroll * 4];
+        unsigned int k_or = 0u, k_and = 0xffffffffu;
+#pragma unroll
+        for (int uu = 0; uu < kIpUnroll; ++uu) {
+          k[4 * uu + 0] = __float_as_uint(v[uu].x + 0.f);  // -0.0 reads as +0.0
+          k[4 * uu + 1] = __float_as_uint(v[uu].y + 0.f);
+          k[4 * uu + 2] = __float_as_uint(v[uu].z + 0.f);
+          k[4 * uu + 3] = __float_as_uint(v[uu].w + 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < kIpUnroll * 4; ++j) {
+          kbits = max(kbits, k[j]);
+          k_or |= k[j];
+          k_and &= k[j];
+        }
+        // all 16 values of this thread in one bin, and the same bin in every lane: one reduction
+        // per word for the warp (zeros can only share bin 0, where they add nothing)
+        const unsigned int my_bin = k[0] >> 20;
+        const bool mine_same = ((k_or ^ k_and) >> 20) == 0u && !(k_or >> 31);  // (a set sign bit: invalid input)
+        const unsigned int bin0 = __shfl_sync(kFull, my_bin, 0);  // (every lane takes part: not inside the &&)
+        if (__all_sync(kFull, mine_same && my_bin == bin0)) {
+          unsigned int lo = 0u, hi = 0u;
+#pragma unroll
+          for (int j = 0; j < kIpUnroll * 4; ++j) {
+            const unsigned int m = mantissa_of(k[j]);
+            lo += m & 0xffffu;
+            hi += m >> 16;
+          }
+          lo = __reduce_add_sync(kFull, lo);
+          hi = __reduce_add_sync(kFull, hi);
+          if (lane == 0) hist_bump(h1, static_cast<int>(my_bin), lo, hi);
+        } else {
+#pragma unroll
+          for (int j = 0; j < kIpUnroll * 4; ++j) {
+            const unsigned int m = mantissa_of(k[j]);
+            if (k[j] != 0u && !(k[j] >> 31)) hist_bump(h1, static_cast<int>(k[j] >> 20), m & 0xffffu, m >> 16);
+          }
+        }
+      }
+      bad |= kbits > 0x7f7fffffu;
+    }
+    // the rest of the slice (and everything, for the variants): bounds and validity per value
+    for (int base = ip_main; base < n4; base += kIpUnroll * kThreads) {
       unsigned int key[kIpUnroll][4];
       bool act[kIpUnroll];
 #pragma unroll
