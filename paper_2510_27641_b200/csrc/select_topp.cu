@@ -801,7 +801,45 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     unsigned int* const lb2 = lvl_base;                                  // level-2 histogram
     const Hist hr = {lb2, lb2 + kL23Bins};
     unsigned int kmin = 0xffffffffu, kmax = 0u;
-    for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
+    // whole iterations: no bounds tests; the histogram is only touched for float4s in which some
+    // lane holds a value of the bin
+    int mp_main = 0;
+    for (; mp_main < n4_main; mp_main += kIpUnroll * kThreads) {
+      float4 v[kIpUnroll];
+#pragma unroll
+      for (int uu = 0; uu < kIpUnroll; ++uu)
+        v[uu] = __ldg(reinterpret_cast<const float4*>(A) + mp_main + uu * kThreads + tid);
+#pragma unroll
+      for (int uu = 0; uu < kIpUnroll; ++uu) {
+        const unsigned int k[4] = {__float_as_uint(v[uu].x + 0.f), __float_as_uint(v[uu].y + 0.f),
+                                   __float_as_uint(v[uu].z + 0.f), __float_as_uint(v[uu].w + 0.f)};
+        bool take[4];
+        bool any_in = false;
+        unsigned int mine = 0u;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const unsigned int top = k[e] >> 20;
+          take[e] = top == prefix;
+          any_in |= take[e];
+          const unsigned int m = __ballot_sync(kFull, top >= prefix);
+          if (lane == e) mine = m;
+        }
+        if (__any_sync(kFull, any_in)) {
+          int bin[4];
+          unsigned int mant[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            bin[e] = static_cast<int>((k[e] >> 10) & 1023u);
+            mant[e] = mantissa_of(k[e]);
+            kmin = take[e] ? min(kmin, k[e]) : kmin;
+            kmax = take[e] ? max(kmax, k[e]) : kmax;
+          }
+          hist_add4(hr, take, bin, mant);
+        }
+        if (lane < 4) keep_words[((mp_main + uu * kThreads + (tid & ~31)) >> 5) * 4 + lane] = mine;
+      }
+    }
+    for (int base = mp_main; base < n4; base += kIpUnroll * kThreads) {
       unsigned int key[kIpUnroll][4];
       bool act[kIpUnroll];
 #pragma unroll
@@ -893,7 +931,38 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
   }
   if (short_cut) {
     if (in_place) {
-        for (int base = 0; base < n4; base += kIpUnroll * kThreads) {
+      // whole iterations: no bounds tests, and the candidate list is only touched for float4s in
+      // which some lane holds a candidate (a few hundred per row)
+      int cp_main = 0;
+      for (; cp_main < n4_main; cp_main += kIpUnroll * kThreads) {
+        float4 v[kIpUnroll];
+#pragma unroll
+        for (int uu = 0; uu < kIpUnroll; ++uu)
+          v[uu] = __ldg(reinterpret_cast<const float4*>(A) + cp_main + uu * kThreads + tid);
+#pragma unroll
+        for (int uu = 0; uu < kIpUnroll; ++uu) {
+          const int i4 = cp_main + uu * kThreads + tid;
+          const unsigned int k[4] = {__float_as_uint(v[uu].x + 0.f), __float_as_uint(v[uu].y + 0.f),
+                                     __float_as_uint(v[uu].z + 0.f), __float_as_uint(v[uu].w + 0.f)};
+          bool is_cand[4];
+          bool any_cand = false;
+          unsigned int mine = 0u;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const unsigned int top = k[e] >> csh;
+            is_cand[e] = top == cpre;
+            any_cand |= is_cand[e];
+            const unsigned int m = __ballot_sync(kFull, top > cpre);
+            if (lane == e) mine = m;
+          }
+          if (__any_sync(kFull, any_cand)) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) cand_add(sh, is_cand[e], k[e], 4 * i4 + e);
+          }
+          if (lane < 4) keep_words[((cp_main + uu * kThreads + (tid & ~31)) >> 5) * 4 + lane] = mine;
+        }
+      }
+        for (int base = cp_main; base < n4; base += kIpUnroll * kThreads) {
           unsigned int key[kIpUnroll][4];
         bool act[kIpUnroll];
 #pragma unroll
