@@ -814,27 +814,40 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
         const unsigned int k[4] = {__float_as_uint(v[uu].x + 0.f), __float_as_uint(v[uu].y + 0.f),
                                    __float_as_uint(v[uu].z + 0.f), __float_as_uint(v[uu].w + 0.f)};
         bool take[4];
-        bool any_in = false;
+        bool all_in = true;
         unsigned int mine = 0u;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const unsigned int top = k[e] >> 20;
           take[e] = top == prefix;
-          any_in |= take[e];
+          all_in &= take[e];
           const unsigned int m = __ballot_sync(kFull, top >= prefix);
           if (lane == e) mine = m;
         }
-        if (__any_sync(kFull, any_in)) {
+        // Every value of the warp's 128 inside the bin (constant or near-constant rows): the tie
+        // test and the warp-wide reduction of hist_add4.  Otherwise the bin holds a few per cent
+        // of the values and each of them updates the histogram on its own.
+        if (__all_sync(kFull, all_in)) {
           int bin[4];
           unsigned int mant[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             bin[e] = static_cast<int>((k[e] >> 10) & 1023u);
             mant[e] = mantissa_of(k[e]);
-            kmin = take[e] ? min(kmin, k[e]) : kmin;
-            kmax = take[e] ? max(kmax, k[e]) : kmax;
+            kmin = min(kmin, k[e]);
+            kmax = max(kmax, k[e]);
           }
           hist_add4(hr, take, bin, mant);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            if (take[e]) {
+              const unsigned int m = mantissa_of(k[e]);
+              hist_bump(hr, static_cast<int>((k[e] >> 10) & 1023u), m & 0xffffu, m >> 16);
+              kmin = min(kmin, k[e]);
+              kmax = max(kmax, k[e]);
+            }
+          }
         }
         if (lane < 4) keep_words[((mp_main + uu * kThreads + (tid & ~31)) >> 5) * 4 + lane] = mine;
       }
