@@ -42,6 +42,7 @@
 #include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <float.h>
+#include <stddef.h>
 #include <stdint.h>
 #include <string.h>
 
@@ -1293,6 +1294,12 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
     int* out = P.idx + out_list * P.idx_stride;
     long long pos = offset + sh.warp_cnt[warp];
     const unsigned int lt = (1u << lane) - 1u;
+    // (the candidate arrays are idle by now -- every peer is past its gather -- and hold the
+    // eight warps' staging lines of 128 positions)
+    static_assert(offsetof(Shared, all_keys) - offsetof(Shared, cand) == 2 * kCandCap * sizeof(int) &&
+                      3 * kCandCap >= kWarps * 128,
+                  "the candidate arrays are contiguous and hold one staging line per warp");
+    int* const stage = reinterpret_cast<int*>(sh.cand) + warp * 128;
     __syncwarp();  // this warp's ballot words are complete
     for (int g4 = w4_lo; g4 < w4_hi; g4 += 32) {
       // 128 consecutive positions, four per lane: ascending order is lane-major
@@ -1305,14 +1312,18 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
         before += __popc(mw[e] & lt);
         total_kept += __popc(mw[e]);
       }
-      long long my = pos + before;
+      // The kept positions of the 128 go through a per-warp staging line, so that the global
+      // stores are whole 128-byte runs (a lane storing its own up to four positions spreads every
+      // store instruction over the whole 512-byte range: four partial writes per sector).
+      unsigned int at = before;
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        if ((mw[e] >> lane) & 1u) {
-          if (my < P.idx_stride) out[my] = lo + 4 * i4 + e;
-          ++my;
-        }
+        if ((mw[e] >> lane) & 1u) stage[at++] = lo + 4 * i4 + e;
       }
+      __syncwarp();
+      for (unsigned int t = lane; t < total_kept; t += 32)
+        if (pos + t < P.idx_stride) out[pos + t] = stage[t];
+      __syncwarp();
       pos += total_kept;
     }
   } else if (!invalid) {
