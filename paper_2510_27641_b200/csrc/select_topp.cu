@@ -1301,11 +1301,18 @@ __global__ void __launch_bounds__(kThreads, kInPlace ? 4 : 2) select_topp_kernel
                   "the candidate arrays are contiguous and hold one staging line per warp");
     int* const stage = reinterpret_cast<int*>(sh.cand) + warp * 128;
     __syncwarp();  // this warp's ballot words are complete
+    // one group of 128 positions per trip; the next group's ballot words are loaded before this
+    // one is worked on, and a group without a kept position (most groups of a peaked row) costs
+    // nothing more
+    uint4 words = (w4_lo < w4_hi) ? *reinterpret_cast<const uint4*>(keep_words + (w4_lo >> 5) * 4)
+                                  : make_uint4(0u, 0u, 0u, 0u);
     for (int g4 = w4_lo; g4 < w4_hi; g4 += 32) {
+      const uint4 cur = words;
+      if (g4 + 32 < w4_hi) words = *reinterpret_cast<const uint4*>(keep_words + ((g4 + 32) >> 5) * 4);
+      if ((cur.x | cur.y | cur.z | cur.w) == 0u) continue;  // (the same words in every lane)
       // 128 consecutive positions, four per lane: ascending order is lane-major
       const int i4 = g4 + lane;
-      const uint4 words = *reinterpret_cast<const uint4*>(keep_words + (g4 >> 5) * 4);
-      const unsigned int mw[4] = {words.x, words.y, words.z, words.w};
+      const unsigned int mw[4] = {cur.x, cur.y, cur.z, cur.w};
       unsigned int before = 0, total_kept = 0;
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
