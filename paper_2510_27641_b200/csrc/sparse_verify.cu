@@ -694,15 +694,22 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         if (!load_q()) { sh.abort_flag = 1; dead = true; break; }
       }
       // lane j resolves tokens j and j + 32 of a tile to the byte offset of their K row:
-      // list -> position -> block table -> page, two dependent loads
-      auto resolve = [&](int t0, long long (&off)[2]) -> bool {
+      // list -> position -> block table -> page, two dependent loads, in two steps so that a
+      // warp can keep the chain one tile of its own ahead (positions of its tile after next,
+      // offsets of its next tile): neither load is then waited for between two tiles
+      auto load_pos = [&](int t0, int (&pos)[2]) {
         const int ntok = min(kStageTok, tok_hi - t0);
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj) {
+          const int k = t0 + min(lane + jj * 32, ntok - 1);  // token index inside the unit: the list first, then the tail
+          pos[jj] = (k >= c_list) ? (kvlen_b + (k - c_list)) : (P.dense ? k : __ldg(list + k));
+        }
+      };
+      auto offs_of = [&](const int (&posv)[2], long long (&off)[2]) -> bool {
         bool bad = false;
 #pragma unroll
         for (int jj = 0; jj < 2; ++jj) {
-          const int jt = min(lane + jj * 32, ntok - 1);
-          const int k = t0 + jt;  // token index inside the unit: the list first, then the tail
-          int pos = (k >= c_list) ? (kvlen_b + (k - c_list)) : (P.dense ? k : __ldg(list + k));
+          int pos = posv[jj];
           if (pos < 0 || pos >= kvlen_b + P.tail) { bad = true; pos = 0; }
           int lp = (P.page_shift >= 0) ? (pos >> P.page_shift) : (pos / P.page_size);
           // a position beyond the sequence's row of the block table (kv_len larger than the
@@ -716,9 +723,16 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         }
         return bad;
       };
+      auto resolve = [&](int t0, long long (&off)[2]) -> bool {
+        int pos[2];
+        load_pos(t0, pos);
+        return offs_of(pos, off);
+      };
       long long off_next[2] = {0, 0};
       bool bad_next = false;
       int t0_next = -1;  // tile whose offsets are already resolved
+      int pos_nn[2] = {0, 0};
+      int t0_nn = -1;    // tile whose positions are already loaded
       for (int t0 = tok_lo; t0 < tok_hi; t0 += kStageTok, ++it) {
         if ((it % kProdWarps) != pw) continue;
         const int s = it % kStages;
@@ -765,7 +779,18 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         // before: while the ring still has free slots the two dependent loads would delay
         // them by ~1.3 us), so that a slot's turnaround holds only the copy itself.
         t0_next = t0 + kProdWarps * kStageTok;
-        if (t0_next < tok_hi) bad_next = resolve(t0_next, off_next); else t0_next = -1;
+        if (t0_next < tok_hi) {
+          if (t0_nn != t0_next) load_pos(t0_next, pos_nn);  // (first tile of the segment only)
+          // positions of the tile after next first (independent), then the block-table loads
+          int pos_new[2] = {0, 0};
+          t0_nn = t0_next + kProdWarps * kStageTok;
+          if (t0_nn < tok_hi) load_pos(t0_nn, pos_new); else t0_nn = -1;
+          bad_next = offs_of(pos_nn, off_next);
+          pos_nn[0] = pos_new[0];
+          pos_nn[1] = pos_new[1];
+        } else {
+          t0_next = -1;
+        }
         if (bad && P.status) atomicOr(P.status + b, SPECATTN_ROW_BAD_INDEX);
         last_it = it;
       }
