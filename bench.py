@@ -410,6 +410,8 @@ def verify_micro(dev, reps=10, flags=0, only=""):
     out = {}
     cases = [("dense_b4_ctx131072_q6x32_kv8", 4, 131072, 6, 32, 8, None),
              ("dense_b4_ctx131072_q5x64_kv8", 4, 131072, 5, 64, 8, None),
+             # a dense cache of the size of the long lists below: same units, tiles and partition
+             ("dense_b8_ctx12288_q6x32_kv8", 8, 12288, 6, 32, 8, None),
              ("sparse1245_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, 1245),
              ("sparse12450_b8_ctx32768_q6x32_kv8", 8, 32768, 6, 32, 8, 12450),
              ("sparse1000_b4_ctx131072_q5x64_kv8", 4, 131072, 5, 64, 8, 1000),
