@@ -371,6 +371,29 @@ def topp_sweep(dev, reps=5, families=None, sizes=None, ps=None, n_rows=256):
     return out
 
 
+def overlapped_schedule(step, reps=20):
+    """The step with one selection per used draft layer, all but the first on a second stream
+    under the attention of earlier layers (VerifyStep(overlap_select=True)), on the step's own
+    buffers: microseconds per step beside the default schedule's, and the outputs compared."""
+    import torch
+    from paper_2510_27641_b200.step import VerifyStep
+    ref_out = [o.clone() for o in step.out]
+    a0 = step.verify_args[0]
+    ov = VerifyStep(layer_map=step.layer_map, n_draft_layers=len(step.draft_probs), batch=a0.batch,
+                    n_draft_heads=step.select_args.n_draft_heads, gamma=step.select_args.gamma,
+                    L_stride=step.select_args.L_stride, n_q_heads=a0.n_q_heads, p=step.select_args.p,
+                    kv_pools=step.kv_pools, kv_len=step.kv_len, block_table=step.block_table,
+                    pages_per_seq=a0.block_table_stride, overlap_select=True)
+    ov.load_inputs(step.draft_probs, step.q)
+    ov.run()
+    torch.cuda.synchronize()
+    same = all(torch.equal(a, b) for a, b in zip(ref_out, ov.out))
+    g, n = capture(ov.run)
+    us = time_replays(g, reps, 3)
+    return {"us_per_step": round(us, 1), "launches_per_step": n, "outputs_identical": bool(same),
+            "note": "not the default: the selections' CTAs take SMs from the attention launches"}
+
+
 def select_variants(step, cfg, reps=5):
     """The selection variants of Alg. 2 on the step's own draft rows (separate output buffers):
     device time per launch and mean kept count, beside the default (aggregate, exact)."""
@@ -793,6 +816,7 @@ def main():
 
     if rank == 0:
         extra("select_variants", lambda: select_variants(step, cfg_r))
+        extra("overlapped_selection_schedule", lambda: overlapped_schedule(step))
         extra("layer_batched_upper_bound", lambda: layer_batched(step, cfg_r, si))
     if rank == 0 and not args.no_cpu_baseline:
         smp = OracleSample(cfg_r, si, n_attn_layers=8, pools=pools)

@@ -10,8 +10,8 @@ from typing import Sequence
 
 import torch
 
-from . import (SelectArgs, VerifyArgs, SpecAttnError, VERIFY_LISTS_STABLE, lib, make_select_args, make_verify_args,
-               verify_plan_buffer, verify_plan_many,
+from . import (SelectArgs, VerifyArgs, SpecAttnError, SELECT_FORM_CLUSTER, VERIFY_LISTS_STABLE, lib, make_select_args,
+               make_verify_args, verify_plan, verify_plan_buffer, verify_plan_many,
                verify_step_host, verify_workspace, _stream_ptr)
 
 __all__ = ["VerifyStep"]
@@ -24,7 +24,8 @@ class VerifyStep:
                  block_table: torch.Tensor | None, pages_per_seq: int | None = None,
                  n_groups: int = 1, head_group: Sequence[int] | None = None,
                  idx_stride: int | None = None, sm_scale: float = 0.0, verify_flags: int = 0,
-                 use_plans: bool = True, select_workspace: bool = True, select_form: int = 0, device=None):
+                 use_plans: bool = True, select_workspace: bool = True, select_form: int = 0,
+                 overlap_select: bool = False, device=None):
         dev = device or kv_pools[0].device
         self.layer_map = [int(x) for x in layer_map]
         self.n_layers = len(self.layer_map)
@@ -51,6 +52,18 @@ class VerifyStep:
                 self.draft_probs, kv_len, self.layer_map, p, n_groups=n_groups, head_group=head_group,
                 idx=self.idx, counts=self.counts, row_status=self.row_status, diag=self.diag,
                 workspace=select_workspace, form=select_form)
+        # overlapped schedule: one selection per used draft layer, so that all but the first run
+        # on a second stream under the attention of the layers mapped to earlier draft layers
+        self.overlap = bool(overlap_select) and len(used) > 1
+        self.select_args_u, self._keep_u, self._side, self._events = {}, [], None, {}
+        if self.overlap:
+            for u in used:
+                a_u, keep_u = make_select_args(
+                    self.draft_probs, kv_len, [u], p, n_groups=n_groups, head_group=head_group,
+                    idx=self.idx, counts=self.counts, row_status=self.row_status, diag=self.diag,
+                    workspace=False, form=SELECT_FORM_CLUSTER)
+                self.select_args_u[u] = a_u
+                self._keep_u.append(keep_u)
         self.verify_args: list[VerifyArgs] = []
         self.workspace = None
         self.plans: dict[int, tuple[torch.Tensor, int]] = {}   # draft layer (-1: dense) -> (plan, a layer using it)
@@ -103,8 +116,64 @@ class VerifyStep:
         if rc != 0:
             raise SpecAttnError(rc, "specattn_sparse_verify")
 
+    def _run_overlapped(self, stream=None):
+        """The selection of the first draft layer in use, then, on a second stream, the selections
+        (and work partitions) of the others in the order of their first use, while the first
+        stream runs the attention of the target layers: a layer waits for its draft layer's
+        selection only (Alg. 1: every verifier layer needs the mask of its mapped draft layer)."""
+        main = stream if stream is not None else torch.cuda.current_stream()
+        if self._side is None:
+            self._side = torch.cuda.Stream(device=main.device)
+        L = lib()
+        order = []
+        for u in self.layer_map:
+            if u >= 0 and u not in order:
+                order.append(u)
+
+        def select_and_plan(u, st):
+            rc = L.specattn_select_topp(C.byref(self.select_args_u[u]), _stream_ptr(st))
+            if rc != 0:
+                raise SpecAttnError(rc, "specattn_select_topp")
+            if u in self.plans:
+                plan, j = self.plans[u]
+                verify_plan(self.verify_args[j], plan, st)
+
+        with torch.cuda.stream(main):
+            select_and_plan(order[0], main)
+            if -1 in self.plans:   # the dense layers' partition does not depend on any selection
+                plan, j = self.plans[-1]
+                verify_plan(self.verify_args[j], plan, main)
+            fork = torch.cuda.Event()
+            fork.record(main)
+        ready = {order[0]}
+        events = {}
+        with torch.cuda.stream(self._side):
+            self._side.wait_event(fork)
+            for u in order[1:]:
+                select_and_plan(u, self._side)
+                events[u] = torch.cuda.Event()
+                events[u].record(self._side)
+        with torch.cuda.stream(main):
+            sp = _stream_ptr(main)
+            for j, a in enumerate(self.verify_args):
+                u = self.layer_map[j]
+                flags = a.flags
+                if u >= 0 and u not in ready:
+                    main.wait_event(events[u])
+                    ready.add(u)
+                    a.flags = flags & ~VERIFY_LISTS_STABLE   # lists and plan are new to this launch
+                rc = L.specattn_sparse_verify(C.byref(a), sp)
+                a.flags = flags
+                if rc != 0:
+                    raise SpecAttnError(rc, "specattn_sparse_verify")
+            for u, ev in events.items():   # join (a draft layer whose layers were all visited is already waited for)
+                if u not in ready:
+                    main.wait_event(ev)
+
     def run(self, stream=None):
         """Device-resident step: 1 select launch + n_layers verify launches."""
+        if self.overlap:
+            return self._run_overlapped(stream)
         sp = _stream_ptr(stream)
         L = lib()
         self.run_select(stream)
@@ -122,6 +191,8 @@ class VerifyStep:
     @property
     def launches_per_step(self) -> int:
         n_select = 0
+        if self.overlap:
+            return len(self.select_args_u) + len(self.plans) + self.n_layers
         if self.select_args is not None:
             n_select = 2 if self.select_args.workspace else 1   # aggregation + search, or the cluster form
         return n_select + (len(self.plans) + 7) // 8 + self.n_layers

@@ -12,7 +12,7 @@ from workloads import bf16
 pytestmark = pytest.mark.gpu
 
 
-def _build(cfg, n_groups=1, head_group=None, dense_first=0, layer_map=None):
+def _build(cfg, n_groups=1, head_group=None, dense_first=0, layer_map=None, **step_kw):
     from paper_2510_27641_b200.step import VerifyStep
     si = wl.make_step_inputs(cfg)
     if layer_map is not None:
@@ -32,7 +32,7 @@ def _build(cfg, n_groups=1, head_group=None, dense_first=0, layer_map=None):
     step = VerifyStep(layer_map=si.layer_map.tolist(), n_draft_layers=cfg.n_draft_layers, batch=cfg.batch,
                       n_draft_heads=cfg.n_draft_heads, gamma=cfg.gamma, L_stride=si.L_stride,
                       n_q_heads=cfg.n_q_heads, p=cfg.p, kv_pools=pools, kv_len=kv_len, block_table=bt,
-                      pages_per_seq=si.pages_per_seq, n_groups=n_groups, head_group=head_group)
+                      pages_per_seq=si.pages_per_seq, n_groups=n_groups, head_group=head_group, **step_kw)
     step.load_inputs([None if x is None else torch.from_numpy(x) for x in si.draft_probs],
                      [bf16.bits_to_torch(q) for q in si.q])
     return si, pools, step
@@ -83,6 +83,44 @@ def test_config1_shape_reduced_layers_and_context():
     torch.cuda.synchronize()
     st, worst = _check_step(cfg, si, pools, step, range(5))
     assert st["n"] == len(set(si.layer_map.tolist()) - {-1}) * 3
+
+
+def test_overlapped_selection_schedule_matches_the_oracle_and_the_plain_schedule():
+    """One selection per draft layer, all but the first on a second stream under the attention of
+    earlier layers (a layer waits for its own draft layer's lists only): same lists, same outputs,
+    launched directly and replayed from a CUDA graph; the map visits the draft layers out of order
+    and comes back to one, and starts with a dense layer."""
+    cfg = wl.config1().scaled(n_target_layers=8, n_draft_layers=4, batch=3, ctx=6000)
+    lmap = [2, 2, 0, 3, 0, 2, 3, 3]
+    si, pools, plain = _build(cfg, dense_first=1, layer_map=lmap)
+    plain.run()
+    torch.cuda.synchronize()
+    si2, pools2, step = _build(cfg, dense_first=1, layer_map=lmap, overlap_select=True)
+    assert step.overlap and step.launches_per_step == 3 + len(step.plans) + 8
+    step.run()
+    torch.cuda.synchronize()
+    st, worst = _check_step(cfg, si2, pools2, step, range(8))
+    assert st["n"] == 3 * 3
+
+    def same():
+        used = sorted(set(si.layer_map.tolist()) - {-1})
+        for u in used:
+            assert torch.equal(step.counts[u], plain.counts[u]) and torch.equal(step.idx[u], plain.idx[u])
+        for j in range(8):
+            assert torch.equal(step.out[j], plain.out[j]) and torch.equal(step.lse[j], plain.lse[j])
+        assert int(step.status.abs().sum()) == 0
+    same()
+    # replayed from a graph (the second stream joins the capture and is joined again at the end)
+    for o in step.out:
+        o.fill_(float("nan"))
+    step.counts.fill_(-1)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step.run()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    same()
 
 
 def test_config3_ragged_reduced():
