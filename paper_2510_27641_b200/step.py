@@ -55,7 +55,7 @@ class VerifyStep:
         # overlapped schedule: one selection per used draft layer, so that all but the first run
         # on a second stream under the attention of the layers mapped to earlier draft layers
         self.overlap = bool(overlap_select) and len(used) > 1
-        self.select_args_u, self._keep_u, self._side, self._events = {}, [], None, {}
+        self.select_args_u, self._keep_u, self._side = {}, [], None
         if self.overlap:
             for u in used:
                 a_u, keep_u = make_select_args(
