@@ -1016,33 +1016,63 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           // Merge every contributor's record in CTA order (the own one included, read back
           // from memory, so the result does not depend on who arrived last).  First the
           // common maxima, then one scaled accumulation pass with independent loads.
-          m0 = m1 = -INFINITY;
-          for (int i = i_lo; i <= i_hi; ++i) {
-            const float4* r2 = reinterpret_cast<const float4*>(P.partials +
+          // (the loads of four records' maxima, then of two records' halves, are in flight together:
+          // walking the records one round trip to L2 at a time took 6 - 8 us for four of them)
+          auto record = [&](int i) -> const float4* {
+            return reinterpret_cast<const float4*>(P.partials +
                 (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * MT + mt) * kRec) + lane;
-            const float4 ml = __ldcg(r2 + 16 * 32);
-            m0 = fmaxf(m0, ml.x);
-            m1 = fmaxf(m1, ml.z);
+          };
+          m0 = m1 = -INFINITY;
+          for (int i = i_lo; i <= i_hi; i += 4) {   // four records' maxima per round trip
+            float4 ml[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) ml[j] = __ldcg(record(min(i + j, i_hi)) + 16 * 32);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              m0 = fmaxf(m0, ml[j].x);
+              m1 = fmaxf(m1, ml[j].z);
+            }
           }
           const float base0 = (m0 == -INFINITY) ? 0.f : m0, base1 = (m1 == -INFINITY) ? 0.f : m1;
           l0 = l1 = 0.f;
 #pragma unroll
           for (int n = 0; n < 16; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-          for (int i = i_lo; i <= i_hi; ++i) {
-            const float4* r2 = reinterpret_cast<const float4*>(P.partials +
-                (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * MT + mt) * kRec) + lane;
-            const float4 ml = __ldcg(r2 + 16 * 32);
-            const float w0 = ex2(ml.x - base0);
-            const float w1 = ex2(ml.z - base1);
-            l0 += ml.y * w0;
-            l1 += ml.w * w1;
 #pragma unroll
-            for (int n = 0; n < 16; ++n) {
-              const float4 r = __ldcg(r2 + n * 32);
-              acc[n][0] += r.x * w0;
-              acc[n][1] += r.y * w0;
-              acc[n][2] += r.z * w1;
-              acc[n][3] += r.w * w1;
+          for (int half = 0; half < 2; ++half) {
+            for (int i = i_lo; i <= i_hi; i += 2) {   // two records' half rows per round trip
+              const bool two = i + 1 <= i_hi;
+              const float4* ra = record(i);
+              const float4* rb = record(two ? i + 1 : i);
+              const float4 mla = __ldcg(ra + 16 * 32), mlb = __ldcg(rb + 16 * 32);
+              float4 xa[8], xb[8];
+#pragma unroll
+              for (int n = 0; n < 8; ++n) {
+                xa[n] = __ldcg(ra + (half * 8 + n) * 32);
+                xb[n] = __ldcg(rb + (half * 8 + n) * 32);
+              }
+              const float wa0 = ex2(mla.x - base0), wa1 = ex2(mla.z - base1);
+              const float wb0 = two ? ex2(mlb.x - base0) : 0.f, wb1 = two ? ex2(mlb.z - base1) : 0.f;
+              if (half == 0) {
+                l0 += mla.y * wa0;
+                l1 += mla.w * wa1;
+                if (two) {
+                  l0 += mlb.y * wb0;
+                  l1 += mlb.w * wb1;
+                }
+              }
+#pragma unroll
+              for (int n = 0; n < 8; ++n) {
+                acc[half * 8 + n][0] += xa[n].x * wa0;
+                acc[half * 8 + n][1] += xa[n].y * wa0;
+                acc[half * 8 + n][2] += xa[n].z * wa1;
+                acc[half * 8 + n][3] += xa[n].w * wa1;
+                if (two) {
+                  acc[half * 8 + n][0] += xb[n].x * wb0;
+                  acc[half * 8 + n][1] += xb[n].y * wb0;
+                  acc[half * 8 + n][2] += xb[n].z * wb1;
+                  acc[half * 8 + n][3] += xb[n].w * wb1;
+                }
+              }
             }
           }
           if (lane == 0) P.counters[u * kCountersPerUnit + mt] = 0u;  // ready for the next call
