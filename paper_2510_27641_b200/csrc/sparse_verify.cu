@@ -106,6 +106,10 @@ struct VShared {
   int cand_max[kCandidates];
   int aligned;                           // 1: unit-aligned partition, 0: contiguous atoms
   volatile int abort_flag;
+  // (kernels with two warps per slab) this CTA arrived last at the cut unit of its final segment:
+  // both warps of the slab merge half of the columns each; with the merge's arguments
+  volatile int merge_last[MT];
+  volatile int merge_arg[MT][5];
   // cluster merge (two CTAs per unit): the odd CTA's records land here, in the even CTA
   unsigned long long peer_full;
   alignas(16) float peer_rec[(MT <= 2) ? MT : 1][(MT <= 2) ? kRec : 1];
@@ -427,6 +431,92 @@ __device__ __forceinline__ void attend_block32(WarpState& st, const uint32_t (&q
     mma_bf16(st.acc[2 * j + 1], plo[0], v0[2], v0[3]);
     mma_bf16(st.acc[2 * j], plo[1], v1[0], v1[1]);
     mma_bf16(st.acc[2 * j + 1], plo[1], v1[2], v1[3]);
+  }
+}
+
+// Merge of a unit cut across CTAs by the CTA that arrived last, for one half of the 128 output
+// columns (8 blocks of 8) and one warp: the common maxima of all records (four per round trip),
+// then one scaled accumulation pass in CTA order with two records' half rows in flight, then rows
+// g and g + 8 of slab mt written out (half 0 also writes the LSE).  Used by the kernels with two
+// warps per slab, whose second warp has nothing left to do on a CTA's last segment; kept out of
+// line so that it costs the tile loop no registers.
+template <int MT>
+__device__ __noinline__ void merge_half(const VerifyParams& P, int mt, int half, int i_lo, int i_hi, bool aligned,
+                                        long long N, long long NP, int us, int b, int kvh) {
+  const int lane = threadIdx.x & 31, g = lane >> 2, tq = lane & 3;
+  auto record = [&](int i) -> const float4* {
+    return reinterpret_cast<const float4*>(P.partials +
+        (static_cast<size_t>(2 * i + ((aligned || cta_first_atom(i, N, NP) >= us) ? 0 : 1)) * MT + mt) * kRec) + lane;
+  };
+  float m0 = -INFINITY, m1 = -INFINITY;
+  for (int i = i_lo; i <= i_hi; i += 4) {
+    float4 ml[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) ml[j] = __ldcg(record(min(i + j, i_hi)) + 16 * 32);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      m0 = fmaxf(m0, ml[j].x);
+      m1 = fmaxf(m1, ml[j].z);
+    }
+  }
+  const float base0 = (m0 == -INFINITY) ? 0.f : m0, base1 = (m1 == -INFINITY) ? 0.f : m1;
+  float l0 = 0.f, l1 = 0.f;
+  float o[8][4];
+#pragma unroll
+  for (int n = 0; n < 8; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+  for (int i = i_lo; i <= i_hi; i += 2) {
+    const bool two = i + 1 <= i_hi;
+    const float4* ra = record(i);
+    const float4* rb = record(two ? i + 1 : i);
+    const float4 mla = __ldcg(ra + 16 * 32), mlb = __ldcg(rb + 16 * 32);
+    float4 xa[8], xb[8];
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      xa[n] = __ldcg(ra + (half * 8 + n) * 32);
+      xb[n] = __ldcg(rb + (half * 8 + n) * 32);
+    }
+    const float wa0 = ex2(mla.x - base0), wa1 = ex2(mla.z - base1);
+    const float wb0 = two ? ex2(mlb.x - base0) : 0.f, wb1 = two ? ex2(mlb.z - base1) : 0.f;
+    l0 += mla.y * wa0;
+    l1 += mla.w * wa1;
+    if (two) {
+      l0 += mlb.y * wb0;
+      l1 += mlb.w * wb1;
+    }
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      o[n][0] += xa[n].x * wa0;
+      o[n][1] += xa[n].y * wa0;
+      o[n][2] += xa[n].z * wa1;
+      o[n][3] += xa[n].w * wa1;
+      if (two) {
+        o[n][0] += xb[n].x * wb0;
+        o[n][1] += xb[n].y * wb0;
+        o[n][2] += xb[n].z * wb1;
+        o[n][3] += xb[n].w * wb1;
+      }
+    }
+  }
+  const float inv0 = (l0 > 0.f) ? 1.f / l0 : 0.f;
+  const float inv1 = (l1 > 0.f) ? 1.f / l1 : 0.f;
+  const int r0 = mt * 16 + g, r1 = r0 + 8;
+  if (r0 < P.M) {
+    const int t = r0 / P.grp, h = kvh * P.grp + r0 % P.grp;
+    const long long row = (static_cast<long long>(b) * P.T + t) * P.Hq + h;
+    float* op = P.out + row * kD + tq * 2;
+#pragma unroll
+    for (int n = 0; n < 8; ++n)
+      *reinterpret_cast<float2*>(op + (half * 8 + n) * 8) = make_float2(o[n][0] * inv0, o[n][1] * inv0);
+    if (half == 0 && tq == 0) P.lse[row] = (l0 > 0.f) ? (m0 + log2f(l0)) * kLn2 : -INFINITY;
+  }
+  if (r1 < P.M) {
+    const int t = r1 / P.grp, h = kvh * P.grp + r1 % P.grp;
+    const long long row = (static_cast<long long>(b) * P.T + t) * P.Hq + h;
+    float* op = P.out + row * kD + tq * 2;
+#pragma unroll
+    for (int n = 0; n < 8; ++n)
+      *reinterpret_cast<float2*>(op + (half * 8 + n) * 8) = make_float2(o[n][2] * inv1, o[n][3] * inv1);
+    if (half == 0 && tq == 0) P.lse[row] = (l1 > 0.f) ? (m1 + log2f(l1)) * kLn2 : -INFINITY;
   }
 }
 
@@ -831,6 +921,8 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
   int a = a0, u = u_first;
   bool ok = true;
   bool peer_seen = false;
+  constexpr bool kShareMerge = (WPM == 2);  // the slab's second warp helps with a final merge
+  bool final_global = false;                // the CTA's last segment ends in a merge through global memory
   while (a < a1) {
     const int us = sh.unit_start[u], ue = sh.unit_start[u + 1];
     const int seg_hi = min(a1, ue);
@@ -957,6 +1049,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
     }
     if (sh.abort_flag) { ok = false; break; }
 
+    if (kShareMerge && seg_hi == a1 && !((a == us) && (seg_hi == ue))) final_global = true;
     if (wr == 0) {
       const bool whole = (a == us) && (seg_hi == ue);
       bool finish = whole;
@@ -1010,7 +1103,22 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         unsigned int old = 0;
         if (lane == 0) old = atomicAdd(P.counters + u * kCountersPerUnit + mt, 1u);
         old = __shfl_sync(0xffffffffu, old, 0);
-        if (old == static_cast<unsigned int>(i_hi - i_lo)) {
+        const bool last = old == static_cast<unsigned int>(i_hi - i_lo);
+        if (kShareMerge && seg_hi == a1) {
+          // final segment: the verdict goes to the slab's other warp; the merge follows the loop
+          if (last) {
+            __threadfence();
+            if (lane == 0) {
+              P.counters[u * kCountersPerUnit + mt] = 0u;  // ready for the next call
+              sh.merge_arg[mt][0] = i_lo;
+              sh.merge_arg[mt][1] = i_hi;
+              sh.merge_arg[mt][2] = us;
+              sh.merge_arg[mt][3] = b;
+              sh.merge_arg[mt][4] = kvh;
+            }
+          }
+          if (lane == 0) sh.merge_last[mt] = last ? 1 : 0;
+        } else if (last) {
           finish = true;
           __threadfence();
           // Merge every contributor's record in CTA order (the own one included, read back
@@ -1109,6 +1217,15 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
       ++u;
       while (u < U && sh.unit_start[u + 1] == sh.unit_start[u]) ++u;
     }
+  }
+  if (kShareMerge && final_global && ok) {
+    // the CTA's last segment was one part of a cut unit: if this CTA arrived last there, each of
+    // the slab's two warps merges half of the columns (after the loop: the verdict comes from
+    // the first warp, and nothing of the unit's state is needed any more)
+    named_bar_sync(1 + mt, WPM * 32);
+    if (sh.merge_last[mt])
+      merge_half<MT>(P, mt, wr, sh.merge_arg[mt][0], sh.merge_arg[mt][1], aligned, N, NP, sh.merge_arg[mt][2],
+                     sh.merge_arg[mt][3], sh.merge_arg[mt][4]);
   }
   if (paired && !peer_seen) cluster_wait();
   if (!ok && P.status && lane == 0) atomicOr(P.status, SPECATTN_ROW_TIMEOUT);
