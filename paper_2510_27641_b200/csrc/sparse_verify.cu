@@ -61,6 +61,11 @@ constexpr int kCandidates = 8;         // candidate target shares tried for it
 // there are CTAs to spare: every part costs a record, an arrival and a share of the merge, which
 // on a small call (one short sequence) outweighs the streaming time saved.
 constexpr int kMinPartAtoms = 8;
+// With CTA pairs available (query blocks of up to 32 rows), a unit of up to this many atoms is cut
+// in two rather than in more parts: the pair's merge through shared memory (~1.7 us) beats the
+// merge of three or more records through global memory (~1 us per record) by more than the
+// longer parts cost.
+constexpr int kPairAtoms = 64;
 constexpr size_t kCounterBytes = static_cast<size_t>(kMaxUnits) * kCountersPerUnit * sizeof(unsigned int);
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -88,6 +93,7 @@ struct VerifyParams {
   int tail_off;      // tail - T: query t may see tail tokens j <= t + tail_off
   const int* plan;   // precomputed work partition (specattn_verify_plan) or nullptr
   int test_lose;     // SPECATTN_VERIFY_TEST_LOSE_ARRIVAL: CTA 0 withholds one barrier arrival
+  int pairs;         // the launch runs as CTA pairs (clusters of two)
 };
 
 // WPM = consumer warps per 16-row slab: 4 -> (stage parity, 32-key half), 2 -> (stage parity).
@@ -210,6 +216,7 @@ __device__ __forceinline__ void plan_body(const VerifyParams& P, int* plan, int 
         if (k < 1) k = 1;
         if (k > atoms) k = atoms;
         if (k * kMinPartAtoms > atoms) k = max(1, atoms / kMinPartAtoms);  // no part shorter than that
+        if (P.pairs && k > 2 && atoms <= kPairAtoms) k = 2;  // short unit: two parts merge through shared memory
         atomicAdd(&cand_parts[c], k);
         atomicMax(&cand_max[c], (atoms + k - 1) / k);
       }
@@ -237,6 +244,7 @@ __device__ __forceinline__ void plan_body(const VerifyParams& P, int* plan, int 
           if (k < 1) k = 1;
           if (k > atoms) k = atoms;
         if (k * kMinPartAtoms > atoms) k = max(1, atoms / kMinPartAtoms);  // no part shorter than that
+        if (P.pairs && k > 2 && atoms <= kPairAtoms) k = 2;  // short unit: two parts merge through shared memory
         }
       }
       int v = k;
@@ -643,6 +651,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
         if (k < 1) k = 1;
         if (k > atoms) k = atoms;
         if (k * kMinPartAtoms > atoms) k = max(1, atoms / kMinPartAtoms);  // no part shorter than that
+        if (P.pairs && k > 2 && atoms <= kPairAtoms) k = 2;  // short unit: two parts merge through shared memory
         atomicAdd(&sh.cand_parts[c], k);
         atomicMax(&sh.cand_max[c], (atoms + k - 1) / k);
       }
@@ -672,6 +681,7 @@ sparse_verify_kernel(const __grid_constant__ VerifyParams P) {
           if (k < 1) k = 1;
           if (k > atoms) k = atoms;
         if (k * kMinPartAtoms > atoms) k = max(1, atoms / kMinPartAtoms);  // no part shorter than that
+        if (P.pairs && k > 2 && atoms <= kPairAtoms) k = 2;  // short unit: two parts merge through shared memory
         }
       }
       int v = k;
@@ -1421,6 +1431,7 @@ VerifyParams make_params(const specattn_verify_args& A) {
 
   P.plan = static_cast<const int*>(A.plan);
   P.test_lose = (A.flags & SPECATTN_VERIFY_TEST_LOSE_ARRIVAL) ? 1 : 0;
+  P.pairs = (m_tiles(A) <= 2 && device_sm_count() % 2 == 0) ? 1 : 0;  // as launch() decides
   return P;
 }
 }  // namespace
