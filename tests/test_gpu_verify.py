@@ -94,6 +94,25 @@ def test_long_lists_are_split_across_ctas_and_merged():
     assert torch.equal(out, out2) and torch.equal(lse, lse2)
 
 
+@pytest.mark.parametrize("T,Hq,counts", [
+    (5, 64, [700, 1250, 2100]),      # 40 query rows (two warps per slab): units of 44 - 132 atoms, cut in 2 - 8 parts
+    (6, 32, [1100, 1700, 2600]),     # 24 rows (CTA pairs): units above 64 atoms, cut in three or more parts
+    (6, 32, [300, 640, 1000]),       # 24 rows: units of up to 64 atoms take the pair's path, cut in two
+])
+def test_units_cut_in_few_parts_merge_like_the_oracle(T, Hq, counts):
+    """Short lists on few sequences: every unit is cut into a handful of parts (odd and even
+    numbers of them), merged by the CTA that arrives last -- alone, with the slab's second warp,
+    or through the pair's shared memory, depending on the shape.  Results are the oracle's and do
+    not depend on who arrives last."""
+    case = _make_case(31, 3, T, Hq, 8, 16, [9000, 9000, 9000], counts=[[c] for c in counts])
+    out, lse, status = _run(case)
+    assert int(status.abs().sum()) == 0
+    check_attention(out, lse, *_oracle(case))
+    for _ in range(3):
+        out2, lse2, _ = _run(case)
+        assert torch.equal(out, out2) and torch.equal(lse, lse2)
+
+
 def test_ragged_batch_with_shared_workspace_reuse():
     import paper_2510_27641_b200 as sa
     rng = np.random.default_rng(3)
